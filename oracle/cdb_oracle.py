@@ -337,3 +337,26 @@ def flop_bound(dims, mean_depth, R=None):
     R = dims.R if R is None else R
     f0 = boundary_to_core_flops(dims)
     return (f0 + R) / (f0 + mean_depth)
+
+
+# --------------------------------------------------------------------------- gate-bias calibration
+
+def calibrate_gate_bias(make_oracle, prompts, T, target_mean_depth, iters=40, lo=-10.0, hi=10.0, back_off=0.05):
+    """Bias b of the learned gate for which the free-running mean exit depth of `prompts` is closest
+    to the target.  Mean depth falls as b grows, so b is bracketed by bisection (fixed bracket and
+    iteration count); the bisection ends on a bias at which some token sits exactly on the
+    threshold, so the result backs off by `back_off` to whichever side lands closer to the target.
+    make_oracle(b) must return an Oracle whose gate bias is b.  Returns (b, mean depth at b)."""
+    def mean_depth(b):
+        orc = make_oracle(b)
+        return float(np.mean(np.concatenate([orc.generate(p, T)["depths"] for p in prompts])))
+    for _ in range(iters):
+        mid = 0.5 * (lo + hi)
+        if mean_depth(mid) > target_mean_depth:
+            lo = mid
+        else:
+            hi = mid
+    b_star = 0.5 * (lo + hi)
+    cands = [(abs(mean_depth(b) - target_mean_depth), b) for b in (b_star - back_off, b_star + back_off)]
+    b = min(cands)[1]
+    return b, mean_depth(b)

@@ -1,0 +1,298 @@
+// Paged decode attention for one query per (row, head): softmax(q K^T / sqrt(Dh)) V over positions
+// 0..position of the row's (sequence, layer, slot) pages (Eq. 1: the core reads K^{(r)}_{<t}; the
+// paged pool is the depth-aware cache of section 4.2).
+//
+// Each KV byte is used once per query (MHA, one query per row), i.e. one FMA per element: the
+// kernel is an HBM streamer, not a contraction.  Work is cut into (row, head, split) items of
+// kSplitTokens tokens (16 pages); a split depends only on the row's own context length, so a
+// row's result is independent of the batch it runs in.  Warps fetch items from a counter; a warp
+// streams a page's K tile and V tile ([16][Dh], contiguous) with 16-byte loads, LPT lanes per
+// token, keeps the online-softmax state in registers, and writes an (o, m, l) partial.  A second
+// kernel merges the partials of a row in split order.
+#include "cdb_internal.h"
+
+namespace cdbk {
+
+template <typename T> struct Chunk;
+template <> struct Chunk<float> {
+    static constexpr int EPC = 4;
+    static __device__ __forceinline__ void unpack(const uint4& v, float* f) {
+        f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y); f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+    }
+};
+template <> struct Chunk<__nv_bfloat16> {
+    static constexpr int EPC = 8;
+    static __device__ __forceinline__ void unpack(const uint4& v, float* f) {
+        f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+        f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+        f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
+        f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
+    }
+};
+
+// streaming 16-byte load: read-only path, do not keep in L1
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+struct AttnParams {
+    const void* q;             // [n_rows][H*Dh]
+    KvPool pool;
+    RowsDev rows;
+    int layer;
+    int max_splits;
+    int max_seqs;
+    float scale_log2;          // log2(e) / sqrt(Dh)
+    float* part;               // [(row*H + head)*max_splits + split][Dh + 2]
+    const int32_t* item_start; // [n_rows + 1]
+    int32_t* counter;
+    int32_t* status;
+};
+
+// splits per row -> exclusive scan; zeroes the per-layer work counters.  One CTA.
+__global__ void __launch_bounds__(1024) attn_plan_kernel(RowsDev rows, int32_t* __restrict__ item_start,
+                                                         int32_t* __restrict__ counters, int n_counters) {
+    __shared__ int warp_tot[32];
+    __shared__ int base;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) base = 0;
+    for (int i = threadIdx.x; i < n_counters; i += 1024) counters[i] = 0;
+    __syncthreads();
+    for (int start = 0; start < rows.n_rows; start += 1024) {
+        const int row = start + threadIdx.x;
+        int ns = 0;
+        if (row < rows.n_rows && rows.seq_id[row] >= 0) {
+            const int pos = rows.position[row];
+            ns = pos >= 0 ? (pos + kSplitTokens) / kSplitTokens : 0;       // ceil((pos+1)/split)
+        }
+        int inc = ns;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
+        if (lane == 31) warp_tot[warp] = inc;
+        __syncthreads();
+        if (warp == 0) {
+            int w = warp_tot[lane];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, w, o); if (lane >= o) w += t; }
+            warp_tot[lane] = w;
+        }
+        __syncthreads();
+        if (row < rows.n_rows) item_start[row] = base + (warp ? warp_tot[warp - 1] : 0) + inc - ns;
+        __syncthreads();
+        if (threadIdx.x == 0) base += warp_tot[31];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) item_start[rows.n_rows] = base;
+}
+
+template <typename T, int DH, int LPT, int CPL>
+__global__ void __launch_bounds__(128) attn_split_kernel(AttnParams p) {
+    constexpr int EPC = Chunk<T>::EPC;
+    static_assert(LPT * CPL * EPC == DH, "lane mapping must cover the head dimension");
+    constexpr int TPI = 32 / LPT;               // tokens per warp iteration
+    constexpr int IPP = kPageSize / TPI;        // iterations per page
+    constexpr int CPT = LPT * CPL;              // 16-byte chunks per token
+    const int lane = threadIdx.x & 31;
+    const int g = lane / LPT, c = lane % LPT;
+    const int H = p.pool.H;
+    const int n_rows = p.rows.n_rows;
+    const int total_items = p.item_start[n_rows] * H;
+    const T* pool_base = (const T*)p.pool.base;
+
+    for (;;) {
+        int item = 0;
+        if (lane == 0) item = atomicAdd(p.counter, 1);
+        item = __shfl_sync(0xffffffffu, item, 0);
+        if (item >= total_items) break;
+        const int pair = item / H, head = item % H;
+        int lo = 0, hi = n_rows;                 // last row with item_start[row] <= pair
+        while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (p.item_start[mid] <= pair) lo = mid; else hi = mid; }
+        const int row = lo, split = pair - p.item_start[lo];
+        const int seq = p.rows.seq_id[row];
+        const int slot = p.rows.slot_of(row);
+        const int ctx = p.rows.position[row] + 1;
+        float* part = p.part + ((size_t)(row * H + head) * p.max_splits + split) * (DH + 2);
+        bool ok = seq >= 0 && seq < p.max_seqs && slot >= 0 && slot < p.rows.n_slots && split < p.max_splits;
+        if (!ok) { if (lane == 0) atomicCAS(p.status, 0, kStatusSeq); continue; }
+        const int tok0 = split * kSplitTokens;
+        const int tok1 = min(ctx, tok0 + kSplitTokens);
+        const int32_t* table = p.rows.page_table + ((size_t)seq * p.rows.n_slots + slot) * p.rows.page_table_stride;
+
+        float qf[CPL][EPC];
+        {
+            const uint4* qp = (const uint4*)((const T*)p.q + (size_t)row * H * DH + (size_t)head * DH);
+#pragma unroll
+            for (int j = 0; j < CPL; ++j) {
+                const uint4 v = qp[c + LPT * j];
+                Chunk<T>::unpack(v, qf[j]);
+#pragma unroll
+                for (int e = 0; e < EPC; ++e) qf[j][e] *= p.scale_log2;
+            }
+        }
+        float m = -INFINITY, l = 0.f;
+        float o[CPL][EPC];
+#pragma unroll
+        for (int j = 0; j < CPL; ++j)
+#pragma unroll
+            for (int e = 0; e < EPC; ++e) o[j][e] = 0.f;
+
+        const int page_lo = tok0 / kPageSize, page_hi = (tok1 - 1) / kPageSize;
+        for (int pi = page_lo; pi <= page_hi; ++pi) {
+            const int page = table[pi];
+            if (page < 0 || page >= p.pool.n_phys_pages) { if (lane == 0) atomicCAS(p.status, 0, kStatusPage); continue; }
+            const uint4* kt = (const uint4*)(pool_base + p.pool.tile_offset(p.layer, page, 0, head));
+            const uint4* vt = (const uint4*)(pool_base + p.pool.tile_offset(p.layer, page, 1, head));
+            uint4 kr[IPP][CPL], vr[IPP][CPL];
+#pragma unroll
+            for (int it = 0; it < IPP; ++it)
+#pragma unroll
+                for (int j = 0; j < CPL; ++j) kr[it][j] = ld_stream(kt + (it * TPI + g) * CPT + c + LPT * j);
+#pragma unroll
+            for (int it = 0; it < IPP; ++it)
+#pragma unroll
+                for (int j = 0; j < CPL; ++j) vr[it][j] = ld_stream(vt + (it * TPI + g) * CPT + c + LPT * j);
+
+            float s[IPP];
+            const int tbase = pi * kPageSize + g;
+            float pmax = -INFINITY;
+#pragma unroll
+            for (int it = 0; it < IPP; ++it) {
+                float acc = 0.f;
+#pragma unroll
+                for (int j = 0; j < CPL; ++j) {
+                    float kf[EPC];
+                    Chunk<T>::unpack(kr[it][j], kf);
+#pragma unroll
+                    for (int e = 0; e < EPC; ++e) acc = fmaf(qf[j][e], kf[e], acc);
+                }
+#pragma unroll
+                for (int x = LPT / 2; x > 0; x >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, x);
+                s[it] = (tbase + it * TPI < tok1) ? acc : -INFINITY;
+                pmax = fmaxf(pmax, s[it]);
+            }
+#pragma unroll
+            for (int x = LPT; x < 32; x <<= 1) pmax = fmaxf(pmax, __shfl_xor_sync(0xffffffffu, pmax, x));
+            const float m_new = fmaxf(m, pmax);                 // finite: the page holds >= 1 valid token
+            const float corr = exp2f(m - m_new);                // 0 on the first page (m = -inf)
+            l *= corr;
+#pragma unroll
+            for (int j = 0; j < CPL; ++j)
+#pragma unroll
+                for (int e = 0; e < EPC; ++e) o[j][e] *= corr;
+#pragma unroll
+            for (int it = 0; it < IPP; ++it) {
+                if (tbase + it * TPI < tok1) {                  // skip slots past the context: they may hold anything
+                    const float pr = exp2f(s[it] - m_new);
+                    l += pr;
+#pragma unroll
+                    for (int j = 0; j < CPL; ++j) {
+                        float vf[EPC];
+                        Chunk<T>::unpack(vr[it][j], vf);
+#pragma unroll
+                        for (int e = 0; e < EPC; ++e) o[j][e] = fmaf(pr, vf[e], o[j][e]);
+                    }
+                }
+            }
+            m = m_new;
+        }
+        // lanes of one token group hold identical l; sum l and o over the groups
+#pragma unroll
+        for (int x = LPT; x < 32; x <<= 1) {
+            l += __shfl_xor_sync(0xffffffffu, l, x);
+#pragma unroll
+            for (int j = 0; j < CPL; ++j)
+#pragma unroll
+                for (int e = 0; e < EPC; ++e) o[j][e] += __shfl_xor_sync(0xffffffffu, o[j][e], x);
+        }
+        if (g == 0) {
+#pragma unroll
+            for (int j = 0; j < CPL; ++j)
+#pragma unroll
+                for (int e = 0; e < EPC; ++e) part[(c + LPT * j) * EPC + e] = o[j][e];
+            if (c == 0) { part[DH] = m; part[DH + 1] = l; }
+        }
+    }
+}
+
+// Merge the splits of each (row, head) in split order and round to T.  One warp per (row, head).
+template <typename T, int DH>
+__global__ void __launch_bounds__(128) attn_merge_kernel(AttnParams p, T* __restrict__ out) {
+    const int lane = threadIdx.x & 31;
+    const int H = p.pool.H;
+    const int wid = blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (blockIdx.x == 0 && threadIdx.x == 0) *p.counter = 0;      // the split kernel is done: re-arm its work counter
+    if (wid >= p.rows.n_rows * H) return;
+    const int row = wid / H, head = wid % H;
+    T* o = out + (size_t)row * H * DH + (size_t)head * DH;
+    constexpr int PER = (DH + 31) / 32;
+    const int ns = p.item_start[row + 1] - p.item_start[row];
+    if (p.rows.seq_id[row] < 0 || ns <= 0) {
+#pragma unroll
+        for (int k = 0; k < PER; ++k) if (lane + 32 * k < DH) o[lane + 32 * k] = T(0.f);
+        return;
+    }
+    const float* part = p.part + (size_t)(row * H + head) * p.max_splits * (DH + 2);
+    float M = -INFINITY;
+    for (int s = 0; s < ns; ++s) M = fmaxf(M, part[(size_t)s * (DH + 2) + DH]);
+    float L = 0.f, acc[PER];
+#pragma unroll
+    for (int k = 0; k < PER; ++k) acc[k] = 0.f;
+    for (int s = 0; s < ns; ++s) {
+        const float* ps = part + (size_t)s * (DH + 2);
+        const float w = exp2f(ps[DH] - M);
+        L = fmaf(ps[DH + 1], w, L);
+#pragma unroll
+        for (int k = 0; k < PER; ++k) if (lane + 32 * k < DH) acc[k] = fmaf(ps[lane + 32 * k], w, acc[k]);
+    }
+    const float inv = 1.f / L;
+#pragma unroll
+    for (int k = 0; k < PER; ++k) if (lane + 32 * k < DH) o[lane + 32 * k] = T(acc[k] * inv);
+}
+
+void launch_attention_plan(const cdb* h, const RowsDev& rows, cudaStream_t st) {
+    attn_plan_kernel<<<1, 1024, 0, st>>>(rows, h->attn_item_start, h->attn_counters, h->cfg.L_pre + h->cfg.L_core + h->cfg.L_coda);
+}
+
+template <typename T, int DH, int LPT, int CPL>
+static void launch_attention_t(const cdb* h, const AttnParams& p, void* o, cudaStream_t st) {
+    static int blocks_per_sm = 0;
+    if (blocks_per_sm == 0) {
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, attn_split_kernel<T, DH, LPT, CPL>, 128, 0);
+        if (blocks_per_sm < 1) blocks_per_sm = 1;
+    }
+    int sms = 148;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int max_items = p.rows.n_rows * p.pool.H * p.max_splits;
+    int grid = sms * blocks_per_sm;
+    if ((max_items + 3) / 4 < grid) grid = (max_items + 3) / 4;
+    attn_split_kernel<T, DH, LPT, CPL><<<grid, 128, 0, st>>>(p);
+    const int warps = p.rows.n_rows * p.pool.H;
+    attn_merge_kernel<T, DH><<<(warps + 3) / 4, 128, 0, st>>>(p, (T*)o);
+}
+
+// Requires launch_attention_plan() for the same rows earlier on the stream (once per set of rows).
+void launch_attention(const cdb* h, int layer, const RowsDev& rows, const void* q, void* o, cudaStream_t st) {
+    if (rows.n_rows <= 0) return;
+    AttnParams p;
+    p.q = q; p.pool = h->pool; p.rows = rows; p.layer = layer; p.max_splits = h->max_splits;
+    p.max_seqs = h->cfg.max_seqs;
+    p.scale_log2 = 1.4426950408889634f / sqrtf((float)h->cfg.Dh);
+    p.part = h->attn_part; p.item_start = h->attn_item_start; p.counter = h->attn_counters + layer; p.status = h->status;
+    const int Dh = h->cfg.Dh;
+    if (h->cfg.dtype == CDB_BF16) {
+        if (Dh == 128) launch_attention_t<__nv_bfloat16, 128, 8, 2>(h, p, o, st);
+        else if (Dh == 96) launch_attention_t<__nv_bfloat16, 96, 4, 3>(h, p, o, st);
+        else launch_attention_t<__nv_bfloat16, 64, 8, 1>(h, p, o, st);
+    } else {
+        if (Dh == 128) launch_attention_t<float, 128, 8, 4>(h, p, o, st);
+        else if (Dh == 96) launch_attention_t<float, 96, 8, 3>(h, p, o, st);
+        else launch_attention_t<float, 64, 8, 2>(h, p, o, st);
+    }
+}
+
+}  // namespace cdbk

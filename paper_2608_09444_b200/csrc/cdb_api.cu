@@ -1,0 +1,397 @@
+// C-ABI entry points of libcdb.so: argument checks, handle life cycle, and the launch sequences of
+// the boundary stages, the loop step, the compaction and the prefill.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "cdb_internal.h"
+
+using namespace cdbk;
+
+namespace {
+
+int fail(cdb_t* h, int code, const char* msg) {
+    if (h) snprintf(h->err, sizeof(h->err), "%s", msg);
+    return code;
+}
+
+int fail_cuda(cdb_t* h, cudaError_t e, const char* where) {
+    if (h) snprintf(h->err, sizeof(h->err), "%s: %s", where, cudaGetErrorString(e));
+    return e == cudaErrorMemoryAllocation ? CDB_ERR_NOMEM : CDB_ERR_CUDA;
+}
+
+int check_launch(cdb_t* h, const char* where) {
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? CDB_OK : fail_cuda(h, e, where);
+}
+
+template <typename T> cudaError_t dev_alloc(T** p, size_t count) {
+    *p = nullptr;
+    return cudaMalloc((void**)p, (count ? count : 1) * sizeof(T));
+}
+
+int slot_of_loop(int layout, int r) {
+    if (layout == CDB_KV_DEPTH_INDEXED) return r - 1;
+    if (layout == CDB_KV_FIRST_THEN_SHARED) return (r < 2 ? r : 2) - 1;
+    return 0;
+}
+
+// Host-side descriptor checks; fills the device view.
+int make_rows(cdb_t* h, const cdb_rows_t* rows, RowsDev* out, bool need_depth) {
+    if (!rows) return fail(h, CDB_ERR_ARG, "rows is NULL");
+    if (rows->n_rows < 0 || rows->n_rows > h->cfg.max_rows) return fail(h, CDB_ERR_CAPACITY, "n_rows exceeds max_rows");
+    if (rows->n_rows > 0 && (!rows->seq_id || !rows->position || !rows->page_table))
+        return fail(h, CDB_ERR_ARG, "rows.seq_id / position / page_table must be device pointers");
+    if (need_depth && rows->n_rows > 0 && (!rows->loop_depth || !rows->kv_slot))
+        return fail(h, CDB_ERR_ARG, "rows.loop_depth / kv_slot must be device pointers");
+    if (rows->page_table_stride * kPageSize < 1) return fail(h, CDB_ERR_ARG, "page_table_stride must be positive");
+    out->n_rows = rows->n_rows;
+    out->seq_id = rows->seq_id;
+    out->loop_depth = rows->loop_depth;
+    out->position = rows->position;
+    out->kv_slot = rows->kv_slot;
+    out->forced_exit = rows->forced_exit;
+    out->page_table = rows->page_table;
+    out->page_table_stride = rows->page_table_stride;
+    out->n_slots = h->cfg.n_slots;
+    out->slot_override = -1;
+    return CDB_OK;
+}
+
+size_t wstride(const cdb_t* h, size_t elems) { return elems * h->elem_size; }
+const void* layer_ptr(const cdb_t* h, const void* base, int layer, size_t elems_per_layer) {
+    return (const char*)base + (size_t)layer * wstride(h, elems_per_layer);
+}
+
+// One transformer layer on `x` (fp32 [n_rows, d], updated in place).  Steps A1-A6 of the loop step:
+// RMSNorm + QKV projection, RoPE + KV page write, paged attention, output projection + residual,
+// RMSNorm + gate/up projections + SwiGLU, down projection + residual.
+void layer_forward(cdb_t* h, int layer, const RowsDev& rows, float* x, cudaStream_t st) {
+    const cdb_config_t& c = h->cfg;
+    const int n = rows.n_rows;
+    const size_t d = c.d, F = c.F;
+    launch_rmsnorm(h, x, h->g_attn + (size_t)layer * d, h->xn, rows, st);
+    launch_linear(h, h->xn, layer_ptr(h, h->w.W_qkv, layer, 3 * d * d), h->qkv, n, 3 * c.d, c.d, Epilogue::Store, st);
+    launch_rope_kv_write(h, layer, rows, st);
+    launch_attention(h, layer, rows, h->qrot, h->attn_o, st);
+    launch_linear(h, h->attn_o, layer_ptr(h, h->w.W_o, layer, d * d), x, n, c.d, c.d, Epilogue::ResidualAdd, st);
+    launch_rmsnorm(h, x, h->g_mlp + (size_t)layer * d, h->xn, rows, st);
+    launch_linear(h, h->xn, layer_ptr(h, h->w.W_gate, layer, F * d), h->gu, n, c.F, c.d, Epilogue::Store, st);
+    launch_linear(h, h->xn, layer_ptr(h, h->w.W_up, layer, F * d), h->gu + (size_t)c.max_rows * F, n, c.F, c.d, Epilogue::Store, st);
+    launch_swiglu(h, n, st);
+    launch_linear(h, h->act, layer_ptr(h, h->w.W_down, layer, d * F), x, n, c.d, c.F, Epilogue::ResidualAdd, st);
+}
+
+// final RMSNorm + LM head + greedy argmax on n rows of x
+void lm_head(cdb_t* h, const RowsDev& rows, const float* x, int32_t* token_out, float* logits_out, cudaStream_t st) {
+    const cdb_config_t& c = h->cfg;
+    float* logits = logits_out ? logits_out : h->logits;
+    launch_rmsnorm(h, x, h->g_final, h->xn, rows, st);
+    launch_linear(h, h->xn, h->w.W_lm, logits, rows.n_rows, c.V, c.d, Epilogue::Store, st);
+    launch_argmax(h, logits, rows.n_rows, token_out, st);
+}
+
+void free_all(cdb_t* h) {
+    void* ptrs[] = {h->rope_cos, h->rope_sin, h->g_attn, h->g_mlp, h->g_final, h->gate_S, h->gate_fire, h->xn, h->qrot,
+                    h->attn_o, h->act, h->qkv, h->gu, h->h_prev, h->h_work, h->logits, h->attn_part,
+                    h->attn_item_start, h->attn_counters, h->exit_flag, h->status, h->emit_tmp};
+    for (void* p : ptrs) if (p) cudaFree(p);
+}
+
+template <typename T> __global__ void to_f32_kernel(const T* in, float* out, size_t n) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        out[i] = (float)in[i];
+}
+
+__global__ void init_gate_state_kernel(float* S, uint8_t* fire, int n) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) { S[i] = 1.f; fire[i] = 0; }
+}
+
+void gains_to_f32(const cdb_t* h, const void* src, float* dst, size_t n) {
+    if (h->cfg.dtype == CDB_FP32) to_f32_kernel<float><<<64, 256>>>((const float*)src, dst, n);
+    else to_f32_kernel<__nv_bfloat16><<<64, 256>>>((const __nv_bfloat16*)src, dst, n);
+}
+
+}  // namespace
+
+extern "C" {
+
+int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
+    if (!cfg || !w || !out) return CDB_ERR_ARG;
+    *out = nullptr;
+    const cdb_config_t& c = *cfg;
+    const int L = c.L_pre + c.L_core + c.L_coda;
+    const int want_slots = c.kv_layout == CDB_KV_SHARED ? 1 : c.kv_layout == CDB_KV_DEPTH_INDEXED ? c.R : 2;
+    if (c.V < 1 || c.d < 1 || c.H < 1 || c.F < 1 || c.d != c.H * c.Dh || (c.Dh != 64 && c.Dh != 96 && c.Dh != 128) ||
+        c.L_pre < 0 || c.L_core < 1 || c.L_coda < 0 || c.R < 1 || c.r_min < 1 || c.page_size != kPageSize ||
+        (c.dtype != CDB_FP32 && c.dtype != CDB_BF16) || c.max_rows < 1 || c.max_seqs < 1 || c.max_position < 1 ||
+        c.kv_layout < 0 || c.kv_layout > 2 || c.n_slots != want_slots || c.gate_kind < 0 || c.gate_kind > 2 ||
+        c.d % 8 != 0 || c.F % 8 != 0)
+        return CDB_ERR_ARG;
+    if (!w->W_qkv || !w->W_o || !w->W_gate || !w->W_up || !w->W_down || !w->g_attn || !w->g_mlp || !w->embed ||
+        !w->g_final || !w->W_lm || (c.gate_kind == CDB_GATE_SIGMOID_CDF && !w->w_gate))
+        return CDB_ERR_ARG;
+    cdb_t* h = new (std::nothrow) cdb_t();
+    if (!h) return CDB_ERR_NOMEM;
+    memset(h, 0, sizeof(*h));
+    h->cfg = c;
+    h->w = *w;
+    h->elem_size = c.dtype == CDB_FP32 ? 4 : 2;
+    h->max_splits = (c.max_position + kSplitTokens - 1) / kSplitTokens;
+    h->pool.H = c.H;
+    h->pool.Dh = c.Dh;
+    const size_t R_ = c.max_rows, d = c.d, F = c.F, half = c.Dh / 2;
+    const size_t wide = d > F ? d : F;
+    cudaError_t e = cudaSuccess;
+#define CDB_ALLOC(ptr, type, count) if (e == cudaSuccess) e = dev_alloc<type>((type**)&(ptr), (count))
+    CDB_ALLOC(h->rope_cos, float, (size_t)c.max_position * half);
+    CDB_ALLOC(h->rope_sin, float, (size_t)c.max_position * half);
+    CDB_ALLOC(h->g_attn, float, (size_t)L * d);
+    CDB_ALLOC(h->g_mlp, float, (size_t)L * d);
+    CDB_ALLOC(h->g_final, float, d);
+    CDB_ALLOC(h->gate_S, float, c.max_seqs);
+    CDB_ALLOC(h->gate_fire, uint8_t, c.max_seqs);
+    CDB_ALLOC(h->xn, char, R_ * wide * h->elem_size);
+    CDB_ALLOC(h->qrot, char, R_ * d * h->elem_size);
+    CDB_ALLOC(h->attn_o, char, R_ * d * h->elem_size);
+    CDB_ALLOC(h->act, char, R_ * F * h->elem_size);
+    CDB_ALLOC(h->qkv, float, R_ * 3 * d);
+    CDB_ALLOC(h->gu, float, R_ * 2 * F);
+    CDB_ALLOC(h->h_prev, float, R_ * d);
+    CDB_ALLOC(h->h_work, float, R_ * d);
+    CDB_ALLOC(h->logits, float, R_ * (size_t)c.V);
+    CDB_ALLOC(h->attn_part, float, R_ * c.H * h->max_splits * (size_t)(c.Dh + 2));
+    CDB_ALLOC(h->attn_item_start, int32_t, R_ + 1);
+    CDB_ALLOC(h->attn_counters, int32_t, L);
+    CDB_ALLOC(h->exit_flag, uint8_t, R_);
+    CDB_ALLOC(h->status, int32_t, 1);
+    CDB_ALLOC(h->emit_tmp, int32_t, R_);
+#undef CDB_ALLOC
+    if (e != cudaSuccess) { free_all(h); delete h; cudaGetLastError(); return e == cudaErrorMemoryAllocation ? CDB_ERR_NOMEM : CDB_ERR_CUDA; }
+
+    // RoPE table: angle = position * theta^(-2i/Dh), evaluated in double, stored as fp32
+    {
+        std::vector<float> cs((size_t)c.max_position * half), sn((size_t)c.max_position * half);
+        for (size_t i = 0; i < half; ++i) {
+            const double inv_freq = std::pow((double)c.rope_theta, -2.0 * (double)i / (double)c.Dh);
+            for (int p = 0; p < c.max_position; ++p) {
+                const double a = (double)p * inv_freq;
+                cs[(size_t)p * half + i] = (float)std::cos(a);
+                sn[(size_t)p * half + i] = (float)std::sin(a);
+            }
+        }
+        e = cudaMemcpy(h->rope_cos, cs.data(), cs.size() * sizeof(float), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemcpy(h->rope_sin, sn.data(), sn.size() * sizeof(float), cudaMemcpyHostToDevice);
+    }
+    if (e == cudaSuccess) {
+        gains_to_f32(h, w->g_attn, h->g_attn, (size_t)L * d);
+        gains_to_f32(h, w->g_mlp, h->g_mlp, (size_t)L * d);
+        gains_to_f32(h, w->g_final, h->g_final, d);
+        init_gate_state_kernel<<<(c.max_seqs + 255) / 256, 256>>>(h->gate_S, h->gate_fire, c.max_seqs);
+        cudaMemset(h->status, 0, sizeof(int32_t));
+        cudaMemset(h->attn_counters, 0, sizeof(int32_t) * L);
+        e = cudaDeviceSynchronize();
+    }
+    if (e != cudaSuccess) { free_all(h); delete h; cudaGetLastError(); return CDB_ERR_CUDA; }
+    *out = h;
+    return CDB_OK;
+}
+
+int cdb_destroy(cdb_t* h) {
+    if (!h) return CDB_OK;
+    cudaDeviceSynchronize();
+    free_all(h);
+    delete h;
+    return CDB_OK;
+}
+
+const char* cdb_last_error(const cdb_t* h) { return h ? h->err : "invalid handle"; }
+
+int cdb_kv_bind(cdb_t* h, void* pool_device, size_t bytes, int32_t n_phys_pages) {
+    if (!h) return CDB_ERR_ARG;
+    if (!pool_device || n_phys_pages < 1) return fail(h, CDB_ERR_ARG, "pool is NULL or has no pages");
+    const size_t L = h->cfg.L_pre + h->cfg.L_core + h->cfg.L_coda;
+    const size_t need = L * n_phys_pages * 2 * h->cfg.H * kPageSize * h->cfg.Dh * h->elem_size;
+    if (bytes < need) return fail(h, CDB_ERR_ARG, "pool is smaller than [L][pages][2][H][16][Dh]");
+    if ((uintptr_t)pool_device % 16) return fail(h, CDB_ERR_ARG, "pool must be 16-byte aligned");
+    h->pool.base = pool_device;
+    h->pool.n_phys_pages = n_phys_pages;
+    return CDB_OK;
+}
+
+int cdb_set_gate(cdb_t* h, float b_gate, float q_or_eps) {
+    if (!h) return CDB_ERR_ARG;
+    h->cfg.b_gate = b_gate;
+    h->cfg.q_or_eps = q_or_eps;
+    return CDB_OK;
+}
+
+static int boundary_in(cdb_t* h, const int32_t* token_ids, const cdb_rows_t* rows, float* h_out, void* stream, bool prelude) {
+    if (!h) return CDB_ERR_ARG;
+    RowsDev rd;
+    int rc = make_rows(h, rows, &rd, false);
+    if (rc) return rc;
+    if (rd.n_rows == 0) return CDB_OK;
+    if (!token_ids || !h_out) return fail(h, CDB_ERR_ARG, "token_ids / h_out is NULL");
+    cudaStream_t st = (cudaStream_t)stream;
+    launch_embed(h, token_ids, rd, h_out, true, st);
+    if (prelude && h->cfg.L_pre > 0) {
+        if (!h->pool.base) return fail(h, CDB_ERR_STATE, "no KV pool bound");
+        rd.slot_override = 0;
+        launch_attention_plan(h, rd, st);
+        for (int l = 0; l < h->cfg.L_pre; ++l) layer_forward(h, l, rd, h_out, st);
+    }
+    return check_launch(h, "cdb_boundary_embed/prelude");
+}
+
+int cdb_boundary_embed(cdb_t* h, const int32_t* token_ids, const cdb_rows_t* rows, float* h_out, void* stream) {
+    return boundary_in(h, token_ids, rows, h_out, stream, false);
+}
+
+int cdb_boundary_prelude(cdb_t* h, const int32_t* token_ids, const cdb_rows_t* rows, float* h_out, void* stream) {
+    return boundary_in(h, token_ids, rows, h_out, stream, true);
+}
+
+int cdb_loop_step(cdb_t* h, const cdb_rows_t* rows, float* h_inout, float* gate_val_out, uint8_t* fire_out, void* stream) {
+    if (!h) return CDB_ERR_ARG;
+    RowsDev rd;
+    int rc = make_rows(h, rows, &rd, true);
+    if (rc) return rc;
+    if (rd.n_rows == 0) return CDB_OK;
+    if (!h_inout) return fail(h, CDB_ERR_ARG, "h_inout is NULL");
+    if (!h->pool.base) return fail(h, CDB_ERR_STATE, "no KV pool bound");
+    cudaStream_t st = (cudaStream_t)stream;
+    const cdb_config_t& c = h->cfg;
+    if (c.gate_kind == CDB_GATE_L2_CONVERGENCE)
+        cudaMemcpyAsync(h->h_prev, h_inout, (size_t)rd.n_rows * c.d * sizeof(float), cudaMemcpyDeviceToDevice, st);
+    launch_attention_plan(h, rd, st);
+    for (int l = c.L_pre; l < c.L_pre + c.L_core; ++l) layer_forward(h, l, rd, h_inout, st);
+    launch_gate(h, rd, h_inout, h->h_prev, gate_val_out, fire_out, st);
+    return check_launch(h, "cdb_loop_step");
+}
+
+int cdb_compact(cdb_t* h, const cdb_rows_t* rows, const uint8_t* fire_prev, const float* h_src, int32_t* survivor_idx,
+                int32_t* exit_idx, int32_t* counts, float* h_next, float* h_exit, void* stream) {
+    if (!h) return CDB_ERR_ARG;
+    RowsDev rd;
+    int rc = make_rows(h, rows, &rd, false);
+    if (rc) return rc;
+    if (rd.n_rows > 0 && !rows->loop_depth) return fail(h, CDB_ERR_ARG, "rows.loop_depth is NULL");
+    if (!survivor_idx || !exit_idx || !counts) return fail(h, CDB_ERR_ARG, "index lists / counts are NULL");
+    cudaStream_t st = (cudaStream_t)stream;
+    launch_compact(h, rd, fire_prev, survivor_idx, exit_idx, counts, st);
+    if (h_src) {
+        if (h_next) launch_gather(h, h_src, survivor_idx, counts, rd.n_rows, h_next, st);
+        if (h_exit) launch_gather(h, h_src, exit_idx, counts + 1, rd.n_rows, h_exit, st);
+    }
+    return check_launch(h, "cdb_compact");
+}
+
+int cdb_gather_rows(cdb_t* h, const float* h_src, const int32_t* idx, const int32_t* count_device, int32_t max_count,
+                    float* h_dst, void* stream) {
+    if (!h) return CDB_ERR_ARG;
+    if (max_count < 0 || max_count > h->cfg.max_rows) return fail(h, CDB_ERR_CAPACITY, "max_count exceeds max_rows");
+    if (max_count == 0) return CDB_OK;
+    if (!h_src || !idx || !h_dst) return fail(h, CDB_ERR_ARG, "NULL argument");
+    launch_gather(h, h_src, idx, count_device, max_count, h_dst, (cudaStream_t)stream);
+    return check_launch(h, "cdb_gather_rows");
+}
+
+int cdb_boundary_coda_lmhead(cdb_t* h, const cdb_rows_t* rows, float* h_exit, int32_t* token_out, float* logits_out, void* stream) {
+    if (!h) return CDB_ERR_ARG;
+    RowsDev rd;
+    int rc = make_rows(h, rows, &rd, false);
+    if (rc) return rc;
+    if (rd.n_rows == 0) return CDB_OK;
+    if (!h_exit || !token_out) return fail(h, CDB_ERR_ARG, "h_exit / token_out is NULL");
+    cudaStream_t st = (cudaStream_t)stream;
+    const cdb_config_t& c = h->cfg;
+    if (c.L_coda > 0) {
+        if (!h->pool.base) return fail(h, CDB_ERR_STATE, "no KV pool bound");
+        rd.slot_override = 0;
+        launch_attention_plan(h, rd, st);
+        for (int l = c.L_pre + c.L_core; l < c.L_pre + c.L_core + c.L_coda; ++l) layer_forward(h, l, rd, h_exit, st);
+    }
+    lm_head(h, rd, h_exit, token_out, logits_out, st);
+    return check_launch(h, "cdb_boundary_coda_lmhead");
+}
+
+int cdb_prefill(cdb_t* h, const int32_t* token_ids, const cdb_rows_t* rows, const int32_t* emit_idx, int32_t n_emit,
+                int32_t* token_out, float* logits_out, void* stream) {
+    if (!h) return CDB_ERR_ARG;
+    RowsDev rd;
+    int rc = make_rows(h, rows, &rd, false);
+    if (rc) return rc;
+    if (rd.n_rows == 0) return CDB_OK;
+    if (!token_ids) return fail(h, CDB_ERR_ARG, "token_ids is NULL");
+    if (n_emit < 0 || n_emit > rd.n_rows || (n_emit > 0 && (!emit_idx || !token_out))) return fail(h, CDB_ERR_ARG, "bad emit list");
+    if (!h->pool.base) return fail(h, CDB_ERR_STATE, "no KV pool bound");
+    cudaStream_t st = (cudaStream_t)stream;
+    const cdb_config_t& c = h->cfg;
+    float* x = h->h_work;
+    launch_embed(h, token_ids, rd, x, true, st);
+    launch_attention_plan(h, rd, st);
+    rd.slot_override = 0;
+    for (int l = 0; l < c.L_pre; ++l) layer_forward(h, l, rd, x, st);
+    for (int r = 1; r <= c.R; ++r) {
+        rd.slot_override = slot_of_loop(c.kv_layout, r);
+        for (int l = c.L_pre; l < c.L_pre + c.L_core; ++l) layer_forward(h, l, rd, x, st);
+    }
+    rd.slot_override = 0;
+    for (int l = c.L_pre + c.L_core; l < c.L_pre + c.L_core + c.L_coda; ++l) layer_forward(h, l, rd, x, st);
+    if (n_emit > 0) {
+        // gather the emitting rows to the front of h_prev (free during prefill), then LM head on them
+        launch_gather(h, x, emit_idx, nullptr, n_emit, h->h_prev, st);
+        RowsDev re = rd;
+        re.n_rows = n_emit;
+        re.seq_id = nullptr;
+        lm_head(h, re, h->h_prev, token_out, logits_out, st);
+    }
+    return check_launch(h, "cdb_prefill");
+}
+
+int cdb_kv_copy_on_exit(cdb_t* h, const cdb_rows_t* rows, const int32_t* exit_depth, void* stream) {
+    if (!h) return CDB_ERR_ARG;
+    if (h->cfg.kv_layout != CDB_KV_DEPTH_INDEXED) return fail(h, CDB_ERR_STATE, "copy-on-exit needs the depth-indexed layout");
+    RowsDev rd;
+    int rc = make_rows(h, rows, &rd, false);
+    if (rc) return rc;
+    if (rd.n_rows == 0) return CDB_OK;
+    if (!exit_depth) return fail(h, CDB_ERR_ARG, "exit_depth is NULL");
+    if (!h->pool.base) return fail(h, CDB_ERR_STATE, "no KV pool bound");
+    launch_copy_on_exit(h, rd, exit_depth, (cudaStream_t)stream);
+    return check_launch(h, "cdb_kv_copy_on_exit");
+}
+
+int cdb_paged_attention(cdb_t* h, const cdb_rows_t* rows, int32_t layer, const void* q, void* o, void* stream) {
+    if (!h) return CDB_ERR_ARG;
+    RowsDev rd;
+    int rc = make_rows(h, rows, &rd, false);
+    if (rc) return rc;
+    if (rd.n_rows == 0) return CDB_OK;
+    if (!q || !o) return fail(h, CDB_ERR_ARG, "q / o is NULL");
+    if (layer < 0 || layer >= h->cfg.L_pre + h->cfg.L_core + h->cfg.L_coda) return fail(h, CDB_ERR_RANGE, "layer out of range");
+    if (!h->pool.base) return fail(h, CDB_ERR_STATE, "no KV pool bound");
+    if (!rows->kv_slot) rd.slot_override = 0;
+    launch_attention_plan(h, rd, (cudaStream_t)stream);
+    launch_attention(h, layer, rd, q, o, (cudaStream_t)stream);
+    return check_launch(h, "cdb_paged_attention");
+}
+
+int cdb_linear(cdb_t* h, const void* x, const void* W, float* y, int32_t n, int32_t N, int32_t K, void* stream) {
+    if (!h) return CDB_ERR_ARG;
+    if (!x || !W || !y || n < 0 || N < 1 || K < 1) return fail(h, CDB_ERR_ARG, "bad argument");
+    launch_linear(h, x, W, y, n, N, K, Epilogue::Store, (cudaStream_t)stream);
+    return check_launch(h, "cdb_linear");
+}
+
+int cdb_poll_status(cdb_t* h, int32_t* status_host) {
+    if (!h || !status_host) return CDB_ERR_ARG;
+    const cudaError_t e = cudaMemcpy(status_host, h->status, sizeof(int32_t), cudaMemcpyDeviceToHost);
+    return e == cudaSuccess ? CDB_OK : fail_cuda(h, e, "cdb_poll_status");
+}
+
+}  // extern "C"

@@ -1,0 +1,100 @@
+// Internal declarations shared by the translation units of libcdb.so (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cdb.h"
+
+namespace cdbk {
+
+constexpr int kPageSize = 16;        // tokens per KV page
+constexpr int kSplitTokens = 256;    // attention split length; depends on nothing but the row's own context
+constexpr int kStatusPage = 1, kStatusPosition = 2, kStatusSeq = 3;
+
+enum class Epilogue : int { Store = 0, ResidualAdd = 1 };
+
+// Device view of a row descriptor plus the KV pool, passed by value to kernels.
+struct RowsDev {
+    int32_t n_rows;
+    const int32_t* seq_id;
+    const int32_t* loop_depth;
+    const int32_t* position;
+    const int32_t* kv_slot;
+    const int32_t* forced_exit;
+    const int32_t* page_table;
+    int32_t page_table_stride;
+    int32_t n_slots;
+    int32_t slot_override;   // >= 0: use this KV slot for every row (prelude / coda layers, prefill)
+    __device__ __forceinline__ int slot_of(int row) const { return slot_override >= 0 ? slot_override : kv_slot[row]; }
+};
+
+struct KvPool {
+    void* base;              // [layer][page][2][H][16][Dh]
+    int32_t n_phys_pages;
+    int32_t H, Dh;
+    // element offsets (not bytes)
+    __host__ __device__ size_t tile_elems() const { return (size_t)kPageSize * Dh; }
+    __host__ __device__ size_t tile_offset(int layer, int page, int kv, int head) const {
+        return ((((size_t)layer * n_phys_pages + page) * 2 + kv) * H + head) * tile_elems();
+    }
+};
+
+}  // namespace cdbk
+
+struct cdb {
+    cdb_config_t cfg;
+    cdb_weights_t w;
+    cdbk::KvPool pool;
+    size_t elem_size;               // bytes of the configured dtype
+    int max_splits;                 // ceil(max_position / kSplitTokens)
+
+    // library-owned device memory
+    float* rope_cos;                // [max_position][Dh/2]
+    float* rope_sin;
+    float* g_attn;                  // fp32 copies of the gains [L][d]
+    float* g_mlp;
+    float* g_final;                 // [d]
+    float* gate_S;                  // [max_seqs] survival of the cumulative exit probability
+    uint8_t* gate_fire;             // [max_seqs] stored exit signal
+    void* xn;                       // [max_rows][max(d,F)] normed activations / attention out / MLP act (dtype)
+    void* qrot;                     // [max_rows][d] rotated queries (dtype)
+    void* attn_o;                   // [max_rows][d] attention output (dtype)
+    void* act;                      // [max_rows][F] SwiGLU output (dtype)
+    float* qkv;                     // [max_rows][3d]
+    float* gu;                      // [max_rows][2F]
+    float* h_prev;                  // [max_rows][d] state at step entry (convergence gate)
+    float* h_work;                  // [max_rows][d] prefill working state
+    float* logits;                  // [max_rows][V]
+    float* attn_part;               // [max_rows*H*max_splits][Dh + 2] split partials (o, m, l)
+    int32_t* attn_item_start;       // [max_rows + 1] exclusive scan of splits per row
+    int32_t* attn_counters;         // [L] work-fetch counters
+    uint8_t* exit_flag;             // [max_rows]
+    int32_t* status;                // [1] first out-of-range access seen (0 = clean)
+    int32_t* emit_tmp;              // [max_rows]
+    char err[256];
+};
+
+namespace cdbk {
+
+// ---- launchers (each enqueues on `st`; none synchronises) -----------------------------------
+void launch_rmsnorm(const cdb* h, const float* x, const float* gain, void* out, const RowsDev& rows, cudaStream_t st);
+void launch_rope_kv_write(const cdb* h, int layer, const RowsDev& rows, cudaStream_t st);
+void launch_attention(const cdb* h, int layer, const RowsDev& rows, const void* q, void* o, cudaStream_t st);
+void launch_attention_plan(const cdb* h, const RowsDev& rows, cudaStream_t st);
+void launch_swiglu(const cdb* h, int n_rows, cudaStream_t st);
+void launch_embed(const cdb* h, const int32_t* tokens, const RowsDev& rows, float* out, bool reset_gate, cudaStream_t st);
+void launch_gate(const cdb* h, const RowsDev& rows, const float* x, const float* x_prev, float* gate_val_out,
+                 uint8_t* fire_out, cudaStream_t st);
+void launch_compact(const cdb* h, const RowsDev& rows, const uint8_t* fire_prev, int32_t* survivor_idx,
+                    int32_t* exit_idx, int32_t* counts, cudaStream_t st);
+void launch_gather(const cdb* h, const float* src, const int32_t* idx, const int32_t* count_dev, int max_count,
+                   float* dst, cudaStream_t st);
+void launch_argmax(const cdb* h, const float* logits, int n_rows, int32_t* token_out, cudaStream_t st);
+void launch_copy_on_exit(const cdb* h, const RowsDev& rows, const int32_t* exit_depth, cudaStream_t st);
+
+// y[n,N] (fp32) = / += x[n,K] . W[N,K]^T ; x and W of the handle's dtype.
+void launch_linear(const cdb* h, const void* x, const void* W, float* y, int n, int N, int K, Epilogue ep, cudaStream_t st);
+
+}  // namespace cdbk

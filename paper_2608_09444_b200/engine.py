@@ -1,0 +1,323 @@
+"""Host-side driver of the CDB hot path: the four queues of the paper's section 4.1 (waiting
+requests, tokens awaiting the prelude, recurrent items, exited tokens awaiting the coda), the
+priority rule (coda > prefill up to the KV budget > recurrent step), refill / no-refill / fixed
+depth modes, and page bookkeeping.  It only builds row descriptors and moves index lists; all
+model arithmetic, the exit decision and the compaction run in libcdb.so.
+
+The deterministic tick mode implemented here runs one stage per tick and waits for its result, so
+that per-tick row lists and page tables are reproducible bit for bit.
+"""
+from __future__ import annotations
+
+import dataclasses
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+@dataclasses.dataclass
+class _Seq:
+    sid: int
+    prompt: np.ndarray
+    T: int
+    tokens: list
+    depths: list
+    gates: list
+    cur_gates: list
+    next_input: int = -1
+
+
+class Engine:
+    def __init__(self, dims, weights, *, max_batch: int, max_live: int, max_len: int, n_pages: int,
+                 kv_layout: int = B.KV_SHARED, gate_kind: int = B.GATE_SIGMOID_CDF, q_or_eps: float = 0.5,
+                 r_min: int = 1, lookahead: bool = True, mode: str = "refill", min_coda_batch: int = 1,
+                 max_prefill_rows: int | None = None, flags: int = 0, record_states: bool = False,
+                 record_logits: bool = False, device: str = "cuda:0"):
+        self.dims, self.mode, self.lookahead = dims, mode, lookahead
+        self.max_batch, self.max_live, self.min_coda_batch = max_batch, max_live, min_coda_batch
+        self.dev = torch.device(device)
+        self.max_pages = (max_len + dims.page_size - 1) // dims.page_size
+        max_rows = max(max_batch, max_prefill_rows or max_batch)
+        self.max_rows = max_rows
+        self.cdb = B.Cdb(dims, weights, max_rows=max_rows, max_seqs=max_live, max_position=self.max_pages * dims.page_size,
+                         kv_layout=kv_layout, gate_kind=gate_kind, q_or_eps=q_or_eps, r_min=r_min, flags=flags)
+        self.n_slots = self.cdb.n_slots
+        self.kv_layout = kv_layout
+        dt = torch.float32 if dims.dtype == "fp32" else torch.bfloat16
+        self.pool = torch.zeros((dims.L, n_pages, 2, dims.H, dims.page_size, dims.Dh), dtype=dt, device=self.dev)
+        self.cdb.kv_bind(self.pool)
+        self.n_pages = n_pages
+        self.free_pages = list(range(n_pages - 1, -1, -1))            # pop() hands out the lowest id first
+        self.page_table_host = np.full((max_live * self.n_slots, self.max_pages), -1, dtype=np.int32)
+        self.page_table = torch.from_numpy(self.page_table_host.copy()).to(self.dev)
+        i32 = dict(dtype=torch.int32, device=self.dev)
+        f32 = dict(dtype=torch.float32, device=self.dev)
+        d = dims.d
+        self.h_rec = torch.zeros((max_rows, d), **f32)                # rows of the next recurrent step
+        self.h_tmp = torch.zeros((max_rows, d), **f32)
+        self.h_exit = torch.zeros((max_rows, d), **f32)               # compaction output: exited rows
+        self.cap = max(max_rows, max_live)
+        self.h_coda = torch.zeros((self.cap, d), **f32)               # coda queue rows
+        self.h_ready = torch.zeros((self.cap, d), **f32)              # prelude output awaiting a batch slot
+        self.gate_val = torch.zeros(max_rows, **f32)
+        self.fire = torch.zeros(max_rows, dtype=torch.uint8, device=self.dev)
+        self.surv_idx = torch.zeros(max_rows, **i32)
+        self.exit_idx = torch.zeros(max_rows, **i32)
+        self.counts = torch.zeros(2, **i32)
+        self.tok_out = torch.zeros(max_rows, **i32)
+        self.logits = torch.zeros((max_rows, dims.V), **f32) if record_logits else None
+        self.record_states, self.record_logits = record_states, record_logits
+        self.stats = {"recurrent_steps": 0, "row_steps": 0, "coda_calls": 0, "prefill_calls": 0, "tick_rows": []}
+        self.trace_states = {}                                        # (sid, token index) -> exit state
+        self.trace_logits = {}
+
+    # ------------------------------------------------------------------ descriptor helpers
+    def _rows(self, seq_ids, positions, depths=None, slots=None, forced=None):
+        t = lambda a: torch.tensor(np.asarray(a, dtype=np.int32), dtype=torch.int32, device=self.dev)
+        return B.Rows(t(seq_ids), t(positions), self.page_table,
+                      loop_depth=None if depths is None else t(depths),
+                      kv_slot=None if slots is None else t(slots),
+                      forced_exit=None if forced is None else t(forced))
+
+    def _slot(self, r):
+        if self.kv_layout == B.KV_DEPTH_INDEXED:
+            return r - 1
+        if self.kv_layout == B.KV_FIRST_THEN_SHARED:
+            return min(r, 2) - 1
+        return 0
+
+    def _reserve_pages(self, slot_id: int, n_tokens: int) -> bool:
+        need = (n_tokens + self.dims.page_size - 1) // self.dims.page_size
+        if need * self.n_slots > len(self.free_pages) or need > self.max_pages:
+            return False
+        for s in range(self.n_slots):
+            row = slot_id * self.n_slots + s
+            for j in range(need):
+                self.page_table_host[row, j] = self.free_pages.pop()
+        rows = slice(slot_id * self.n_slots, (slot_id + 1) * self.n_slots)
+        self.page_table[rows].copy_(torch.from_numpy(self.page_table_host[rows]))
+        return True
+
+    def _release_pages(self, slot_id: int):
+        for s in reversed(range(self.n_slots)):
+            row = slot_id * self.n_slots + s
+            used = self.page_table_host[row][self.page_table_host[row] >= 0]
+            for p in reversed(used):
+                self.free_pages.append(int(p))
+            self.page_table_host[row] = -1
+
+    # ------------------------------------------------------------------ generation
+    def generate(self, prompts, T, forced_depths=None, teacher_tokens=None):
+        """prompts: list of int arrays; T: generated tokens per sequence (int or list).  forced_depths[s][j]
+        replays the exit depth of adaptive pass j of sequence s (0 / None = decided by the gate);
+        teacher_tokens[s][j] replaces the token fed back after generated token j (lock-step replay)."""
+        dims, cdb = self.dims, self.cdb
+        n = len(prompts)
+        Ts = [T] * n if np.isscalar(T) else list(T)
+        seqs = [_Seq(i, np.asarray(prompts[i], dtype=np.int32), Ts[i], [], [], [], []) for i in range(n)]
+        waiting = list(range(n))
+        live_slot = {}                       # sid -> live slot id (index into gate state / page table)
+        free_slots = list(range(self.max_live - 1, -1, -1))
+        ready = []                           # [(sid, h row index in h_ready)] awaiting the recurrent batch (FIFO)
+        ready_free = list(range(self.cap - 1, -1, -1))
+        rec = []                             # current recurrent rows: [sid, depth] in row order (h in h_rec)
+        coda_q = []                          # [(sid, depth, row in h_coda)]
+        coda_free = list(range(self.cap - 1, -1, -1))
+        fixed_depth = self.mode == "cb"
+
+        def forced_for(sq):
+            j = len(sq.tokens) - 1           # index of the adaptive pass in flight
+            if fixed_depth:
+                return dims.R
+            if forced_depths is not None and forced_depths[sq.sid] is not None:
+                return int(forced_depths[sq.sid][j])
+            return 0
+
+        def position_of(sq):
+            return len(sq.prompt) + len(sq.tokens) - 1
+
+        def start_tokens(sids):
+            """prelude for the next input token of each sequence -> ready queue"""
+            if not sids:
+                return
+            toks, pos, sl = [], [], []
+            for s in sids:
+                sq = seqs[s]
+                toks.append(sq.next_input)
+                pos.append(position_of(sq))
+                sl.append(live_slot[s])
+            rows = self._rows(sl, pos)
+            tok_t = torch.tensor(toks, dtype=torch.int32, device=self.dev)
+            out = self.h_tmp[:len(sids)]
+            if dims.L_pre > 0:
+                cdb.boundary_prelude(tok_t, rows, out)
+            else:
+                cdb.boundary_embed(tok_t, rows, out)
+            for k, s in enumerate(sids):
+                slot = ready_free.pop()
+                self.h_ready[slot].copy_(out[k])
+                ready.append((s, slot))
+
+        def finish_or_continue(s, token):
+            sq = seqs[s]
+            sq.tokens.append(int(token))
+            if len(sq.tokens) >= sq.T:
+                self._release_pages(live_slot[s])
+                free_slots.append(live_slot.pop(s))
+                return None
+            j = len(sq.tokens) - 1
+            sq.next_input = int(teacher_tokens[s][j]) if teacher_tokens is not None else int(token)
+            return s
+
+        def run_prefill():
+            admitted = []
+            rows_total = 0
+            while waiting and free_slots:
+                s = waiting[0]
+                sq = seqs[s]
+                P = len(sq.prompt)
+                if rows_total + P > self.max_rows:
+                    break
+                slot = free_slots[-1]
+                if not self._reserve_pages(slot, P + sq.T):
+                    break
+                free_slots.pop()
+                waiting.pop(0)
+                live_slot[s] = slot
+                self.stats.setdefault("admissions", []).append(
+                    (s, slot, self.page_table_host[slot * self.n_slots:(slot + 1) * self.n_slots].copy()))
+                admitted.append(s)
+                rows_total += P
+            if not admitted:
+                return False
+            toks = np.concatenate([seqs[s].prompt for s in admitted])
+            sl = np.concatenate([np.full(len(seqs[s].prompt), live_slot[s]) for s in admitted])
+            pos = np.concatenate([np.arange(len(seqs[s].prompt)) for s in admitted])
+            ends = np.cumsum([len(seqs[s].prompt) for s in admitted]) - 1
+            rows = self._rows(sl, pos)
+            emit = torch.tensor(ends, dtype=torch.int32, device=self.dev)
+            tok_t = torch.tensor(toks, dtype=torch.int32, device=self.dev)
+            lg = self.logits[:len(admitted)] if self.record_logits else None
+            cdb.prefill(tok_t, rows, emit, self.tok_out[:len(admitted)], lg)
+            out = self.tok_out[:len(admitted)].cpu().numpy()
+            self.stats["prefill_calls"] += 1
+            cont = []
+            for k, s in enumerate(admitted):
+                if self.record_logits:
+                    self.trace_logits[(s, 0)] = lg[k].cpu().numpy()
+                r = finish_or_continue(s, out[k])
+                if r is not None:
+                    cont.append(r)
+            start_tokens(cont)
+            return True
+
+        def run_coda():
+            items = list(coda_q)
+            coda_q.clear()
+            k = len(items)
+            idx = torch.tensor([it[2] for it in items], dtype=torch.int32, device=self.dev)
+            hin = self.h_tmp[:k]
+            cdb.gather_rows(self.h_coda, idx, None, k, hin)
+            sl = [live_slot[it[0]] for it in items]
+            pos = [position_of(seqs[it[0]]) for it in items]
+            rows = self._rows(sl, pos)
+            if self.record_states:
+                states = hin.cpu().numpy()
+            if self.kv_layout == B.KV_DEPTH_INDEXED:
+                cdb.kv_copy_on_exit(rows, torch.tensor([it[1] for it in items], dtype=torch.int32, device=self.dev))
+            lg = self.logits[:k] if self.record_logits else None
+            cdb.boundary_coda_lmhead(rows, hin, self.tok_out[:k], lg)
+            out = self.tok_out[:k].cpu().numpy()
+            self.stats["coda_calls"] += 1
+            cont = []
+            for j, (s, depth, slot) in enumerate(items):
+                coda_free.append(slot)
+                sq = seqs[s]
+                sq.depths.append(depth)
+                sq.gates.append(sq.cur_gates)
+                sq.cur_gates = []
+                if self.record_states:
+                    self.trace_states[(s, len(sq.tokens))] = states[j]
+                if self.record_logits:
+                    self.trace_logits[(s, len(sq.tokens))] = lg[j].cpu().numpy()
+                r = finish_or_continue(s, out[j])
+                if r is not None:
+                    cont.append(r)
+            start_tokens(cont)
+
+        def run_recurrent(allow_refill):
+            nonlocal rec
+            # survivors are already at the front of h_rec in stable order; append refills (FIFO)
+            while allow_refill and ready and len(rec) < self.max_batch:
+                s, slot = ready.pop(0)
+                self.h_rec[len(rec)].copy_(self.h_ready[slot])
+                ready_free.append(slot)
+                rec.append([s, 1])
+            k = len(rec)
+            if k == 0:
+                return False
+            sl = [live_slot[s] for s, _ in rec]
+            pos = [position_of(seqs[s]) for s, _ in rec]
+            dep = [r for _, r in rec]
+            rows = self._rows(sl, pos, depths=dep, slots=[self._slot(r) for r in dep],
+                              forced=[forced_for(seqs[s]) for s, _ in rec])
+            hx = self.h_rec[:k]
+            if self.lookahead:               # the stored signal is the previous step's: lists before the step
+                cdb.compact(rows, self.surv_idx, self.exit_idx, self.counts)
+                cdb.loop_step(rows, hx, self.gate_val, self.fire)
+                cdb.gather_rows(hx, self.surv_idx, self.counts[0:1], k, self.h_tmp)
+                cdb.gather_rows(hx, self.exit_idx, self.counts[1:2], k, self.h_exit)
+            else:
+                cdb.loop_step(rows, hx, self.gate_val, self.fire)
+                cdb.compact(rows, self.surv_idx, self.exit_idx, self.counts, h_src=hx, h_next=self.h_tmp, h_exit=self.h_exit)
+            cnt = self.counts.cpu().numpy()
+            ns, ne = int(cnt[0]), int(cnt[1])
+            surv = self.surv_idx[:ns].cpu().numpy()
+            ex = self.exit_idx[:ne].cpu().numpy()
+            gv = self.gate_val[:k].cpu().numpy()
+            self.stats["recurrent_steps"] += 1
+            self.stats["row_steps"] += k
+            self.stats["tick_rows"].append([(s, len(seqs[s].tokens), r) for s, r in rec])
+            for i, (s, r) in enumerate(rec):
+                seqs[s].cur_gates.append(float(gv[i]))
+            for j, i in enumerate(ex):
+                s, r = rec[int(i)]
+                slot = coda_free.pop()
+                self.h_coda[slot].copy_(self.h_exit[j])
+                coda_q.append((s, r, slot))
+            self.h_rec, self.h_tmp = self.h_tmp, self.h_rec        # survivors become the front of the next batch
+            rec = [[rec[int(i)][0], rec[int(i)][1] + 1] for i in surv]
+            self.last_lists = (surv.copy(), ex.copy())
+            return True
+
+        while waiting or live_slot:
+            if self.mode == "refill":
+                runnable_other = bool(rec) or bool(ready) or (bool(waiting) and bool(free_slots))
+                if coda_q and (len(coda_q) >= self.min_coda_batch or not runnable_other):
+                    run_coda()
+                elif waiting and free_slots and run_prefill():
+                    pass
+                elif not run_recurrent(True):
+                    if coda_q:
+                        run_coda()
+                    else:
+                        raise RuntimeError("scheduler stalled: KV pool too small for any waiting request")
+            else:                               # no-refill and fixed-depth: prelude, core until empty, coda
+                if not rec and not ready and not coda_q:
+                    if not (waiting and free_slots and run_prefill()):
+                        if not live_slot:
+                            raise RuntimeError("scheduler stalled: KV pool too small for any waiting request")
+                elif rec or ready:
+                    run_recurrent(allow_refill=not rec)
+                    while rec:
+                        run_recurrent(False)
+                else:
+                    run_coda()
+                    while waiting and free_slots and run_prefill():
+                        pass
+        torch.cuda.synchronize(self.dev)
+        return {"tokens": [np.asarray(s.tokens, dtype=np.int32) for s in seqs],
+                "depths": [np.asarray(s.depths, dtype=np.int32) for s in seqs],
+                "gates": [s.gates for s in seqs]}

@@ -1,0 +1,39 @@
+"""The C-ABI library loads and exports every entry point that include/cdb.h declares (no compute)."""
+import ctypes
+import os
+import re
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "cdb.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(cdb_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_entry_point():
+    import __graft_entry__
+    __graft_entry__.build()
+    from paper_2608_09444_b200 import binding
+    names = declared_symbols()
+    assert len(names) >= 16
+    lib = ctypes.CDLL(os.path.join(ROOT, "paper_2608_09444_b200", "libcdb.so"))
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(binding.EXPORTS) == set(names)                     # the binding wraps exactly what the header declares
+
+
+def test_struct_sizes_match_the_header():
+    from paper_2608_09444_b200 import binding
+    assert ctypes.sizeof(binding.Config) == 18 * 4 + 4 * 4 + 4
+    assert ctypes.sizeof(binding.Weights) == 11 * 8
+    assert ctypes.sizeof(binding.RowsStruct) == 4 + 4 + 6 * 8 + 4 + 4     # int, pad, six pointers, int, pad
+
+
+def test_null_handle_is_an_error_not_a_crash():
+    from paper_2608_09444_b200 import binding
+    assert binding.lib.cdb_destroy(None) == 0
+    assert binding.lib.cdb_set_gate(None, 0.0, 0.0) == binding.ERR_ARG
+    assert binding.lib.cdb_poll_status(None, None) == binding.ERR_ARG
+    assert binding.lib.cdb_last_error(None) == b"invalid handle"
