@@ -112,7 +112,7 @@ def test_c1_without_lookahead(oracle_runs):
 
 def test_c1_exits_disabled_equals_fixed_depth(oracle_runs):
     ref = oracle_runs["fixed"]
-    eng, res = run_engine("cb")
+    eng, res = run_engine("cb", gate=False)
     compare(eng, res, ref)
     eng, res = run_engine("refill", gate=False)
     compare(eng, res, ref)
