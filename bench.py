@@ -1,0 +1,241 @@
+"""Benchmark of the CDB hot path: the Ouro-1.4B-shaped single loop-step microbenchmark (256 ragged
+rows, loop depths 1..4, contexts 128..2048, paged KV with 16-token pages, bf16, random init).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl cdb|reference]
+
+Prints one JSON line.  `value` is token-loop-steps/s with inputs resident in HBM; `e2e` is the same
+metric through host buffers; `roofline` is the paged-attention kernel (the step's dominant kernel)
+against the measured HBM copy bandwidth; `cpu_baseline` is the CPU oracle timed on a bounded sample.
+With --impl reference the CPU oracle itself is timed (rank 0 only).  N > 1 runs one replica per
+GPU on its own rows (sequences are independent: no data-path collective), weak scaling.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "token_loop_steps_per_s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples of one GPU while a region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])), mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(wl, row_ids):
+    """Builds the CPU oracle and its inputs for a few rows of the workload (untimed set-up)."""
+    import numpy as np
+    from oracle import cdb_oracle as O
+    from paper_2608_09444_b200 import synth
+    dm = wl.dims
+    core = {k: v[dm.L_pre:dm.L_pre + dm.L_core] if v.dim() >= 2 and v.shape[0] == dm.L else v for k, v in wl.weights.items()}
+    wn = synth.weights_to_numpy({k: core[k] for k in ("W_qkv", "W_o", "W_gate", "W_up", "W_down", "g_attn", "g_mlp", "w_gate", "b_gate")})
+    wn["g_final"] = np.ones(dm.d, dtype=np.float32)
+    only_core = dm.replace(L_pre=0, L_coda=0)
+    orc = O.Oracle(only_core, wn, gate_kind=O.GATE_SIGMOID_CDF, q_or_eps=0.5)
+    items = wl.oracle_inputs(row_ids)
+    for it in items:
+        kv = [O.gather_pages(it["pages"][l], it["table"], it["ctx"]) for l in range(dm.L_pre, dm.L_pre + dm.L_core)]
+        it["K"], it["V"] = [k for k, _ in kv], [v for _, v in kv]
+        del it["pages"]
+    return orc, items
+
+
+def oracle_step(orc, items):
+    t0 = time.perf_counter()
+    for it in items:
+        orc.loop_step_row(it["h"], it["ctx"] - 1, it["depth"], it["K"], it["V"])
+    return time.perf_counter() - t0
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        return len(os.sched_getaffinity(0))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cdb", choices=["cdb", "reference"])
+    ap.add_argument("--rows", type=int, default=256)
+    ap.add_argument("--ctx-lo", type=int, default=128)
+    ap.add_argument("--ctx-hi", type=int, default=2048)
+    ap.add_argument("--layers", type=int, default=0, help="override the core layer count (small ncu captures only)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--simt-gemm", action="store_true", help="run projections on the plain-FMA cross-check kernel")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "cdb" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference" and rank != 0:
+        return 0
+
+    import numpy as np
+    import torch
+    import __graft_entry__
+    if local_rank == 0:
+        __graft_entry__.build()
+    from paper_2608_09444_b200 import synth
+
+    dims = synth.OURO_1P4B if args.layers <= 0 else synth.OURO_1P4B.replace(L_core=args.layers)
+    workload = f"ouro-1.4b-shaped loop step, {args.rows} rows, depth U{{1..{dims.R}}}, context U{{{args.ctx_lo}..{args.ctx_hi}}}, 16-token pages"
+    config = {"workload": workload, "rows": args.rows, "core_layers": dims.L_core, "page_table": "random permutation",
+              "l2": "inputs larger than L2 (each step streams the whole KV pool and all core weights)"}
+
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl" if args.impl == "cdb" else "gloo")
+    torch.cuda.set_device(local_rank)
+    from paper_2608_09444_b200 import binding as B
+    from paper_2608_09444_b200.workloads import LoopStepWorkload
+    wl = LoopStepWorkload(dims, n_rows=args.rows, seed=1 + rank, ctx_lo=args.ctx_lo, ctx_hi=args.ctx_hi,
+                          device=f"cuda:{local_rank}", flags=B.FLAG_SIMT_GEMM if args.simt_gemm else 0)
+    alg = wl.algorithmic()
+    cores = len(os.sched_getaffinity(0))
+
+    if args.impl == "reference":
+        sample_rows = [0, 1]
+        orc, items = oracle_sample(wl, sample_rows)
+        for _ in range(args.warmup):
+            oracle_step(orc, items)
+        t = sum(oracle_step(orc, items) for _ in range(args.steps))
+        value = len(items) * args.steps / t
+        print(json.dumps({"impl": "reference", "metric": METRIC, "value": value, "unit": "token-loop-steps/s",
+                          "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+                          "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True, "scaling": "weak",
+                          "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
+                          "cpu_baseline": {"value": value, "unit": "token-loop-steps/s", "cores": blas_threads(), "kind": "oracle",
+                                           "sample": f"rows {sample_rows} of the workload per step (one loop step each, serial)"},
+                          "e2e": {"value": value, "unit": "token-loop-steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                          "gpu_launches": 0}))
+        return 0
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        ms = torch.tensor([e0.elapsed_time(e1)], device=f"cuda:{local_rank}")
+        if world > 1:
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item())
+
+    for _ in range(args.warmup):
+        wl.step_resident()
+    sampler = ClockSampler(local_rank)
+    wl.cdb.profile_begin(True)
+    if rank == 0:
+        sampler.start()
+    ms = timed(wl.step_resident, args.steps)
+    clocks = sampler.stop() if rank == 0 else {}
+    prof = wl.cdb.profile_read()
+    wl.cdb.profile_begin(False)
+    assert wl.cdb.poll_status() == 0
+    for _ in range(2):
+        wl.step_e2e()
+    ms_e2e = timed(wl.step_e2e, args.steps)
+
+    if rank != 0:
+        return 0
+    peak, peak_kind = measured_peak()
+    ms_step = ms / args.steps
+    att = prof["attention"]
+    att_ms = att["ms"] / max(att["count"], 1)
+    achieved = alg["attention_per_launch"] / (att_ms * 1e-3) / 1e9 if att_ms > 0 else 0.0
+    out = {"metric": METRIC, "value": world * args.rows / (ms_step * 1e-3), "unit": "token-loop-steps/s",
+           "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+           "config": config,
+           "hbm_step": {"algorithmic_bytes": alg["total"], "achieved_gbs": alg["total"] / (ms_step * 1e-3) / 1e9,
+                        "frac_of_measured_copy_peak": alg["total"] / (ms_step * 1e-3) / 1e9 / peak,
+                        "frac_of_nominal_8tbs": alg["total"] / (ms_step * 1e-3) / 1e9 / 8000.0},
+           "roofline": {"kernel": "attn_split_kernel (paged decode attention)", "bound": "hbm", "achieved": achieved,
+                        "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                        "traffic": None, "launches": att["count"], "avg_launch_ms": att_ms,
+                        "algorithmic_bytes_per_launch": alg["attention_per_launch"]},
+           "kernel_time_ms_per_step": {"attention": att["ms"] / args.steps, "projections": prof["linear"]["ms"] / args.steps},
+           "e2e": {"value": world * args.rows / (ms_e2e / args.steps * 1e-3), "unit": "token-loop-steps/s",
+                   "h2d_bytes_per_step": wl.h2d_bytes(), "d2h_bytes_per_step": wl.d2h_bytes()},
+           "gpu_launches": prof["launches"], "clocks": clocks}
+    if args.no_cpu_baseline or world > 1:
+        out["cpu_baseline"] = None
+    else:
+        sample_rows = [0, 1, 2, 3]
+        orc, items = oracle_sample(wl, sample_rows)
+        t = oracle_step(orc, items)
+        out["cpu_baseline"] = {"value": len(items) / t, "unit": "token-loop-steps/s", "cores": blas_threads(), "kind": "oracle",
+                               "sample": f"one loop step of rows {sample_rows} of the workload, serial, {t:.1f} s",
+                               "host_cores": cores}
+    print(json.dumps(out))
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -188,6 +188,19 @@ int cdb_linear(cdb_t* h, const void* x, const void* W, float* y, int32_t n, int3
  * out-of-range page id / position / sequence id a kernel met (the access was skipped). */
 int cdb_poll_status(cdb_t* h, int32_t* status_host);
 
+/* Instrumentation (not an operation of the paper): how many kernels the handle has launched, and
+ * device time of the two heavy kernel classes measured by CUDA events recorded on the launching
+ * stream.  cdb_profile_begin(h, 1) resets the counters and turns event recording on (0: counters
+ * only); cdb_profile_read synchronises the device and fills `out`.  Index 0 = paged-attention
+ * split kernel, 1 = projection kernels. */
+typedef struct {
+    uint64_t launches;          /* kernels launched since cdb_profile_begin */
+    int32_t  count[2];          /* bracketed launches per class */
+    float    ms[2];             /* summed device time per class, milliseconds */
+} cdb_profile_t;
+int cdb_profile_begin(cdb_t* h, int32_t record_events);
+int cdb_profile_read(cdb_t* h, cdb_profile_t* out);
+
 #ifdef __cplusplus
 }
 #endif

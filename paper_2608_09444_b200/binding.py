@@ -25,7 +25,8 @@ FLAG_SIMT_GEMM = 1
 
 EXPORTS = ["cdb_create", "cdb_destroy", "cdb_last_error", "cdb_kv_bind", "cdb_set_gate", "cdb_boundary_embed",
            "cdb_boundary_prelude", "cdb_loop_step", "cdb_compact", "cdb_gather_rows", "cdb_boundary_coda_lmhead",
-           "cdb_prefill", "cdb_kv_copy_on_exit", "cdb_paged_attention", "cdb_linear", "cdb_poll_status"]
+           "cdb_prefill", "cdb_kv_copy_on_exit", "cdb_paged_attention", "cdb_linear", "cdb_poll_status",
+           "cdb_profile_begin", "cdb_profile_read"]
 
 
 class Config(C.Structure):
@@ -47,6 +48,10 @@ class RowsStruct(C.Structure):
                 ("page_table_stride", C.c_int32)]
 
 
+class Profile(C.Structure):
+    _fields_ = [("launches", C.c_uint64), ("count", C.c_int32 * 2), ("ms", C.c_float * 2)]
+
+
 _P = C.c_void_p
 lib.cdb_create.argtypes = [C.POINTER(Config), C.POINTER(Weights), C.POINTER(_P)]
 lib.cdb_destroy.argtypes = [_P]
@@ -65,6 +70,8 @@ lib.cdb_kv_copy_on_exit.argtypes = [_P, C.POINTER(RowsStruct), _P, _P]
 lib.cdb_paged_attention.argtypes = [_P, C.POINTER(RowsStruct), C.c_int32, _P, _P, _P]
 lib.cdb_linear.argtypes = [_P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P]
 lib.cdb_poll_status.argtypes = [_P, C.POINTER(C.c_int32)]
+lib.cdb_profile_begin.argtypes = [_P, C.c_int32]
+lib.cdb_profile_read.argtypes = [_P, C.POINTER(Profile)]
 for _n in EXPORTS:
     if _n != "cdb_last_error":
         getattr(lib, _n).restype = C.c_int
@@ -202,3 +209,12 @@ class Cdb:
         v = C.c_int32(0)
         self._check(lib.cdb_poll_status(self.h, C.byref(v)))
         return v.value
+
+    def profile_begin(self, record_events: bool = True):
+        self._check(lib.cdb_profile_begin(self.h, 1 if record_events else 0))
+
+    def profile_read(self) -> dict:
+        p = Profile()
+        self._check(lib.cdb_profile_read(self.h, C.byref(p)))
+        return {"launches": int(p.launches), "attention": {"count": p.count[0], "ms": p.ms[0]},
+                "linear": {"count": p.count[1], "ms": p.ms[1]}}

@@ -253,6 +253,7 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(AttnParams p, T* __rest
 }
 
 void launch_attention_plan(const cdb* h, const RowsDev& rows, cudaStream_t st) {
+    CDB_LAUNCH(h);
     attn_plan_kernel<<<1, 1024, 0, st>>>(rows, h->attn_item_start, h->attn_counters, h->cfg.L_pre + h->cfg.L_core + h->cfg.L_coda);
 }
 
@@ -270,7 +271,12 @@ static void launch_attention_t(const cdb* h, const AttnParams& p, void* o, cudaS
     const int max_items = p.rows.n_rows * p.pool.H * p.max_splits;
     int grid = sms * blocks_per_sm;
     if ((max_items + 3) / 4 < grid) grid = (max_items + 3) / 4;
-    attn_split_kernel<T, DH, LPT, CPL><<<grid, 128, 0, st>>>(p);
+    {
+        ProfScope ps(h, kProfAttention, st);
+        CDB_LAUNCH(h);
+        attn_split_kernel<T, DH, LPT, CPL><<<grid, 128, 0, st>>>(p);
+    }
+    CDB_LAUNCH(h);
     const int warps = p.rows.n_rows * p.pool.H;
     attn_merge_kernel<T, DH><<<(warps + 3) / 4, 128, 0, st>>>(p, (T*)o);
 }

@@ -23,6 +23,7 @@ int fail_cuda(cdb_t* h, cudaError_t e, const char* where) {
 }
 
 int check_launch(cdb_t* h, const char* where) {
+    if (h->launch_error) { h->launch_error = 0; return fail(h, CDB_ERR_CUDA, "tensor-map encode failed: projection not launched"); }
     const cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? CDB_OK : fail_cuda(h, e, where);
 }
@@ -98,6 +99,12 @@ void free_all(cdb_t* h) {
                     h->attn_o, h->act, h->qkv, h->gu, h->h_prev, h->h_work, h->logits, h->attn_part,
                     h->attn_item_start, h->attn_counters, h->exit_flag, h->status, h->emit_tmp};
     for (void* p : ptrs) if (p) cudaFree(p);
+    if (h->prof_ev) {
+        for (int i = 0; i < 2 * kProfCap; ++i) if (h->prof_ev[i]) cudaEventDestroy(h->prof_ev[i]);
+        delete[] h->prof_ev;
+        delete[] h->prof_cls;
+        h->prof_ev = nullptr;
+    }
 }
 
 template <typename T> __global__ void to_f32_kernel(const T* in, float* out, size_t n) {
@@ -392,6 +399,37 @@ int cdb_poll_status(cdb_t* h, int32_t* status_host) {
     if (!h || !status_host) return CDB_ERR_ARG;
     const cudaError_t e = cudaMemcpy(status_host, h->status, sizeof(int32_t), cudaMemcpyDeviceToHost);
     return e == cudaSuccess ? CDB_OK : fail_cuda(h, e, "cdb_poll_status");
+}
+
+int cdb_profile_begin(cdb_t* h, int32_t record_events) {
+    if (!h) return CDB_ERR_ARG;
+    if (record_events && !h->prof_ev) {
+        h->prof_ev = new (std::nothrow) cudaEvent_t[2 * kProfCap]();
+        h->prof_cls = new (std::nothrow) uint8_t[kProfCap]();
+        if (!h->prof_ev || !h->prof_cls) return fail(h, CDB_ERR_NOMEM, "no memory for profiling events");
+        for (int i = 0; i < 2 * kProfCap; ++i)
+            if (cudaEventCreate(&h->prof_ev[i]) != cudaSuccess) return fail(h, CDB_ERR_CUDA, "cudaEventCreate failed");
+    }
+    h->launches = 0;
+    h->prof_used = 0;
+    h->prof_on = record_events ? 1 : 0;
+    return CDB_OK;
+}
+
+int cdb_profile_read(cdb_t* h, cdb_profile_t* out) {
+    if (!h || !out) return CDB_ERR_ARG;
+    const cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return fail_cuda(h, e, "cdb_profile_read");
+    memset(out, 0, sizeof(*out));
+    out->launches = h->launches;
+    for (int i = 0; i < h->prof_used; ++i) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, h->prof_ev[2 * i], h->prof_ev[2 * i + 1]) != cudaSuccess) continue;
+        const int c = h->prof_cls[i] < kProfClasses ? h->prof_cls[i] : 0;
+        out->count[c] += 1;
+        out->ms[c] += ms;
+    }
+    return CDB_OK;
 }
 
 }  // extern "C"

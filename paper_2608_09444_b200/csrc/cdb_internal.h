@@ -74,7 +74,33 @@ struct cdb {
     int32_t* status;                // [1] first out-of-range access seen (0 = clean)
     int32_t* emit_tmp;              // [max_rows]
     char err[256];
+
+    // instrumentation: kernel launch count, and CUDA-event pairs around the two heavy kernel classes
+    mutable uint64_t launches;
+    mutable int launch_error;       // a launcher could not set up its kernel (tensor-map encode failed)
+    mutable int prof_on, prof_used;
+    cudaEvent_t* prof_ev;           // [2 * kProfCap]
+    uint8_t* prof_cls;              // [kProfCap]
 };
+
+#define CDB_LAUNCH(h) (++(h)->launches)
+
+namespace cdbk {
+constexpr int kProfCap = 8192;
+enum { kProfAttention = 0, kProfLinear = 1, kProfClasses = 2 };
+// Brackets the kernels launched during its lifetime with an event pair when profiling is on.
+struct ProfScope {
+    const cdb* h; cudaStream_t st; int slot;
+    ProfScope(const cdb* h_, int cls, cudaStream_t st_) : h(h_), st(st_), slot(-1) {
+        if (h->prof_on && h->prof_used < kProfCap) {
+            slot = h->prof_used++;
+            h->prof_cls[slot] = (uint8_t)cls;
+            cudaEventRecord(h->prof_ev[2 * slot], st);
+        }
+    }
+    ~ProfScope() { if (slot >= 0) cudaEventRecord(h->prof_ev[2 * slot + 1], st); }
+};
+}  // namespace cdbk
 
 namespace cdbk {
 

@@ -5,7 +5,7 @@
 
 namespace cdbk {
 
-void launch_linear_tc(const cdb* h, const void* x, const void* W, float* y, int n, int N, int K, Epilogue ep, cudaStream_t st);
+bool launch_linear_tc(const cdb* h, const void* x, const void* W, float* y, int n, int N, int K, Epilogue ep, cudaStream_t st);
 bool linear_tc_supported(const cdb* h, int n, int N, int K);
 
 template <typename T> __device__ __forceinline__ float ldf(const T* p);
@@ -75,8 +75,13 @@ static void launch_simt(const void* x, const void* W, float* y, int n, int N, in
 
 void launch_linear(const cdb* h, const void* x, const void* W, float* y, int n, int N, int K, Epilogue ep, cudaStream_t st) {
     if (n <= 0 || N <= 0) return;
+    ProfScope ps(h, kProfLinear, st);
+    CDB_LAUNCH(h);
     if (h->cfg.dtype == CDB_FP32) { launch_simt<float>(x, W, y, n, N, K, ep, st); return; }
-    if (!(h->cfg.flags & CDB_FLAG_SIMT_GEMM) && linear_tc_supported(h, n, N, K)) { launch_linear_tc(h, x, W, y, n, N, K, ep, st); return; }
+    if (!(h->cfg.flags & CDB_FLAG_SIMT_GEMM) && linear_tc_supported(h, n, N, K)) {
+        if (!launch_linear_tc(h, x, W, y, n, N, K, ep, st)) h->launch_error = 1;      // reported by the entry point
+        return;
+    }
     launch_simt<__nv_bfloat16>(x, W, y, n, N, K, ep, st);
 }
 

@@ -1,9 +1,302 @@
-// bf16 tensor-core projections (tcgen05 + TMEM accumulators, operands staged by TMA).
+// bf16 projections on the 5th-generation tensor cores: y[n,N] (fp32) = or += x[n,K] . W[N,K]^T.
+//
+// At the row counts of a loop step (n <= a few hundred) the projections stream the weights: the
+// arithmetic intensity is about n flop per weight byte.  The kernel therefore puts the WEIGHT's
+// output features on the MMA's M axis (128 per tile) and the batch rows on its N axis (one MMA
+// covers up to 256 rows), so that each weight tile is read exactly once and small batches waste no
+// tensor work ("swap-AB").  Per CTA:
+//   warp 0 (one lane)  TMA producer: W tile [128][64] and x tile [BN][64] (128-byte swizzle) into a
+//                      shared-memory ring, completion on mbarriers;
+//   warp 1 (one lane)  issues tcgen05.mma (M=128, N=BN, K=16) into one of two TMEM accumulators,
+//                      releases ring stages and publishes accumulators with tcgen05.commit;
+//   warps 2-5          epilogue: tcgen05.ld their 32-lane quarter of the accumulator and store / add
+//                      it to y (lanes = consecutive features -> coalesced rows of y).
+// CTAs are persistent over (feature tile, row tile) pairs.  Every mbarrier wait is bounded: on
+// expiry the CTA records a status word, lets its outstanding copies land, frees its TMEM and
+// returns.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
 #include "cdb_internal.h"
 
 namespace cdbk {
 
-bool linear_tc_supported(const cdb*, int, int, int) { return false; }
-void launch_linear_tc(const cdb*, const void*, const void*, float*, int, int, int, Epilogue, cudaStream_t) {}
+namespace {
+
+constexpr int BM = 128;            // features per tile (MMA M)
+constexpr int BK = 64;             // bf16 elements per k-block = one 128-byte swizzle span
+constexpr int UMMA_K = 16;
+constexpr int kThreads = 192;
+constexpr long long kWaitCycles = 1500000000LL;     // about a second of SM clocks
+constexpr int kStatusTimeout = 4;
+constexpr int kMaxSmem = 225 * 1024;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    const long long t0 = clock64();
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitCycles) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c_inner, int c_outer) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(c_inner), "r"(c_outer) : "memory");
+}
+
+// K-major operand tile with 128-byte swizzle: rows of 128 bytes, groups of 8 rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);            // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                             // leading-dimension byte offset (unused with swizzle): 1
+    d |= (uint64_t)(1024 >> 4) << 32;                   // stride-dimension byte offset: 8 rows * 128 B
+    d |= (uint64_t)1 << 46;                             // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                             // layout: 128-byte swizzle
+    return d;
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                   "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                   "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                 : "r"(taddr) : "memory");
+}
+
+struct GemmParams {
+    float* y;
+    int n, N, K;
+    int BN;             // rows per tile (MMA N): 64, 128 or 256
+    int stages;
+    int accumulate;     // 1: y += result
+    int32_t* status;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bars[2 * 8 + 4];          // full[stages], empty[stages], acc_full[2], acc_empty[2]
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int S = p.stages, BN = p.BN;
+    const uint32_t w_bytes = BM * BK * 2, x_bytes = (uint32_t)BN * BK * 2, stage_bytes = w_bytes + x_bytes;
+    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;            // swizzled tiles need 1024-byte alignment
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (8 + s); };
+    auto acc_full_bar = [&](int a) { return bar0 + 8u * (16 + a); };
+    auto acc_empty_bar = [&](int a) { return bar0 + 8u * (18 + a); };
+    const uint32_t tmem_cols = 2u * BN < 32u ? 32u : 2u * BN;               // 128, 256 or 512: a power of two
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+
+    const int n_ftiles = (p.N + BM - 1) / BM, n_rtiles = (p.n + BN - 1) / BN;
+    const int n_tiles = n_ftiles * n_rtiles;
+    const int n_kb = (p.K + BK - 1) / BK;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int s = 0; uint32_t ph = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+                const int f0 = (t % n_ftiles) * BM, r0 = (t / n_ftiles) * BN;
+                for (int kb = 0; kb < n_kb; ++kb) {
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abortp)) { ok = false; break; }
+                    mbar_expect_tx(full_bar(s), stage_bytes);
+                    const uint32_t dst = ring + (uint32_t)s * stage_bytes;
+                    tma_load_2d(dst, &map_w, full_bar(s), kb * BK, f0);
+                    tma_load_2d(dst + w_bytes, &map_x, full_bar(s), kb * BK, r0);
+                    if (++s == S) { s = 0; ph ^= 1u; }
+                }
+            }
+            if (!ok || *abortp) {                        // give copies already in flight time to land
+                for (int i = 0; i < 64; ++i) __nanosleep(1000);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, N = BN, M = 128
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            int s = 0; uint32_t ph = 0;
+            int it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
+                const int acc = it & 1;
+                const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
+                if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, abortp)) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                for (int kb = 0; kb < n_kb; ++kb) {
+                    if (!mbar_wait(full_bar(s), ph, abortp)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_addr = ring + (uint32_t)s * stage_bytes;
+                    const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(a_addr + w_bytes);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k)   // advance 32 bytes inside the swizzle span per UMMA_K
+                        umma_bf16(d_tmem, a_desc + (uint64_t)(k * UMMA_K * 2 >> 4), b_desc + (uint64_t)(k * UMMA_K * 2 >> 4),
+                                  idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    umma_commit(empty_bar(s));              // stage is free once these MMAs have read it
+                    if (++s == S) { s = 0; ph ^= 1u; }
+                }
+                if (ok) umma_commit(acc_full_bar(acc));     // accumulator complete
+            }
+        }
+        __syncwarp();
+    } else {
+        const int q = warp & 3;                             // TMEM lane quarter this warp may read
+        int it = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
+            const int acc = it & 1;
+            const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
+            const int f = (t % n_ftiles) * BM + q * 32 + lane, r0 = (t / n_ftiles) * BN;
+            if (!mbar_wait(acc_full_bar(acc), acc_ph, abortp)) { ok = false; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                if (r0 + c0 >= p.n) break;                  // warp-uniform: nothing but padding rows left
+                uint32_t v[32];
+                tmem_ld32(t_addr + (uint32_t)c0, v);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (f < p.N) {
+                    float* dst = p.y + (size_t)(r0 + c0) * p.N + f;
+                    if (p.accumulate) {
+                        float prev[32];                      // all residual loads in flight before the first add
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) prev[j] = (r0 + c0 + j < p.n) ? __ldcg(dst + (size_t)j * p.N) : 0.f;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (r0 + c0 + j < p.n) dst[(size_t)j * p.N] = prev[j] + __uint_as_float(v[j]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (r0 + c0 + j < p.n) dst[(size_t)j * p.N] = __uint_as_float(v[j]);
+                    }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+        }
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag) atomicCAS(p.status, 0, kStatusTimeout);
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
+PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
+    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &p, 12000, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (PFN_cuTensorMapEncodeTiled_v12000)p;
+    }
+    return fn;
+}
+
+// 2-D bf16 row-major [rows][cols] tensor, box [box_rows][64 columns], 128-byte swizzle, zero fill outside.
+bool make_map(CUtensorMap* m, const void* base, int rows, int cols, int box_rows) {
+    auto fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool linear_tc_supported(const cdb* h, int n, int N, int K) {
+    (void)h;
+    return n >= 1 && N >= 1 && K % 8 == 0 && encode_fn() != nullptr;
+}
+
+bool launch_linear_tc(const cdb* h, const void* x, const void* W, float* y, int n, int N, int K, Epilogue ep, cudaStream_t st) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        attr_set = true;
+    }
+    GemmParams p;
+    p.y = y; p.n = n; p.N = N; p.K = K;
+    p.BN = n <= 64 ? 64 : n <= 128 ? 128 : 256;
+    const int stage_bytes = BM * BK * 2 + p.BN * BK * 2;
+    p.stages = (kMaxSmem - 1024) / stage_bytes;
+    if (p.stages > 8) p.stages = 8;
+    p.accumulate = ep == Epilogue::ResidualAdd ? 1 : 0;
+    p.status = h->status;
+    CUtensorMap map_w, map_x;
+    if (!make_map(&map_w, W, N, K, BM) || !make_map(&map_x, x, n, K, p.BN)) return false;
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int n_tiles = ((N + BM - 1) / BM) * ((n + p.BN - 1) / p.BN);
+    const int grid = n_tiles < sms ? n_tiles : sms;
+    const size_t smem = (size_t)p.stages * stage_bytes + 1024;
+    gemm_bf16_tcgen05_kernel<<<grid, kThreads, smem, st>>>(map_w, map_x, p);
+    return true;
+}
 
 }  // namespace cdbk

@@ -53,6 +53,7 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ 
 }
 
 void launch_rmsnorm(const cdb* h, const float* x, const float* gain, void* out, const RowsDev& rows, cudaStream_t st) {
+    CDB_LAUNCH(h);
     if (rows.n_rows <= 0) return;
     if (h->cfg.dtype == CDB_FP32)
         rmsnorm_kernel<float><<<rows.n_rows, 256, 0, st>>>(x, gain, (float*)out, rows.seq_id, h->cfg.d, h->cfg.eps);
@@ -99,6 +100,7 @@ __global__ void __launch_bounds__(256) rope_kv_write_kernel(const float* __restr
 }
 
 void launch_rope_kv_write(const cdb* h, int layer, const RowsDev& rows, cudaStream_t st) {
+    CDB_LAUNCH(h);
     if (rows.n_rows <= 0) return;
     if (h->cfg.dtype == CDB_FP32)
         rope_kv_write_kernel<float><<<rows.n_rows, 256, 0, st>>>(h->qkv, (float*)h->qrot, h->pool, rows, layer,
@@ -119,6 +121,7 @@ __global__ void swiglu_kernel(const float* __restrict__ g, const float* __restri
 }
 
 void launch_swiglu(const cdb* h, int n_rows, cudaStream_t st) {
+    CDB_LAUNCH(h);
     if (n_rows <= 0) return;
     const size_t n = (size_t)n_rows * h->cfg.F;
     const int blocks = (int)((n + 255) / 256 < 148 * 8 ? (n + 255) / 256 : 148 * 8);
@@ -149,6 +152,7 @@ __global__ void __launch_bounds__(256) embed_kernel(const T* __restrict__ table,
 }
 
 void launch_embed(const cdb* h, const int32_t* tokens, const RowsDev& rows, float* out, bool reset_gate, cudaStream_t st) {
+    CDB_LAUNCH(h);
     if (rows.n_rows <= 0) return;
     if (h->cfg.dtype == CDB_FP32)
         embed_kernel<float><<<rows.n_rows, 256, 0, st>>>((const float*)h->w.embed, tokens, rows.seq_id, out, h->cfg.d,
@@ -204,6 +208,7 @@ __global__ void __launch_bounds__(256) gate_kernel(const float* __restrict__ x, 
 
 void launch_gate(const cdb* h, const RowsDev& rows, const float* x, const float* x_prev, float* gate_val_out,
                  uint8_t* fire_out, cudaStream_t st) {
+    CDB_LAUNCH(h);
     if (rows.n_rows <= 0) return;
     gate_kernel<<<rows.n_rows, 256, 0, st>>>(x, x_prev, h->w.w_gate, rows, h->cfg.d, h->cfg.gate_kind, h->cfg.eps,
                                              h->cfg.b_gate, h->cfg.q_or_eps, h->cfg.max_seqs, h->gate_S, h->gate_fire,
@@ -269,6 +274,7 @@ __global__ void __launch_bounds__(1024) compact_kernel(RowsDev rows, const uint8
 
 void launch_compact(const cdb* h, const RowsDev& rows, const uint8_t* fire_prev, int32_t* survivor_idx,
                     int32_t* exit_idx, int32_t* counts, cudaStream_t st) {
+    CDB_LAUNCH(h);
     compact_kernel<<<1, 1024, 0, st>>>(rows, fire_prev, h->gate_fire, h->cfg.R, h->cfg.r_min, h->cfg.max_seqs,
                                        survivor_idx, exit_idx, counts, h->exit_flag);
 }
@@ -287,6 +293,7 @@ __global__ void __launch_bounds__(256) gather_kernel(const float* __restrict__ s
 
 void launch_gather(const cdb* h, const float* src, const int32_t* idx, const int32_t* count_dev, int max_count,
                    float* dst, cudaStream_t st) {
+    CDB_LAUNCH(h);
     if (max_count <= 0) return;
     gather_kernel<<<max_count, 256, 0, st>>>(src, idx, count_dev, max_count, dst, h->cfg.d);
 }
@@ -317,6 +324,7 @@ __global__ void __launch_bounds__(256) argmax_kernel(const float* __restrict__ l
 }
 
 void launch_argmax(const cdb* h, const float* logits, int n_rows, int32_t* token_out, cudaStream_t st) {
+    CDB_LAUNCH(h);
     if (n_rows <= 0) return;
     argmax_kernel<<<n_rows, 256, 0, st>>>(logits, h->cfg.V, token_out);
 }
@@ -349,6 +357,7 @@ __global__ void __launch_bounds__(256) copy_on_exit_kernel(KvPool pool, RowsDev 
 }
 
 void launch_copy_on_exit(const cdb* h, const RowsDev& rows, const int32_t* exit_depth, cudaStream_t st) {
+    CDB_LAUNCH(h);
     if (rows.n_rows <= 0 || h->cfg.L_core <= 0) return;
     dim3 grid(rows.n_rows, h->cfg.L_core);
     if (h->cfg.dtype == CDB_FP32)

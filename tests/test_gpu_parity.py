@@ -138,7 +138,8 @@ def test_paged_attention_is_page_permutation_invariant():
 # ------------------------------------------------------------------ projections
 
 @pytest.mark.parametrize("dtype,n,N,K", [("fp32", 5, 688, 256), ("fp32", 70, 130, 688), ("bf16", 33, 264, 256),
-                                          ("bf16", 256, 512, 2048), ("bf16", 1, 96, 64)])
+                                          ("bf16", 256, 512, 2048), ("bf16", 1, 96, 64), ("bf16", 300, 1000, 200),
+                                          ("bf16", 100, 6144, 2048), ("bf16", 515, 2048, 5632)])
 def test_linear_matches_matmul(dtype, n, N, K):
     binding = B()
     dims = synth.Dims(V=32, d=128, H=2, Dh=64, F=64, L_pre=0, L_core=1, L_coda=0, R=2, dtype=dtype)
