@@ -14,6 +14,8 @@
 // CTAs are persistent over (feature tile, row tile) pairs.  Every mbarrier wait is bounded: on
 // expiry the CTA records a status word, lets its outstanding copies land, frees its TMEM and
 // returns.
+#include <cstdlib>
+
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
@@ -281,7 +283,20 @@ bool launch_linear_tc(const cdb* h, const void* x, const void* W, float* y, int 
     }
     GemmParams p;
     p.y = y; p.n = n; p.N = N; p.K = K;
-    p.BN = n <= 64 ? 64 : n <= 128 ? 128 : 256;
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    // Rows per tile: as wide as possible (fewest re-reads of W through L2) while there are still about
+    // as many tiles as SMs; a narrower tile only helps when the wide one would leave SMs idle.
+    const int n_ft = (N + BM - 1) / BM;
+    static const int forced_bn = getenv("CDB_GEMM_BN") ? atoi(getenv("CDB_GEMM_BN")) : 0;     // tuning aid
+    p.BN = 64;
+    for (int bn = 256; bn >= 64; bn >>= 1) {
+        if (bn / 2 >= n && bn > 64) continue;                       // tile wider than needed for n rows
+        const int tiles = n_ft * ((n + bn - 1) / bn);
+        if (tiles >= sms / 2 + sms / 8 || bn == 64) { p.BN = bn; break; }
+    }
+    if (forced_bn == 64 || forced_bn == 128 || forced_bn == 256) p.BN = forced_bn;
     const int stage_bytes = BM * BK * 2 + p.BN * BK * 2;
     p.stages = (kMaxSmem - 1024) / stage_bytes;
     if (p.stages > 8) p.stages = 8;
@@ -289,9 +304,6 @@ bool launch_linear_tc(const cdb* h, const void* x, const void* W, float* y, int 
     p.status = h->status;
     CUtensorMap map_w, map_x;
     if (!make_map(&map_w, W, N, K, BM) || !make_map(&map_x, x, n, K, p.BN)) return false;
-    int sms = 148, dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int n_tiles = ((N + BM - 1) / BM) * ((n + p.BN - 1) / p.BN);
     const int grid = n_tiles < sms ? n_tiles : sms;
     const size_t smem = (size_t)p.stages * stage_bytes + 1024;
