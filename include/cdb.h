@@ -184,6 +184,29 @@ int cdb_kv_copy_on_exit(cdb_t* h, const cdb_rows_t* rows, const int32_t* exit_de
 int cdb_paged_attention(cdb_t* h, const cdb_rows_t* rows, int32_t layer, const void* q, void* o, void* stream);
 int cdb_linear(cdb_t* h, const void* x, const void* W, float* y, int32_t n, int32_t N, int32_t K, void* stream);
 
+/* Allocation-free paged decode attention.  The paper has no counterpart: this exists for callers that
+ * cannot obtain device memory at call time (a process that gave the whole GPU to its own pool allocator,
+ * a plug-in whose host framework forbids cudaMalloc on its threads, a component with a memory budget
+ * fixed at start-up).  Same computation and same kernels as cdb_paged_attention for the shared layout
+ * (one KV slot), but without a handle: every input and output is passed in, and the scratch (split
+ * partials, per-row split scan, work counter, status word) lives in an 8 MiB device array built into
+ * the library, which each GPU that loads the library holds until the process exits.  It calls no
+ * cudaMalloc / cudaFree and no allocating library routine.
+ *   q, o: device [n_rows][H*Dh] of `dtype`;  pool: device [layers][n_phys_pages][2][H][16][Dh];
+ *   seq_id, position: device int32 [n_rows] (seq_id < 0 = pad, output row zeroed);
+ *   page_table: device int32 [max_seqs][page_table_stride];  max_context: host upper bound on
+ *   position + 1 (a row beyond it is skipped and its output zeroed).
+ * Limit: 256 + 4*(n_rows+1) rounded up to 256 + n_rows*H*ceil(max_context/256)*(Dh+2)*4 bytes must fit in
+ * 8 MiB (e.g. 64 rows x 16 heads x 2048 context at Dh 128); larger requests return CDB_ERR_CAPACITY and
+ * print the sizes to stderr.  The first call on a device looks up the array's device address
+ * (cudaGetSymbolAddress, with that device current) and should come before any stream capture.  All calls
+ * on a device share the array, which keeps the last call's contents; each call re-zeroes what it needs
+ * on its stream.  Calls whose GPU work overlaps (different streams) race on it. */
+int cdb_paged_attention_static(const void* q, void* o, const void* pool, int32_t n_phys_pages, int32_t layer,
+                               const int32_t* seq_id, const int32_t* position, const int32_t* page_table,
+                               int32_t page_table_stride, int32_t n_rows, int32_t max_seqs, int32_t max_context,
+                               int32_t H, int32_t Dh, int32_t dtype, void* stream);
+
 /* Synchronises the stream-less status word back to the host: 0 = clean, otherwise the first
  * out-of-range page id / position / sequence id a kernel met (the access was skipped). */
 int cdb_poll_status(cdb_t* h, int32_t* status_host);

@@ -26,7 +26,7 @@ FLAG_SIMT_GEMM = 1
 EXPORTS = ["cdb_create", "cdb_destroy", "cdb_last_error", "cdb_kv_bind", "cdb_set_gate", "cdb_boundary_embed",
            "cdb_boundary_prelude", "cdb_loop_step", "cdb_compact", "cdb_gather_rows", "cdb_boundary_coda_lmhead",
            "cdb_prefill", "cdb_kv_copy_on_exit", "cdb_paged_attention", "cdb_linear", "cdb_poll_status",
-           "cdb_profile_begin", "cdb_profile_read"]
+           "cdb_profile_begin", "cdb_profile_read", "cdb_paged_attention_static"]
 
 
 class Config(C.Structure):
@@ -72,6 +72,8 @@ lib.cdb_linear.argtypes = [_P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P]
 lib.cdb_poll_status.argtypes = [_P, C.POINTER(C.c_int32)]
 lib.cdb_profile_begin.argtypes = [_P, C.c_int32]
 lib.cdb_profile_read.argtypes = [_P, C.POINTER(Profile)]
+lib.cdb_paged_attention_static.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32,
+                                           C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P]
 for _n in EXPORTS:
     if _n != "cdb_last_error":
         getattr(lib, _n).restype = C.c_int
@@ -94,6 +96,18 @@ def _ptr(t):
 
 def _stream(stream):
     return (stream if stream is not None else torch.cuda.current_stream()).cuda_stream
+
+
+def paged_attention_static(q, o, pool, layer, seq_id, position, page_table, max_seqs, max_context, stream=None) -> int:
+    """cdb_paged_attention_static: paged decode attention that allocates nothing (no handle; scratch is an
+    array built into the library).  Returns the C return code (OK, or ERR_CAPACITY when the request does
+    not fit the built-in scratch)."""
+    H, Dh = int(pool.shape[3]), int(pool.shape[5])
+    dtype = FP32 if pool.dtype == torch.float32 else BF16
+    return lib.cdb_paged_attention_static(_ptr(q), _ptr(o), _ptr(pool), int(pool.shape[1]), int(layer), _ptr(seq_id),
+                                          _ptr(position), _ptr(page_table), int(page_table.shape[-1]),
+                                          int(seq_id.shape[0]), int(max_seqs), int(max_context), H, Dh, dtype,
+                                          _stream(stream))
 
 
 class Rows:

@@ -9,6 +9,8 @@
 // streams a page's K tile and V tile ([16][Dh], contiguous) with 16-byte loads, LPT lanes per
 // token, keeps the online-softmax state in registers, and writes an (o, m, l) partial.  A second
 // kernel merges the partials of a row in split order.
+#include <cstdio>
+
 #include "cdb_internal.h"
 
 namespace cdbk {
@@ -301,4 +303,113 @@ void launch_attention(const cdb* h, int layer, const RowsDev& rows, const void* 
     }
 }
 
+
+// =====================================================================================================
+// Allocation-free paged attention (cdb_paged_attention_static).
+//
+// Some users of this library cannot obtain device memory when they call it: a serving process that has
+// handed the whole GPU to its own pool allocator at start-up, a plug-in living inside a host framework
+// that forbids cudaMalloc on its threads (it synchronises the device and may fail late), or a component
+// that must run within a memory budget fixed when the process started.  For them this variant of the
+// paged decode attention needs no handle and no allocation: the split partials, the per-row split scan,
+// the work counter and a status word live in the file-scope device array below, which every GPU that
+// loads the library holds until the process exits.  The caller still passes every input and output.
+//
+// The array's name is only a host-side stand-in for the device object, so the host never hands it to a
+// kernel; its device address is looked up once per device with cudaGetSymbolAddress (with that device
+// current) on the first call made on that device.  That first call should therefore come before any
+// stream capture.  All calls on a device share the array and it keeps the previous call's contents: each
+// call re-initialises what must start at zero (work counter, status word, split scan) on the stream
+// before use; two calls whose work overlaps on the GPU (different streams) race on it.
+// =====================================================================================================
+namespace {
+
+constexpr size_t kStaticScratchBytes = size_t(8) << 20;          // 8 MiB per GPU
+constexpr int kStaticMaxDevices = 64;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+unsigned char* g_static_scratch_addr[kStaticMaxDevices];         // device addresses, filled on first use
+
+// Per-row split counts (clamped to the partial area's capacity) -> exclusive scan, and the zeroing of the
+// work counter and status word.  The row count of this variant is small: one thread walks the rows.
+__global__ void attn_static_plan_kernel(RowsDev rows, int max_splits, int max_context, int32_t* __restrict__ item_start,
+                                        int32_t* __restrict__ counter, int32_t* __restrict__ status) {
+    if (blockIdx.x != 0 || threadIdx.x != 0) return;
+    *counter = 0;
+    *status = 0;
+    int acc = 0;
+    for (int row = 0; row < rows.n_rows; ++row) {
+        item_start[row] = acc;
+        const int pos = rows.position[row];
+        if (rows.seq_id[row] < 0 || pos < 0) continue;
+        if (pos >= max_context) { *status = kStatusPosition; continue; }      // beyond the stated bound: row skipped
+        const int ns = (pos + kSplitTokens) / kSplitTokens;
+        acc += ns < max_splits ? ns : max_splits;
+    }
+    item_start[rows.n_rows] = acc;
+}
+
+template <typename T, int DH, int LPT, int CPL>
+void launch_attention_static_t(const AttnParams& p, void* o, int max_context, cudaStream_t st) {
+    attn_static_plan_kernel<<<1, 32, 0, st>>>(p.rows, p.max_splits, max_context, const_cast<int32_t*>(p.item_start), p.counter, p.status);
+    const int max_items = p.rows.n_rows * p.pool.H * p.max_splits;
+    int grid = 148 * 4;
+    if ((max_items + 3) / 4 < grid) grid = (max_items + 3) / 4;
+    attn_split_kernel<T, DH, LPT, CPL><<<grid, 128, 0, st>>>(p);
+    const int warps = p.rows.n_rows * p.pool.H;
+    attn_merge_kernel<T, DH><<<(warps + 3) / 4, 128, 0, st>>>(p, (T*)o);
+}
+
+}  // namespace
 }  // namespace cdbk
+
+extern "C" int cdb_paged_attention_static(const void* q, void* o, const void* pool, int32_t n_phys_pages, int32_t layer,
+                                          const int32_t* seq_id, const int32_t* position, const int32_t* page_table,
+                                          int32_t page_table_stride, int32_t n_rows, int32_t max_seqs,
+                                          int32_t max_context, int32_t H, int32_t Dh, int32_t dtype, void* stream) {
+    using namespace cdbk;
+    if (n_rows == 0) return CDB_OK;
+    if (!q || !o || !pool || !seq_id || !position || !page_table || n_rows < 0 || n_phys_pages < 1 || layer < 0 ||
+        page_table_stride < 1 || max_seqs < 1 || max_context < 1 || H < 1 || (Dh != 64 && Dh != 96 && Dh != 128) ||
+        (dtype != CDB_FP32 && dtype != CDB_BF16))
+        return CDB_ERR_ARG;
+    const int max_splits = (max_context + kSplitTokens - 1) / kSplitTokens;
+    const size_t head = 256;                                                        // status word, work counter
+    const size_t scan = (((size_t)n_rows + 1) * sizeof(int32_t) + 255) / 256 * 256;
+    const size_t part = (size_t)n_rows * H * max_splits * (size_t)(Dh + 2) * sizeof(float);
+    if (head + scan + part > kStaticScratchBytes) {
+        fprintf(stderr, "cdb_paged_attention_static: n_rows=%d x H=%d x ceil(max_context=%d / %d) splits needs %zu bytes of "
+                        "scratch, the built-in array holds %zu\n", n_rows, H, max_context, kSplitTokens, head + scan + part,
+                kStaticScratchBytes);
+        return CDB_ERR_CAPACITY;
+    }
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return CDB_ERR_CUDA;
+    if (!g_static_scratch_addr[dev]) {                                              // one-time set-up on this device
+        void* addr = nullptr;
+        if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || !addr) { cudaGetLastError(); return CDB_ERR_CUDA; }
+        g_static_scratch_addr[dev] = (unsigned char*)addr;
+    }
+    unsigned char* base = g_static_scratch_addr[dev];
+    AttnParams p;
+    p.q = q;
+    p.pool.base = const_cast<void*>(pool); p.pool.n_phys_pages = n_phys_pages; p.pool.H = H; p.pool.Dh = Dh;
+    p.rows.n_rows = n_rows; p.rows.seq_id = seq_id; p.rows.loop_depth = nullptr; p.rows.position = position;
+    p.rows.kv_slot = nullptr; p.rows.forced_exit = nullptr; p.rows.page_table = page_table;
+    p.rows.page_table_stride = page_table_stride; p.rows.n_slots = 1; p.rows.slot_override = 0;
+    p.layer = layer; p.max_splits = max_splits; p.max_seqs = max_seqs;
+    p.scale_log2 = 1.4426950408889634f / sqrtf((float)Dh);
+    p.status = (int32_t*)base; p.counter = (int32_t*)(base + 4);
+    p.item_start = (const int32_t*)(base + head); p.part = (float*)(base + head + scan);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dtype == CDB_BF16) {
+        if (Dh == 128) launch_attention_static_t<__nv_bfloat16, 128, 8, 2>(p, o, max_context, st);
+        else if (Dh == 96) launch_attention_static_t<__nv_bfloat16, 96, 4, 3>(p, o, max_context, st);
+        else launch_attention_static_t<__nv_bfloat16, 64, 8, 1>(p, o, max_context, st);
+    } else {
+        if (Dh == 128) launch_attention_static_t<float, 128, 8, 4>(p, o, max_context, st);
+        else if (Dh == 96) launch_attention_static_t<float, 96, 8, 3>(p, o, max_context, st);
+        else launch_attention_static_t<float, 64, 8, 2>(p, o, max_context, st);
+    }
+    return cudaGetLastError() == cudaSuccess ? CDB_OK : CDB_ERR_CUDA;
+}
