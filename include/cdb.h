@@ -67,7 +67,9 @@ typedef struct {
     int32_t flags;                     /* CDB_FLAG_* */
 } cdb_config_t;
 
-enum { CDB_FLAG_SIMT_GEMM = 1 };       /* run bf16 projections on the plain-FMA kernel (cross-check) */
+enum { CDB_FLAG_SIMT_GEMM = 1,         /* run bf16 projections on the plain-FMA kernel (cross-check) */
+       CDB_FLAG_TWO_STREAM = 2,        /* run a loop step of >= 64 rows as two half-batches on two streams (experimental) */
+       CDB_FLAG_UNFUSED_LAYER = 4 };   /* one launch per projection, separate norm and SwiGLU kernels (cross-check) */
 
 /* Row-major [out_features, in_features] ("K-major") weights of the configured dtype, layers
  * stacked in the order prelude, core, coda (L = L_pre + L_core + L_coda).  All device pointers. */

@@ -22,6 +22,8 @@ FP32, BF16 = 0, 1
 KV_SHARED, KV_DEPTH_INDEXED, KV_FIRST_THEN_SHARED = 0, 1, 2
 GATE_NONE, GATE_SIGMOID_CDF, GATE_L2_CONVERGENCE = 0, 1, 2
 FLAG_SIMT_GEMM = 1
+FLAG_TWO_STREAM = 2
+FLAG_UNFUSED_LAYER = 4
 
 EXPORTS = ["cdb_create", "cdb_destroy", "cdb_last_error", "cdb_kv_bind", "cdb_set_gate", "cdb_boundary_embed",
            "cdb_boundary_prelude", "cdb_loop_step", "cdb_compact", "cdb_gather_rows", "cdb_boundary_coda_lmhead",

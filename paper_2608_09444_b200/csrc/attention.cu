@@ -10,6 +10,7 @@
 // token, keeps the online-softmax state in registers, and writes an (o, m, l) partial.  A second
 // kernel merges the partials of a row in split order.
 #include <cstdio>
+#include <cstdlib>
 
 #include "cdb_internal.h"
 
@@ -40,6 +41,8 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
     return v;
 }
 
+constexpr int kAttnSharedCarveoutPct = -1;   // -1: driver default (largest L1)   // share of the SM's L1/shared array configured as shared memory
+
 struct AttnParams {
     const void* q;             // [n_rows][H*Dh]
     KvPool pool;
@@ -57,6 +60,8 @@ struct AttnParams {
 // splits per row -> exclusive scan; zeroes the per-layer work counters.  One CTA.
 __global__ void __launch_bounds__(1024) attn_plan_kernel(RowsDev rows, int32_t* __restrict__ item_start,
                                                          int32_t* __restrict__ counters, int n_counters) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ int warp_tot[32];
     __shared__ int base;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -91,7 +96,9 @@ __global__ void __launch_bounds__(1024) attn_plan_kernel(RowsDev rows, int32_t* 
 }
 
 template <typename T, int DH, int LPT, int CPL>
-__global__ void __launch_bounds__(128) attn_split_kernel(AttnParams p) {
+__global__ void __maxnreg__(96) attn_split_kernel(AttnParams p) {
+    pdl_trigger();
+    pdl_wait();
     constexpr int EPC = Chunk<T>::EPC;
     static_assert(LPT * CPL * EPC == DH, "lane mapping must cover the head dimension");
     constexpr int TPI = 32 / LPT;               // tokens per warp iteration
@@ -222,6 +229,8 @@ __global__ void __launch_bounds__(128) attn_split_kernel(AttnParams p) {
 // Merge the splits of each (row, head) in split order and round to T.  One warp per (row, head).
 template <typename T, int DH>
 __global__ void __launch_bounds__(128) attn_merge_kernel(AttnParams p, T* __restrict__ out) {
+    pdl_trigger();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int H = p.pool.H;
     const int wid = blockIdx.x * 4 + (threadIdx.x >> 5);
@@ -254,15 +263,19 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(AttnParams p, T* __rest
     for (int k = 0; k < PER; ++k) if (lane + 32 * k < DH) o[lane + 32 * k] = T(acc[k] * inv);
 }
 
-void launch_attention_plan(const cdb* h, const RowsDev& rows, cudaStream_t st) {
+void launch_attention_plan(const cdb* h, int ln, const RowsDev& rows, cudaStream_t st) {
     CDB_LAUNCH(h);
-    attn_plan_kernel<<<1, 1024, 0, st>>>(rows, h->attn_item_start, h->attn_counters, h->cfg.L_pre + h->cfg.L_core + h->cfg.L_coda);
+    launch_pdl(attn_plan_kernel, dim3(1), dim3(1024), 0, st, rows, h->lane[ln].attn_item_start, h->lane[ln].attn_counters, h->cfg.L_pre + h->cfg.L_core + h->cfg.L_coda);
 }
 
 template <typename T, int DH, int LPT, int CPL>
 static void launch_attention_t(const cdb* h, const AttnParams& p, void* o, cudaStream_t st) {
     static int blocks_per_sm = 0;
     if (blocks_per_sm == 0) {
+        // The kernel uses no shared memory; asking for the largest shared-memory carve-out keeps the SM in the
+        // configuration the projection kernel needs, so that its CTAs can become resident beside this one.
+        cudaFuncSetAttribute(attn_split_kernel<T, DH, LPT, CPL>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             getenv("CDB_ATTN_CARVEOUT") ? atoi(getenv("CDB_ATTN_CARVEOUT")) : kAttnSharedCarveoutPct);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, attn_split_kernel<T, DH, LPT, CPL>, 128, 0);
         if (blocks_per_sm < 1) blocks_per_sm = 1;
     }
@@ -271,26 +284,35 @@ static void launch_attention_t(const cdb* h, const AttnParams& p, void* o, cudaS
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int max_items = p.rows.n_rows * p.pool.H * p.max_splits;
-    int grid = sms * blocks_per_sm;
-    if ((max_items + 3) / 4 < grid) grid = (max_items + 3) / 4;
+    // Warps are independent, so the CTA shape only decides how the block scheduler packs the SMs.
+    // Alone: CTAs of 4 warps, as many as fit.  Sharing the GPU with the other half-batch's kernels: one
+    // CTA of 4 * cap warps per SM, which leaves registers free on EVERY SM for a projection CTA
+    // (small CTAs may be packed unevenly and fill some SMs completely).
+    int grid = sms * blocks_per_sm, threads = 128;
+    static const int forced_cap = getenv("CDB_ATTN_CAP") ? atoi(getenv("CDB_ATTN_CAP")) : 0;                  // tuning aid
+    const int cap = forced_cap > 0 ? forced_cap : h->attn_ctas_per_sm_cap;
+    if (cap > 0 && cap < blocks_per_sm) { grid = sms; threads = 128 * cap; }
+    const int warps_per_cta = threads / 32;
+    if ((max_items + warps_per_cta - 1) / warps_per_cta < grid) grid = (max_items + warps_per_cta - 1) / warps_per_cta;
     {
         ProfScope ps(h, kProfAttention, st);
         CDB_LAUNCH(h);
-        attn_split_kernel<T, DH, LPT, CPL><<<grid, 128, 0, st>>>(p);
+        launch_pdl(attn_split_kernel<T, DH, LPT, CPL>, dim3(grid), dim3(threads), 0, st, p);
     }
+    if (h->attn_split_done) cudaEventRecord(h->attn_split_done, st);     // the KV stream is over: the merge is tiny
     CDB_LAUNCH(h);
     const int warps = p.rows.n_rows * p.pool.H;
-    attn_merge_kernel<T, DH><<<(warps + 3) / 4, 128, 0, st>>>(p, (T*)o);
+    launch_pdl(attn_merge_kernel<T, DH>, dim3((warps + 3) / 4), dim3(128), 0, st, p, (T*)o);
 }
 
 // Requires launch_attention_plan() for the same rows earlier on the stream (once per set of rows).
-void launch_attention(const cdb* h, int layer, const RowsDev& rows, const void* q, void* o, cudaStream_t st) {
+void launch_attention(const cdb* h, int ln, int layer, const RowsDev& rows, const void* q, void* o, cudaStream_t st) {
     if (rows.n_rows <= 0) return;
     AttnParams p;
     p.q = q; p.pool = h->pool; p.rows = rows; p.layer = layer; p.max_splits = h->max_splits;
     p.max_seqs = h->cfg.max_seqs;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)h->cfg.Dh);
-    p.part = h->attn_part; p.item_start = h->attn_item_start; p.counter = h->attn_counters + layer; p.status = h->status;
+    p.part = h->lane[ln].attn_part; p.item_start = h->lane[ln].attn_item_start; p.counter = h->lane[ln].attn_counters + layer; p.status = h->status;
     const int Dh = h->cfg.Dh;
     if (h->cfg.dtype == CDB_BF16) {
         if (Dh == 128) launch_attention_t<__nv_bfloat16, 128, 8, 2>(h, p, o, st);
@@ -334,6 +356,8 @@ unsigned char* g_static_scratch_addr[kStaticMaxDevices];         // device addre
 // work counter and status word.  The row count of this variant is small: one thread walks the rows.
 __global__ void attn_static_plan_kernel(RowsDev rows, int max_splits, int max_context, int32_t* __restrict__ item_start,
                                         int32_t* __restrict__ counter, int32_t* __restrict__ status) {
+    pdl_trigger();
+    pdl_wait();
     if (blockIdx.x != 0 || threadIdx.x != 0) return;
     *counter = 0;
     *status = 0;
@@ -351,13 +375,13 @@ __global__ void attn_static_plan_kernel(RowsDev rows, int max_splits, int max_co
 
 template <typename T, int DH, int LPT, int CPL>
 void launch_attention_static_t(const AttnParams& p, void* o, int max_context, cudaStream_t st) {
-    attn_static_plan_kernel<<<1, 32, 0, st>>>(p.rows, p.max_splits, max_context, const_cast<int32_t*>(p.item_start), p.counter, p.status);
+    launch_pdl(attn_static_plan_kernel, dim3(1), dim3(32), 0, st, p.rows, p.max_splits, max_context, const_cast<int32_t*>(p.item_start), p.counter, p.status);
     const int max_items = p.rows.n_rows * p.pool.H * p.max_splits;
     int grid = 148 * 4;
     if ((max_items + 3) / 4 < grid) grid = (max_items + 3) / 4;
-    attn_split_kernel<T, DH, LPT, CPL><<<grid, 128, 0, st>>>(p);
+    launch_pdl(attn_split_kernel<T, DH, LPT, CPL>, dim3(grid), dim3(128), 0, st, p);
     const int warps = p.rows.n_rows * p.pool.H;
-    attn_merge_kernel<T, DH><<<(warps + 3) / 4, 128, 0, st>>>(p, (T*)o);
+    launch_pdl(attn_merge_kernel<T, DH>, dim3((warps + 3) / 4), dim3(128), 0, st, p, (T*)o);
 }
 
 }  // namespace

@@ -2,6 +2,7 @@
 // the boundary stages, the loop step, the compaction and the prefill.
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -9,6 +10,10 @@
 #include "cdb_internal.h"
 
 using namespace cdbk;
+
+constexpr int kMinSplitRows = 64;          // below this a loop step runs as one batch on one stream
+constexpr int kSplitGemmSmemBytes = 0;            // no cap: a projection CTA co-resides with attention only when its ring is large
+constexpr int kSplitAttnCtasPerSm = 3;     // attention CTAs per SM when two half-batches share the GPU
 
 namespace {
 
@@ -69,36 +74,107 @@ const void* layer_ptr(const cdb_t* h, const void* base, int layer, size_t elems_
 // One transformer layer on `x` (fp32 [n_rows, d], updated in place).  Steps A1-A6 of the loop step:
 // RMSNorm + QKV projection, RoPE + KV page write, paged attention, output projection + residual,
 // RMSNorm + gate/up projections + SwiGLU, down projection + residual.
-void layer_forward(cdb_t* h, int layer, const RowsDev& rows, float* x, cudaStream_t st) {
+void layer_forward(cdb_t* h, int ln, int layer, const RowsDev& rows, float* x, cudaStream_t st,
+                   cudaEvent_t attn_after = nullptr, cudaEvent_t attn_done = nullptr) {
     const cdb_config_t& c = h->cfg;
+    const Lane& L = h->lane[ln];
     const int n = rows.n_rows;
     const size_t d = c.d, F = c.F;
-    launch_rmsnorm(h, x, h->g_attn + (size_t)layer * d, h->xn, rows, st);
-    launch_linear(h, h->xn, layer_ptr(h, h->w.W_qkv, layer, 3 * d * d), h->qkv, n, 3 * c.d, c.d, Epilogue::Store, st);
-    launch_rope_kv_write(h, layer, rows, st);
-    launch_attention(h, layer, rows, h->qrot, h->attn_o, st);
-    launch_linear(h, h->attn_o, layer_ptr(h, h->w.W_o, layer, d * d), x, n, c.d, c.d, Epilogue::ResidualAdd, st);
-    launch_rmsnorm(h, x, h->g_mlp + (size_t)layer * d, h->xn, rows, st);
-    launch_linear(h, h->xn, layer_ptr(h, h->w.W_gate, layer, F * d), h->gu, n, c.F, c.d, Epilogue::Store, st);
-    launch_linear(h, h->xn, layer_ptr(h, h->w.W_up, layer, F * d), h->gu + (size_t)c.max_rows * F, n, c.F, c.d, Epilogue::Store, st);
-    launch_swiglu(h, n, st);
-    launch_linear(h, h->act, layer_ptr(h, h->w.W_down, layer, d * F), x, n, c.d, c.F, Epilogue::ResidualAdd, st);
+    launch_rmsnorm(h, x, h->g_attn + (size_t)layer * d, L.xn, rows, st);
+    launch_linear(h, L.xn, layer_ptr(h, h->w.W_qkv, layer, 3 * d * d), L.qkv, n, 3 * c.d, c.d, Epilogue::Store, st);
+    launch_rope_kv_write(h, ln, layer, rows, st);
+    if (attn_after) cudaStreamWaitEvent(st, attn_after, 0);      // the other half-batch's attention goes first
+    h->attn_split_done = attn_done;
+    launch_attention(h, ln, layer, rows, L.qrot, L.attn_o, st);
+    h->attn_split_done = nullptr;
+    launch_linear(h, L.attn_o, layer_ptr(h, h->w.W_o, layer, d * d), x, n, c.d, c.d, Epilogue::ResidualAdd, st);
+    launch_rmsnorm(h, x, h->g_mlp + (size_t)layer * d, L.xn, rows, st);
+    launch_linear(h, L.xn, layer_ptr(h, h->w.W_gate, layer, F * d), L.gu, n, c.F, c.d, Epilogue::Store, st);
+    launch_linear(h, L.xn, layer_ptr(h, h->w.W_up, layer, F * d), L.gu + (size_t)L.rows_cap * F, n, c.F, c.d, Epilogue::Store, st);
+    launch_swiglu(h, ln, n, st);
+    launch_linear(h, L.act, layer_ptr(h, h->w.W_down, layer, d * F), x, n, c.d, c.F, Epilogue::ResidualAdd, st);
+}
+
+// The same layer on the bf16 tensor-core path, with fewer and fatter launches: the two residual
+// projections run split-K into a workspace and one row-wise kernel reduces the parts in fixed order,
+// adds the residual and produces the next projection's normed input; gate and up run as one launch
+// with SwiGLU in its epilogue.  xn_ready: L.xn already holds RMSNorm(x; g_attn[layer]).  next_gain:
+// gain of the norm that follows this layer on the same rows (NULL: none).
+void layer_forward_tc(cdb_t* h, int ln, int layer, const RowsDev& rows, float* x, cudaStream_t st, bool xn_ready,
+                      const float* next_gain, cudaEvent_t attn_after = nullptr, cudaEvent_t attn_done = nullptr) {
+    const cdb_config_t& c = h->cfg;
+    const Lane& L = h->lane[ln];
+    const int n = rows.n_rows;
+    const size_t d = c.d, F = c.F;
+    if (!xn_ready) launch_rmsnorm(h, x, h->g_attn + (size_t)layer * d, L.xn, rows, st);
+    launch_linear(h, L.xn, layer_ptr(h, h->w.W_qkv, layer, 3 * d * d), L.qkv, n, 3 * c.d, c.d, Epilogue::Store, st);
+    launch_rope_kv_write(h, ln, layer, rows, st);
+    if (attn_after) cudaStreamWaitEvent(st, attn_after, 0);      // the other half-batch's attention goes first
+    h->attn_split_done = attn_done;
+    launch_attention(h, ln, layer, rows, L.qrot, L.attn_o, st);
+    h->attn_split_done = nullptr;
+    {
+        ProfScope ps(h, kProfLinear, st);
+        CDB_LAUNCH(h);
+        const int s = launch_linear_splitk_tc(h, L.attn_o, layer_ptr(h, h->w.W_o, layer, d * d), L.ws, kMaxKSplits, n, c.d, c.d, st);
+        if (!s) h->launch_error = 1;
+        launch_reduce_residual_norm(h, L.ws, s, (size_t)n * d, x, h->g_mlp + (size_t)layer * d, L.xn, rows, st);
+    }
+    {
+        ProfScope ps(h, kProfLinear, st);
+        CDB_LAUNCH(h);
+        if (!launch_gate_up_swiglu_tc(h, L.xn, layer_ptr(h, h->w.W_gate, layer, F * d), layer_ptr(h, h->w.W_up, layer, F * d),
+                                      L.act, n, c.F, c.d, st))
+            h->launch_error = 1;
+    }
+    {
+        ProfScope ps(h, kProfLinear, st);
+        CDB_LAUNCH(h);
+        const int s = launch_linear_splitk_tc(h, L.act, layer_ptr(h, h->w.W_down, layer, d * F), L.ws, kMaxKSplits, n, c.d, c.F, st);
+        if (!s) h->launch_error = 1;
+        launch_reduce_residual_norm(h, L.ws, s, (size_t)n * d, x, next_gain, L.xn, rows, st);
+    }
+}
+
+bool use_tc_layers(const cdb_t* h) {
+    return h->cfg.dtype == CDB_BF16 && !(h->cfg.flags & (CDB_FLAG_SIMT_GEMM | CDB_FLAG_UNFUSED_LAYER)) && h->cfg.d <= 24 * 256 &&
+           linear_tc_supported(h, 1, h->cfg.d, h->cfg.d);
+}
+
+// core layers [first, last) on one lane; picks the fused tensor-core flow when available
+void core_layers(cdb_t* h, int ln, const RowsDev& rows, float* x, cudaStream_t st, cudaEvent_t attn_after_first,
+                 cudaEvent_t attn_after, cudaEvent_t attn_done, int layer) {
+    const cdb_config_t& c = h->cfg;
+    const int first = c.L_pre, last = c.L_pre + c.L_core;
+    cudaEvent_t after = layer == first ? attn_after_first : attn_after;
+    if (use_tc_layers(h))
+        layer_forward_tc(h, ln, layer, rows, x, st, layer > first, layer + 1 < last ? h->g_attn + (size_t)(layer + 1) * c.d : nullptr,
+                         after, attn_done);
+    else
+        layer_forward(h, ln, layer, rows, x, st, after, attn_done);
 }
 
 // final RMSNorm + LM head + greedy argmax on n rows of x
 void lm_head(cdb_t* h, const RowsDev& rows, const float* x, int32_t* token_out, float* logits_out, cudaStream_t st) {
     const cdb_config_t& c = h->cfg;
     float* logits = logits_out ? logits_out : h->logits;
-    launch_rmsnorm(h, x, h->g_final, h->xn, rows, st);
-    launch_linear(h, h->xn, h->w.W_lm, logits, rows.n_rows, c.V, c.d, Epilogue::Store, st);
+    launch_rmsnorm(h, x, h->g_final, h->lane[0].xn, rows, st);
+    launch_linear(h, h->lane[0].xn, h->w.W_lm, logits, rows.n_rows, c.V, c.d, Epilogue::Store, st);
     launch_argmax(h, logits, rows.n_rows, token_out, st);
 }
 
 void free_all(cdb_t* h) {
-    void* ptrs[] = {h->rope_cos, h->rope_sin, h->g_attn, h->g_mlp, h->g_final, h->gate_S, h->gate_fire, h->xn, h->qrot,
-                    h->attn_o, h->act, h->qkv, h->gu, h->h_prev, h->h_work, h->logits, h->attn_part,
-                    h->attn_item_start, h->attn_counters, h->exit_flag, h->status, h->emit_tmp};
+    void* ptrs[] = {h->rope_cos, h->rope_sin, h->g_attn, h->g_mlp, h->g_final, h->gate_S, h->gate_fire,
+                    h->h_prev, h->h_work, h->logits, h->exit_flag, h->status, h->emit_tmp};
     for (void* p : ptrs) if (p) cudaFree(p);
+    for (Lane& L : h->lane) {
+        void* lp[] = {L.xn, L.qrot, L.attn_o, L.act, L.qkv, L.gu, L.ws, L.attn_part, L.attn_item_start, L.attn_counters};
+        for (void* p : lp) if (p) cudaFree(p);
+    }
+    if (h->side) cudaStreamDestroy(h->side);
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_join) cudaEventDestroy(h->ev_join);
+    for (cudaEvent_t e : h->ev_attn) if (e) cudaEventDestroy(e);
     if (h->prof_ev) {
         for (int i = 0; i < 2 * kProfCap; ++i) if (h->prof_ev[i]) cudaEventDestroy(h->prof_ev[i]);
         delete[] h->prof_ev;
@@ -152,6 +228,7 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
     h->pool.Dh = c.Dh;
     const size_t R_ = c.max_rows, d = c.d, F = c.F, half = c.Dh / 2;
     const size_t wide = d > F ? d : F;
+    const int n_layers = L;
     cudaError_t e = cudaSuccess;
 #define CDB_ALLOC(ptr, type, count) if (e == cudaSuccess) e = dev_alloc<type>((type**)&(ptr), (count))
     CDB_ALLOC(h->rope_cos, float, (size_t)c.max_position * half);
@@ -161,18 +238,24 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
     CDB_ALLOC(h->g_final, float, d);
     CDB_ALLOC(h->gate_S, float, c.max_seqs);
     CDB_ALLOC(h->gate_fire, uint8_t, c.max_seqs);
-    CDB_ALLOC(h->xn, char, R_ * wide * h->elem_size);
-    CDB_ALLOC(h->qrot, char, R_ * d * h->elem_size);
-    CDB_ALLOC(h->attn_o, char, R_ * d * h->elem_size);
-    CDB_ALLOC(h->act, char, R_ * F * h->elem_size);
-    CDB_ALLOC(h->qkv, float, R_ * 3 * d);
-    CDB_ALLOC(h->gu, float, R_ * 2 * F);
+    for (int ln = 0; ln < 2; ++ln) {
+        Lane& L = h->lane[ln];
+        L.rows_cap = ln == 0 ? c.max_rows : (c.max_rows + 1) / 2;
+        const size_t r = L.rows_cap;
+        CDB_ALLOC(L.xn, char, r * wide * h->elem_size);
+        CDB_ALLOC(L.qrot, char, r * d * h->elem_size);
+        CDB_ALLOC(L.attn_o, char, r * d * h->elem_size);
+        CDB_ALLOC(L.act, char, r * F * h->elem_size);
+        CDB_ALLOC(L.qkv, float, r * 3 * d);
+        CDB_ALLOC(L.gu, float, r * 2 * F);
+        CDB_ALLOC(L.ws, float, (size_t)kMaxKSplits * r * d);
+        CDB_ALLOC(L.attn_part, float, r * c.H * h->max_splits * (size_t)(c.Dh + 2));
+        CDB_ALLOC(L.attn_item_start, int32_t, r + 1);
+        CDB_ALLOC(L.attn_counters, int32_t, n_layers);
+    }
     CDB_ALLOC(h->h_prev, float, R_ * d);
     CDB_ALLOC(h->h_work, float, R_ * d);
     CDB_ALLOC(h->logits, float, R_ * (size_t)c.V);
-    CDB_ALLOC(h->attn_part, float, R_ * c.H * h->max_splits * (size_t)(c.Dh + 2));
-    CDB_ALLOC(h->attn_item_start, int32_t, R_ + 1);
-    CDB_ALLOC(h->attn_counters, int32_t, L);
     CDB_ALLOC(h->exit_flag, uint8_t, R_);
     CDB_ALLOC(h->status, int32_t, 1);
     CDB_ALLOC(h->emit_tmp, int32_t, R_);
@@ -199,7 +282,12 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
         gains_to_f32(h, w->g_final, h->g_final, d);
         init_gate_state_kernel<<<(c.max_seqs + 255) / 256, 256>>>(h->gate_S, h->gate_fire, c.max_seqs);
         cudaMemset(h->status, 0, sizeof(int32_t));
-        cudaMemset(h->attn_counters, 0, sizeof(int32_t) * L);
+        for (int ln = 0; ln < 2; ++ln) cudaMemset(h->lane[ln].attn_counters, 0, sizeof(int32_t) * L);
+        if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess) h->side = nullptr;
+        cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
+        cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
+        cudaEventCreateWithFlags(&h->ev_attn[0], cudaEventDisableTiming);
+        cudaEventCreateWithFlags(&h->ev_attn[1], cudaEventDisableTiming);
         e = cudaDeviceSynchronize();
     }
     if (e != cudaSuccess) { free_all(h); delete h; cudaGetLastError(); return CDB_ERR_CUDA; }
@@ -248,8 +336,8 @@ static int boundary_in(cdb_t* h, const int32_t* token_ids, const cdb_rows_t* row
     if (prelude && h->cfg.L_pre > 0) {
         if (!h->pool.base) return fail(h, CDB_ERR_STATE, "no KV pool bound");
         rd.slot_override = 0;
-        launch_attention_plan(h, rd, st);
-        for (int l = 0; l < h->cfg.L_pre; ++l) layer_forward(h, l, rd, h_out, st);
+        launch_attention_plan(h, 0, rd, st);
+        for (int l = 0; l < h->cfg.L_pre; ++l) layer_forward(h, 0, l, rd, h_out, st);
     }
     return check_launch(h, "cdb_boundary_embed/prelude");
 }
@@ -274,8 +362,40 @@ int cdb_loop_step(cdb_t* h, const cdb_rows_t* rows, float* h_inout, float* gate_
     const cdb_config_t& c = h->cfg;
     if (c.gate_kind == CDB_GATE_L2_CONVERGENCE)
         cudaMemcpyAsync(h->h_prev, h_inout, (size_t)rd.n_rows * c.d * sizeof(float), cudaMemcpyDeviceToDevice, st);
-    launch_attention_plan(h, rd, st);
-    for (int l = c.L_pre; l < c.L_pre + c.L_core; ++l) layer_forward(h, l, rd, h_inout, st);
+    const int n0 = (rd.n_rows + 1) / 2;
+    const bool split = (c.flags & CDB_FLAG_TWO_STREAM) && h->side && rd.n_rows >= kMinSplitRows;
+    if (!split) {
+        h->attn_ctas_per_sm_cap = 0;
+        launch_attention_plan(h, 0, rd, st);
+        for (int l = c.L_pre; l < c.L_pre + c.L_core; ++l) core_layers(h, 0, rd, h_inout, st, nullptr, nullptr, nullptr, l);
+    } else {
+        // Two half-batches on two streams: while one half streams its KV pages through the attention
+        // kernel (HBM-bound), the other half's projections and row-wise kernels run beside it.  Rows
+        // are independent, so the halves never synchronise inside the step.
+        RowsDev half[2] = {rd, rd};
+        half[0].n_rows = n0;
+        half[1].n_rows = rd.n_rows - n0;
+        half[1].seq_id += n0; half[1].loop_depth += n0; half[1].position += n0; half[1].kv_slot += n0;
+        if (half[1].forced_exit) half[1].forced_exit += n0;
+        h->attn_ctas_per_sm_cap = kSplitAttnCtasPerSm;
+        h->gemm_smem_cap = kSplitGemmSmemBytes;
+        cudaEventRecord(h->ev_fork, st);
+        cudaStreamWaitEvent(h->side, h->ev_fork, 0);
+        cudaStream_t ss[2] = {st, h->side};
+        float* xs[2] = {h_inout, h_inout + (size_t)n0 * c.d};
+        for (int ln = 0; ln < 2; ++ln) launch_attention_plan(h, ln, half[ln], ss[ln]);
+        // The two attention kernels are chained A(l), B(l), A(l+1), ...: each then streams at full HBM
+        // bandwidth, and the other half's projections fill the SMs' spare issue slots meanwhile.
+        // Without the chain both halves drift into lock-step (attention together, projections together).
+        for (int l = c.L_pre; l < c.L_pre + c.L_core; ++l) {
+            core_layers(h, 0, half[0], xs[0], ss[0], nullptr, h->ev_attn[1], h->ev_attn[0], l);
+            core_layers(h, 1, half[1], xs[1], ss[1], h->ev_attn[0], h->ev_attn[0], h->ev_attn[1], l);
+        }
+        cudaEventRecord(h->ev_join, h->side);
+        cudaStreamWaitEvent(st, h->ev_join, 0);
+        h->attn_ctas_per_sm_cap = 0;
+        h->gemm_smem_cap = 0;
+    }
     launch_gate(h, rd, h_inout, h->h_prev, gate_val_out, fire_out, st);
     return check_launch(h, "cdb_loop_step");
 }
@@ -319,8 +439,8 @@ int cdb_boundary_coda_lmhead(cdb_t* h, const cdb_rows_t* rows, float* h_exit, in
     if (c.L_coda > 0) {
         if (!h->pool.base) return fail(h, CDB_ERR_STATE, "no KV pool bound");
         rd.slot_override = 0;
-        launch_attention_plan(h, rd, st);
-        for (int l = c.L_pre + c.L_core; l < c.L_pre + c.L_core + c.L_coda; ++l) layer_forward(h, l, rd, h_exit, st);
+        launch_attention_plan(h, 0, rd, st);
+        for (int l = c.L_pre + c.L_core; l < c.L_pre + c.L_core + c.L_coda; ++l) layer_forward(h, 0, l, rd, h_exit, st);
     }
     lm_head(h, rd, h_exit, token_out, logits_out, st);
     return check_launch(h, "cdb_boundary_coda_lmhead");
@@ -340,15 +460,15 @@ int cdb_prefill(cdb_t* h, const int32_t* token_ids, const cdb_rows_t* rows, cons
     const cdb_config_t& c = h->cfg;
     float* x = h->h_work;
     launch_embed(h, token_ids, rd, x, true, st);
-    launch_attention_plan(h, rd, st);
+    launch_attention_plan(h, 0, rd, st);
     rd.slot_override = 0;
-    for (int l = 0; l < c.L_pre; ++l) layer_forward(h, l, rd, x, st);
+    for (int l = 0; l < c.L_pre; ++l) layer_forward(h, 0, l, rd, x, st);
     for (int r = 1; r <= c.R; ++r) {
         rd.slot_override = slot_of_loop(c.kv_layout, r);
-        for (int l = c.L_pre; l < c.L_pre + c.L_core; ++l) layer_forward(h, l, rd, x, st);
+        for (int l = c.L_pre; l < c.L_pre + c.L_core; ++l) layer_forward(h, 0, l, rd, x, st);
     }
     rd.slot_override = 0;
-    for (int l = c.L_pre + c.L_core; l < c.L_pre + c.L_core + c.L_coda; ++l) layer_forward(h, l, rd, x, st);
+    for (int l = c.L_pre + c.L_core; l < c.L_pre + c.L_core + c.L_coda; ++l) layer_forward(h, 0, l, rd, x, st);
     if (n_emit > 0) {
         // gather the emitting rows to the front of h_prev (free during prefill), then LM head on them
         launch_gather(h, x, emit_idx, nullptr, n_emit, h->h_prev, st);
@@ -383,8 +503,8 @@ int cdb_paged_attention(cdb_t* h, const cdb_rows_t* rows, int32_t layer, const v
     if (layer < 0 || layer >= h->cfg.L_pre + h->cfg.L_core + h->cfg.L_coda) return fail(h, CDB_ERR_RANGE, "layer out of range");
     if (!h->pool.base) return fail(h, CDB_ERR_STATE, "no KV pool bound");
     if (!rows->kv_slot) rd.slot_override = 0;
-    launch_attention_plan(h, rd, (cudaStream_t)stream);
-    launch_attention(h, layer, rd, q, o, (cudaStream_t)stream);
+    launch_attention_plan(h, 0, rd, (cudaStream_t)stream);
+    launch_attention(h, 0, layer, rd, q, o, (cudaStream_t)stream);
     return check_launch(h, "cdb_paged_attention");
 }
 
@@ -422,6 +542,17 @@ int cdb_profile_read(cdb_t* h, cdb_profile_t* out) {
     if (e != cudaSuccess) return fail_cuda(h, e, "cdb_profile_read");
     memset(out, 0, sizeof(*out));
     out->launches = h->launches;
+    if (const char* path = getenv("CDB_PROF_DUMP")) {           // tuning aid: (class, start, end) of every bracketed launch
+        if (FILE* f = fopen(path, "w")) {
+            for (int i = 0; i < h->prof_used; ++i) {
+                float a = 0.f, b = 0.f;
+                cudaEventElapsedTime(&a, h->prof_ev[0], h->prof_ev[2 * i]);
+                cudaEventElapsedTime(&b, h->prof_ev[0], h->prof_ev[2 * i + 1]);
+                fprintf(f, "%d,%.4f,%.4f\n", (int)h->prof_cls[i], a, b);
+            }
+            fclose(f);
+        }
+    }
     for (int i = 0; i < h->prof_used; ++i) {
         float ms = 0.f;
         if (cudaEventElapsedTime(&ms, h->prof_ev[2 * i], h->prof_ev[2 * i + 1]) != cudaSuccess) continue;

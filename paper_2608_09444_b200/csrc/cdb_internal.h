@@ -11,6 +11,7 @@ namespace cdbk {
 
 constexpr int kPageSize = 16;        // tokens per KV page
 constexpr int kSplitTokens = 256;    // attention split length; depends on nothing but the row's own context
+constexpr int kMaxKSplits = 4;       // split-K parts of the residual projections
 constexpr int kStatusPage = 1, kStatusPosition = 2, kStatusSeq = 3;
 
 enum class Epilogue : int { Store = 0, ResidualAdd = 1 };
@@ -41,6 +42,21 @@ struct KvPool {
     }
 };
 
+// Scratch of one half-batch ("lane"): activations between the kernels of a layer, attention partials.
+struct Lane {
+    int rows_cap;                   // rows this lane's buffers hold
+    void* xn;                       // [rows_cap][max(d,F)] normed activations (dtype)
+    void* qrot;                     // [rows_cap][d] rotated queries (dtype)
+    void* attn_o;                   // [rows_cap][d] attention output (dtype)
+    void* act;                      // [rows_cap][F] SwiGLU output (dtype)
+    float* qkv;                     // [rows_cap][3d]
+    float* gu;                      // [2][rows_cap][F] gate and up projections
+    float* ws;                      // [kMaxKSplits][rows_cap][d] split-K partial products
+    float* attn_part;               // [rows_cap*H*max_splits][Dh + 2] split partials (o, m, l)
+    int32_t* attn_item_start;       // [rows_cap + 1] exclusive scan of splits per row
+    int32_t* attn_counters;         // [L] work-fetch counters
+};
+
 }  // namespace cdbk
 
 struct cdb {
@@ -58,24 +74,24 @@ struct cdb {
     float* g_final;                 // [d]
     float* gate_S;                  // [max_seqs] survival of the cumulative exit probability
     uint8_t* gate_fire;             // [max_seqs] stored exit signal
-    void* xn;                       // [max_rows][max(d,F)] normed activations / attention out / MLP act (dtype)
-    void* qrot;                     // [max_rows][d] rotated queries (dtype)
-    void* attn_o;                   // [max_rows][d] attention output (dtype)
-    void* act;                      // [max_rows][F] SwiGLU output (dtype)
-    float* qkv;                     // [max_rows][3d]
-    float* gu;                      // [max_rows][2F]
+    // per-lane scratch: lane 0 holds max_rows rows, lane 1 half of that (second half-batch of a split step)
+    cdbk::Lane lane[2];
     float* h_prev;                  // [max_rows][d] state at step entry (convergence gate)
     float* h_work;                  // [max_rows][d] prefill working state
     float* logits;                  // [max_rows][V]
-    float* attn_part;               // [max_rows*H*max_splits][Dh + 2] split partials (o, m, l)
-    int32_t* attn_item_start;       // [max_rows + 1] exclusive scan of splits per row
-    int32_t* attn_counters;         // [L] work-fetch counters
     uint8_t* exit_flag;             // [max_rows]
     int32_t* status;                // [1] first out-of-range access seen (0 = clean)
     int32_t* emit_tmp;              // [max_rows]
     char err[256];
 
     // instrumentation: kernel launch count, and CUDA-event pairs around the two heavy kernel classes
+    // two-stream execution of a loop step: second half-batch on `side`, joined by events
+    cudaStream_t side;
+    cudaEvent_t ev_fork, ev_join, ev_attn[2];
+    mutable cudaEvent_t attn_split_done; // recorded right after the next attention split kernel when set
+    mutable int attn_ctas_per_sm_cap;
+    mutable int gemm_smem_cap;          // > 0: projection kernels keep their shared-memory ring below this many bytes   // > 0: leave room on every SM for the other half-batch's kernels
+
     mutable uint64_t launches;
     mutable int launch_error;       // a launcher could not set up its kernel (tensor-map encode failed)
     mutable int prof_on, prof_used;
@@ -84,6 +100,26 @@ struct cdb {
 };
 
 #define CDB_LAUNCH(h) (++(h)->launches)
+
+namespace cdbk {
+// Programmatic dependent launch: the kernel may be scheduled while its predecessor on the stream is
+// still draining; it runs its set-up, then pdl_wait() blocks until the predecessor has completed and
+// its writes are visible.  Every kernel of the library calls pdl_trigger() first (lets ITS successor
+// be scheduled early) and pdl_wait() before its first global-memory access.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+}  // namespace cdbk
 
 namespace cdbk {
 constexpr int kProfCap = 8192;
@@ -106,10 +142,10 @@ namespace cdbk {
 
 // ---- launchers (each enqueues on `st`; none synchronises) -----------------------------------
 void launch_rmsnorm(const cdb* h, const float* x, const float* gain, void* out, const RowsDev& rows, cudaStream_t st);
-void launch_rope_kv_write(const cdb* h, int layer, const RowsDev& rows, cudaStream_t st);
-void launch_attention(const cdb* h, int layer, const RowsDev& rows, const void* q, void* o, cudaStream_t st);
-void launch_attention_plan(const cdb* h, const RowsDev& rows, cudaStream_t st);
-void launch_swiglu(const cdb* h, int n_rows, cudaStream_t st);
+void launch_rope_kv_write(const cdb* h, int ln, int layer, const RowsDev& rows, cudaStream_t st);
+void launch_attention(const cdb* h, int ln, int layer, const RowsDev& rows, const void* q, void* o, cudaStream_t st);
+void launch_attention_plan(const cdb* h, int ln, const RowsDev& rows, cudaStream_t st);
+void launch_swiglu(const cdb* h, int ln, int n_rows, cudaStream_t st);
 void launch_embed(const cdb* h, const int32_t* tokens, const RowsDev& rows, float* out, bool reset_gate, cudaStream_t st);
 void launch_gate(const cdb* h, const RowsDev& rows, const float* x, const float* x_prev, float* gate_val_out,
                  uint8_t* fire_out, cudaStream_t st);
@@ -119,6 +155,14 @@ void launch_gather(const cdb* h, const float* src, const int32_t* idx, const int
                    float* dst, cudaStream_t st);
 void launch_argmax(const cdb* h, const float* logits, int n_rows, int32_t* token_out, cudaStream_t st);
 void launch_copy_on_exit(const cdb* h, const RowsDev& rows, const int32_t* exit_depth, cudaStream_t st);
+
+// x[row] += sum_s ws[s][row] (fixed order), then out[row] = RMSNorm(x[row]) * gain when gain != NULL.
+void launch_reduce_residual_norm(const cdb* h, const float* ws, int splits, size_t split_stride, float* x, const float* gain,
+                                 void* out, const RowsDev& rows, cudaStream_t st);
+// bf16 tensor-core variants (gemm_tcgen05.cu)
+bool linear_tc_supported(const cdb* h, int n, int N, int K);
+bool launch_gate_up_swiglu_tc(const cdb* h, const void* x, const void* Wg, const void* Wu, void* act, int n, int F, int K, cudaStream_t st);
+int launch_linear_splitk_tc(const cdb* h, const void* x, const void* W, float* ws, int max_splits, int n, int N, int K, cudaStream_t st);
 
 // y[n,N] (fp32) = / += x[n,K] . W[N,K]^T ; x and W of the handle's dtype.
 void launch_linear(const cdb* h, const void* x, const void* W, float* y, int n, int N, int K, Epilogue ep, cudaStream_t st);

@@ -17,6 +17,8 @@ constexpr int BM = 64, BN = 64, BK = 16;
 template <typename T, int EP>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ A, const T* __restrict__ W,
                                                         float* __restrict__ C, int n, int N, int K) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float As[BK][BM + 4];
     __shared__ float Ws[BK][BN + 4];
     const int tid = threadIdx.x;
@@ -68,9 +70,9 @@ template <typename T>
 static void launch_simt(const void* x, const void* W, float* y, int n, int N, int K, Epilogue ep, cudaStream_t st) {
     dim3 grid((N + BN - 1) / BN, (n + BM - 1) / BM);
     if (ep == Epilogue::ResidualAdd)
-        gemm_simt_kernel<T, 1><<<grid, 256, 0, st>>>((const T*)x, (const T*)W, y, n, N, K);
+        launch_pdl(gemm_simt_kernel<T, 1>, dim3(grid), dim3(256), 0, st, (const T*)x, (const T*)W, y, n, N, K);
     else
-        gemm_simt_kernel<T, 0><<<grid, 256, 0, st>>>((const T*)x, (const T*)W, y, n, N, K);
+        launch_pdl(gemm_simt_kernel<T, 0>, dim3(grid), dim3(256), 0, st, (const T*)x, (const T*)W, y, n, N, K);
 }
 
 void launch_linear(const cdb* h, const void* x, const void* W, float* y, int n, int N, int K, Epilogue ep, cudaStream_t st) {

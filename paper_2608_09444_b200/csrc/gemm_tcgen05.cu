@@ -98,17 +98,33 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
                  : "r"(taddr) : "memory");
 }
 
+enum { kModeStore = 0, kModeAccumulate = 1, kModeSwiGLU = 2 };
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                 : "r"(taddr) : "memory");
+}
+
 struct GemmParams {
-    float* y;
+    float* y;                   // store / accumulate: [k_splits][n][N] fp32 (split s at y + s * split_stride)
+    __nv_bfloat16* act;         // SwiGLU mode: [n][N] bf16 = SiLU(x.Wg^T) * (x.Wu^T)
     int n, N, K;
-    int BN;             // rows per tile (MMA N): 64, 128 or 256
+    int BN;                     // rows per tile (MMA N): 64, 128 or 256 (<= 128 in SwiGLU mode)
     int stages;
-    int accumulate;     // 1: y += result
+    int mode;
+    int k_splits;               // the K range is cut into this many parts, each a tile of its own
+    size_t split_stride;
     int32_t* status;
 };
 
-__global__ void __launch_bounds__(kThreads, 1)
-gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, GemmParams p) {
+// at most 72 registers per thread, so that a CTA fits on an SM beside four attention CTAs
+__global__ void __maxnreg__(72)
+gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w2,
+                         const __grid_constant__ CUtensorMap map_x, GemmParams p) {
+    pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2 * 8 + 4];          // full[stages], empty[stages], acc_full[2], acc_empty[2]
     __shared__ uint32_t tmem_base_slot;
@@ -116,14 +132,17 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int S = p.stages, BN = p.BN;
-    const uint32_t w_bytes = BM * BK * 2, x_bytes = (uint32_t)BN * BK * 2, stage_bytes = w_bytes + x_bytes;
+    const bool dual = p.mode == kModeSwiGLU;                                 // two weight tiles, two accumulators
+    const uint32_t w_bytes = BM * BK * 2, x_bytes = (uint32_t)BN * BK * 2;
+    const uint32_t x_off = dual ? 2 * w_bytes : w_bytes, stage_bytes = x_off + x_bytes;
+    const uint32_t acc_cols = dual ? 2u * BN : (uint32_t)BN;                 // TMEM columns of one accumulator set
     const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;            // swizzled tiles need 1024-byte alignment
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (8 + s); };
     auto acc_full_bar = [&](int a) { return bar0 + 8u * (16 + a); };
     auto acc_empty_bar = [&](int a) { return bar0 + 8u * (18 + a); };
-    const uint32_t tmem_cols = 2u * BN < 32u ? 32u : 2u * BN;               // 128, 256 or 512: a power of two
+    const uint32_t tmem_cols = 2u * acc_cols;                               // double-buffered; 128, 256 or 512
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -140,23 +159,27 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_slot;
     volatile int* abortp = &abort_flag;
+    pdl_wait();                 // set-up above overlaps the previous kernel's tail; operands are read only from here on
 
     const int n_ftiles = (p.N + BM - 1) / BM, n_rtiles = (p.n + BN - 1) / BN;
-    const int n_tiles = n_ftiles * n_rtiles;
+    const int n_tiles = n_ftiles * n_rtiles * p.k_splits;                   // tile t = (split, row tile, feature tile)
     const int n_kb = (p.K + BK - 1) / BK;
+    auto kb_begin = [&](int t) { return (int)((long long)(t / (n_ftiles * n_rtiles)) * n_kb / p.k_splits); };
+    auto kb_end = [&](int t) { return (int)((long long)(t / (n_ftiles * n_rtiles) + 1) * n_kb / p.k_splits); };
 
     if (warp == 0) {
         if (lane == 0) {
             int s = 0; uint32_t ph = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-                const int f0 = (t % n_ftiles) * BM, r0 = (t / n_ftiles) * BN;
-                for (int kb = 0; kb < n_kb; ++kb) {
+                const int f0 = (t % n_ftiles) * BM, r0 = (t / n_ftiles % n_rtiles) * BN;
+                for (int kb = kb_begin(t); kb < kb_end(t); ++kb) {
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abortp)) { ok = false; break; }
                     mbar_expect_tx(full_bar(s), stage_bytes);
                     const uint32_t dst = ring + (uint32_t)s * stage_bytes;
                     tma_load_2d(dst, &map_w, full_bar(s), kb * BK, f0);
-                    tma_load_2d(dst + w_bytes, &map_x, full_bar(s), kb * BK, r0);
+                    if (dual) tma_load_2d(dst + w_bytes, &map_w2, full_bar(s), kb * BK, f0);
+                    tma_load_2d(dst + x_off, &map_x, full_bar(s), kb * BK, r0);
                     if (++s == S) { s = 0; ph ^= 1u; }
                 }
             }
@@ -177,16 +200,21 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
                 const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
                 if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, abortp)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-                for (int kb = 0; kb < n_kb; ++kb) {
+                const uint32_t d_tmem = tmem_base + (uint32_t)acc * acc_cols;
+                const int kb0 = kb_begin(t), kb1 = kb_end(t);
+                for (int kb = kb0; kb < kb1; ++kb) {
                     if (!mbar_wait(full_bar(s), ph, abortp)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a_addr = ring + (uint32_t)s * stage_bytes;
-                    const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(a_addr + w_bytes);
+                    const uint64_t a_desc = smem_desc_sw128(a_addr), a2_desc = smem_desc_sw128(a_addr + w_bytes);
+                    const uint64_t b_desc = smem_desc_sw128(a_addr + x_off);
 #pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k)   // advance 32 bytes inside the swizzle span per UMMA_K
-                        umma_bf16(d_tmem, a_desc + (uint64_t)(k * UMMA_K * 2 >> 4), b_desc + (uint64_t)(k * UMMA_K * 2 >> 4),
-                                  idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    for (int k = 0; k < BK / UMMA_K; ++k) { // advance 32 bytes inside the swizzle span per UMMA_K
+                        const uint64_t adv = (uint64_t)(k * UMMA_K * 2 >> 4);
+                        const uint32_t accum = (kb > kb0 || k > 0) ? 1u : 0u;
+                        umma_bf16(d_tmem, a_desc + adv, b_desc + adv, idesc, accum);
+                        if (dual) umma_bf16(d_tmem + (uint32_t)BN, a2_desc + adv, b_desc + adv, idesc, accum);
+                    }
                     umma_commit(empty_bar(s));              // stage is free once these MMAs have read it
                     if (++s == S) { s = 0; ph ^= 1u; }
                 }
@@ -201,27 +229,46 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
         for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
             const int acc = it & 1;
             const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
-            const int f = (t % n_ftiles) * BM + q * 32 + lane, r0 = (t / n_ftiles) * BN;
+            const int f = (t % n_ftiles) * BM + q * 32 + lane, r0 = (t / n_ftiles % n_rtiles) * BN;
+            const int split = t / (n_ftiles * n_rtiles);
             if (!mbar_wait(acc_full_bar(acc), acc_ph, abortp)) { ok = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
-            for (int c0 = 0; c0 < BN; c0 += 32) {
+            const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * acc_cols;
+            // 16 columns (= 16 batch rows) of this thread's feature per pass keeps the epilogue's register
+            // footprint small enough for the CTA to share an SM with the attention kernel
+            for (int c0 = 0; c0 < BN; c0 += 16) {
                 if (r0 + c0 >= p.n) break;                  // warp-uniform: nothing but padding rows left
-                uint32_t v[32];
-                tmem_ld32(t_addr + (uint32_t)c0, v);
+                uint32_t v[16];
+                tmem_ld16(t_addr + (uint32_t)c0, v);
+                if (dual) {
+                    uint32_t u[16];
+                    tmem_ld16(t_addr + (uint32_t)(BN + c0), u);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (f < p.N) {
+                        __nv_bfloat16* dst = p.act + (size_t)(r0 + c0) * p.N + f;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            if (r0 + c0 + j < p.n) {
+                                const float g = __uint_as_float(v[j]);
+                                dst[(size_t)j * p.N] = __float2bfloat16_rn(g / (1.f + expf(-g)) * __uint_as_float(u[j]));
+                            }
+                        }
+                    }
+                    continue;
+                }
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 if (f < p.N) {
-                    float* dst = p.y + (size_t)(r0 + c0) * p.N + f;
-                    if (p.accumulate) {
-                        float prev[32];                      // all residual loads in flight before the first add
+                    float* dst = p.y + (size_t)split * p.split_stride + (size_t)(r0 + c0) * p.N + f;
+                    if (p.mode == kModeAccumulate) {
+                        float prev[16];                      // all residual loads in flight before the first add
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) prev[j] = (r0 + c0 + j < p.n) ? __ldcg(dst + (size_t)j * p.N) : 0.f;
+                        for (int j = 0; j < 16; ++j) prev[j] = (r0 + c0 + j < p.n) ? __ldcg(dst + (size_t)j * p.N) : 0.f;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
+                        for (int j = 0; j < 16; ++j)
                             if (r0 + c0 + j < p.n) dst[(size_t)j * p.N] = prev[j] + __uint_as_float(v[j]);
                     } else {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
+                        for (int j = 0; j < 16; ++j)
                             if (r0 + c0 + j < p.n) dst[(size_t)j * p.N] = __uint_as_float(v[j]);
                     }
                 }
@@ -275,40 +322,71 @@ bool linear_tc_supported(const cdb* h, int n, int N, int K) {
     return n >= 1 && N >= 1 && K % 8 == 0 && encode_fn() != nullptr;
 }
 
-bool launch_linear_tc(const cdb* h, const void* x, const void* W, float* y, int n, int N, int K, Epilogue ep, cudaStream_t st) {
+// Common launcher.  W2 / act only in SwiGLU mode.  k_splits > 1 only with kModeStore (y = workspace).
+static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* W2, float* y, __nv_bfloat16* act, int n,
+                        int N, int K, int mode, int k_splits, size_t split_stride, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
         cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (getenv("CDB_GEMM_CARVEOUT"))
+            cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, atoi(getenv("CDB_GEMM_CARVEOUT")));
         attr_set = true;
     }
     GemmParams p;
-    p.y = y; p.n = n; p.N = N; p.K = K;
+    p.y = y; p.act = act; p.n = n; p.N = N; p.K = K; p.mode = mode; p.k_splits = k_splits; p.split_stride = split_stride;
     int sms = 148, dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    // Rows per tile: as wide as possible (fewest re-reads of W through L2) while there are still about
-    // as many tiles as SMs; a narrower tile only helps when the wide one would leave SMs idle.
     const int n_ft = (N + BM - 1) / BM;
     static const int forced_bn = getenv("CDB_GEMM_BN") ? atoi(getenv("CDB_GEMM_BN")) : 0;     // tuning aid
+    const int bn_max = mode == kModeSwiGLU ? 128 : 256;
+    // Rows per tile: the width that minimises (waves of tiles over the SMs) x (bytes a tile pulls per k-block).
     p.BN = 64;
-    for (int bn = 256; bn >= 64; bn >>= 1) {
+    long best = -1;
+    for (int bn = bn_max; bn >= 64; bn >>= 1) {
         if (bn / 2 >= n && bn > 64) continue;                       // tile wider than needed for n rows
-        const int tiles = n_ft * ((n + bn - 1) / bn);
-        if (tiles >= sms / 2 + sms / 8 || bn == 64) { p.BN = bn; break; }
+        const int tiles = n_ft * ((n + bn - 1) / bn) * k_splits;
+        const long cost = (long)((tiles + sms - 1) / sms) * ((mode == kModeSwiGLU ? 2 : 1) * BM + bn);
+        if (best < 0 || cost < best) { best = cost; p.BN = bn; }
     }
-    if (forced_bn == 64 || forced_bn == 128 || forced_bn == 256) p.BN = forced_bn;
-    const int stage_bytes = BM * BK * 2 + p.BN * BK * 2;
-    p.stages = (kMaxSmem - 1024) / stage_bytes;
+    if ((forced_bn == 64 || forced_bn == 128 || forced_bn == 256) && forced_bn <= bn_max) p.BN = forced_bn;
+    const int stage_bytes = (mode == kModeSwiGLU ? 2 : 1) * BM * BK * 2 + p.BN * BK * 2;
+    static const int smem_cap = getenv("CDB_GEMM_SMEM_KB") ? atoi(getenv("CDB_GEMM_SMEM_KB")) * 1024 : kMaxSmem;   // tuning aid
+    int budget = smem_cap < kMaxSmem ? smem_cap : kMaxSmem;
+    if (h->gemm_smem_cap > 0 && h->gemm_smem_cap < budget) budget = h->gemm_smem_cap;
+    p.stages = (budget - 1024) / stage_bytes;
+    if (p.stages < 2) p.stages = 2;
     if (p.stages > 8) p.stages = 8;
-    p.accumulate = ep == Epilogue::ResidualAdd ? 1 : 0;
     p.status = h->status;
-    CUtensorMap map_w, map_x;
+    CUtensorMap map_w, map_w2, map_x;
     if (!make_map(&map_w, W, N, K, BM) || !make_map(&map_x, x, n, K, p.BN)) return false;
-    const int n_tiles = ((N + BM - 1) / BM) * ((n + p.BN - 1) / p.BN);
+    if (!make_map(&map_w2, W2 ? W2 : W, N, K, BM)) return false;
+    const int n_tiles = n_ft * ((n + p.BN - 1) / p.BN) * k_splits;
     const int grid = n_tiles < sms ? n_tiles : sms;
     const size_t smem = (size_t)p.stages * stage_bytes + 1024;
-    gemm_bf16_tcgen05_kernel<<<grid, kThreads, smem, st>>>(map_w, map_x, p);
+    launch_pdl(gemm_bf16_tcgen05_kernel, dim3(grid), dim3(kThreads), smem, st, map_w, map_w2, map_x, p);
     return true;
+}
+
+bool launch_linear_tc(const cdb* h, const void* x, const void* W, float* y, int n, int N, int K, Epilogue ep, cudaStream_t st) {
+    return launch_gemm(h, x, W, nullptr, y, nullptr, n, N, K, ep == Epilogue::ResidualAdd ? kModeAccumulate : kModeStore, 1, 0, st);
+}
+
+// act[n,F] (bf16) = SiLU(x.Wg^T) * (x.Wu^T): both projections in one launch, SwiGLU in the epilogue.
+bool launch_gate_up_swiglu_tc(const cdb* h, const void* x, const void* Wg, const void* Wu, void* act, int n, int F, int K, cudaStream_t st) {
+    return launch_gemm(h, x, Wg, Wu, nullptr, (__nv_bfloat16*)act, n, F, K, kModeSwiGLU, 1, 0, st);
+}
+
+// Split-K: partial products ws[s][n][N] (fp32), s < returned split count; the caller reduces them in
+// split order (deterministic).
+int launch_linear_splitk_tc(const cdb* h, const void* x, const void* W, float* ws, int max_splits, int n, int N, int K, cudaStream_t st) {
+    // The part count depends on K alone, never on the number of rows, so that a row's result does not
+    // depend on the batch it is computed in.
+    (void)n;
+    int splits = (K + BK - 1) / BK / 8;                              // at least eight k-blocks per part
+    if (splits > max_splits) splits = max_splits;
+    if (splits < 1) splits = 1;
+    return launch_gemm(h, x, W, nullptr, ws, nullptr, n, N, K, kModeStore, splits, (size_t)n * N, st) ? splits : 0;
 }
 
 }  // namespace cdbk

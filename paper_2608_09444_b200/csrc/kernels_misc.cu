@@ -36,6 +36,8 @@ template <typename T>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain,
                                                       T* __restrict__ out, const int32_t* __restrict__ seq_id,
                                                       int d, float eps) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float red[8];
     const int row = blockIdx.x;
     const bool pad = seq_id != nullptr && seq_id[row] < 0;
@@ -56,9 +58,60 @@ void launch_rmsnorm(const cdb* h, const float* x, const float* gain, void* out, 
     CDB_LAUNCH(h);
     if (rows.n_rows <= 0) return;
     if (h->cfg.dtype == CDB_FP32)
-        rmsnorm_kernel<float><<<rows.n_rows, 256, 0, st>>>(x, gain, (float*)out, rows.seq_id, h->cfg.d, h->cfg.eps);
+        launch_pdl(rmsnorm_kernel<float>, dim3(rows.n_rows), dim3(256), 0, st, x, gain, (float*)out, rows.seq_id, h->cfg.d, h->cfg.eps);
     else
-        rmsnorm_kernel<__nv_bfloat16><<<rows.n_rows, 256, 0, st>>>(x, gain, (__nv_bfloat16*)out, rows.seq_id, h->cfg.d, h->cfg.eps);
+        launch_pdl(rmsnorm_kernel<__nv_bfloat16>, dim3(rows.n_rows), dim3(256), 0, st, x, gain, (__nv_bfloat16*)out, rows.seq_id, h->cfg.d, h->cfg.eps);
+}
+
+// ------------------------------------------------------------------------------- split-K reduce + residual + RMSNorm
+// x[row] += ws[0][row] + ws[1][row] + ... (fixed order); when gain != NULL also out[row] = RMSNorm(x[row]) * gain,
+// i.e. the normed input of the projection that follows.  d <= 24 * 256.
+template <typename T>
+__global__ void __launch_bounds__(256) reduce_residual_norm_kernel(const float* __restrict__ ws, int splits, size_t split_stride,
+                                                                   float* __restrict__ x, const float* __restrict__ gain,
+                                                                   T* __restrict__ out, const int32_t* __restrict__ seq_id,
+                                                                   int d, float eps) {
+    pdl_trigger();
+    pdl_wait();
+    __shared__ float red[8];
+    constexpr int MAXV = 24;
+    const int row = blockIdx.x;
+    if (seq_id != nullptr && seq_id[row] < 0) {
+        if (gain) for (int i = threadIdx.x; i < d; i += 256) out[(size_t)row * d + i] = from_f32<T>(0.f);
+        return;
+    }
+    float v[MAXV];
+    float ss = 0.f;
+#pragma unroll
+    for (int k = 0; k < MAXV; ++k) {
+        const int i = threadIdx.x + 256 * k;
+        if (i < d) {
+            const size_t at = (size_t)row * d + i;
+            float a = x[at];
+            for (int s = 0; s < splits; ++s) a += ws[(size_t)s * split_stride + at];
+            x[at] = a;
+            v[k] = a;
+            ss = fmaf(a, a, ss);
+        }
+    }
+    if (!gain) return;
+    ss = block_sum<256>(ss, red);
+    const float inv = rsqrtf(ss / (float)d + eps);
+#pragma unroll
+    for (int k = 0; k < MAXV; ++k) {
+        const int i = threadIdx.x + 256 * k;
+        if (i < d) out[(size_t)row * d + i] = from_f32<T>(v[k] * inv * gain[i]);
+    }
+}
+
+void launch_reduce_residual_norm(const cdb* h, const float* ws, int splits, size_t split_stride, float* x, const float* gain,
+                                 void* out, const RowsDev& rows, cudaStream_t st) {
+    if (rows.n_rows <= 0) return;
+    CDB_LAUNCH(h);
+    if (h->cfg.dtype == CDB_FP32)
+        launch_pdl(reduce_residual_norm_kernel<float>, dim3(rows.n_rows), dim3(256), 0, st, ws, splits, split_stride, x, gain, (float*)out, rows.seq_id, h->cfg.d, h->cfg.eps);
+    else
+        launch_pdl(reduce_residual_norm_kernel<__nv_bfloat16>, dim3(rows.n_rows), dim3(256), 0, st, ws, splits, split_stride, x, gain, (__nv_bfloat16*)out, rows.seq_id, h->cfg.d, h->cfg.eps);
 }
 
 // ------------------------------------------------------------------------------- RoPE + KV write
@@ -70,6 +123,8 @@ __global__ void __launch_bounds__(256) rope_kv_write_kernel(const float* __restr
                                                             const float* __restrict__ rope_cos,
                                                             const float* __restrict__ rope_sin, int d,
                                                             int max_position, int max_seqs, int32_t* status) {
+    pdl_trigger();
+    pdl_wait();
     const int row = blockIdx.x;
     const int seq = rows.seq_id[row];
     if (seq < 0) return;
@@ -99,36 +154,38 @@ __global__ void __launch_bounds__(256) rope_kv_write_kernel(const float* __restr
     }
 }
 
-void launch_rope_kv_write(const cdb* h, int layer, const RowsDev& rows, cudaStream_t st) {
+void launch_rope_kv_write(const cdb* h, int ln, int layer, const RowsDev& rows, cudaStream_t st) {
     CDB_LAUNCH(h);
     if (rows.n_rows <= 0) return;
     if (h->cfg.dtype == CDB_FP32)
-        rope_kv_write_kernel<float><<<rows.n_rows, 256, 0, st>>>(h->qkv, (float*)h->qrot, h->pool, rows, layer,
+        launch_pdl(rope_kv_write_kernel<float>, dim3(rows.n_rows), dim3(256), 0, st, h->lane[ln].qkv, (float*)h->lane[ln].qrot, h->pool, rows, layer,
             h->rope_cos, h->rope_sin, h->cfg.d, h->cfg.max_position, h->cfg.max_seqs, h->status);
     else
-        rope_kv_write_kernel<__nv_bfloat16><<<rows.n_rows, 256, 0, st>>>(h->qkv, (__nv_bfloat16*)h->qrot, h->pool, rows,
+        launch_pdl(rope_kv_write_kernel<__nv_bfloat16>, dim3(rows.n_rows), dim3(256), 0, st, h->lane[ln].qkv, (__nv_bfloat16*)h->lane[ln].qrot, h->pool, rows,
             layer, h->rope_cos, h->rope_sin, h->cfg.d, h->cfg.max_position, h->cfg.max_seqs, h->status);
 }
 
 // ------------------------------------------------------------------------------- SwiGLU
-// act = SiLU(g) * u, rounded to T.  g = gu[0], u = gu[1], each [max_rows][F] fp32.
+// act = SiLU(g) * u, rounded to T.  g = gu[0], u = gu[1], each [rows_cap][F] fp32.
 template <typename T>
 __global__ void swiglu_kernel(const float* __restrict__ g, const float* __restrict__ u, T* __restrict__ act, size_t n) {
+    pdl_trigger();
+    pdl_wait();
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         const float a = g[i];
         act[i] = from_f32<T>(a / (1.f + expf(-a)) * u[i]);
     }
 }
 
-void launch_swiglu(const cdb* h, int n_rows, cudaStream_t st) {
+void launch_swiglu(const cdb* h, int ln, int n_rows, cudaStream_t st) {
     CDB_LAUNCH(h);
     if (n_rows <= 0) return;
     const size_t n = (size_t)n_rows * h->cfg.F;
     const int blocks = (int)((n + 255) / 256 < 148 * 8 ? (n + 255) / 256 : 148 * 8);
-    const float* g = h->gu;
-    const float* u = h->gu + (size_t)h->cfg.max_rows * h->cfg.F;
-    if (h->cfg.dtype == CDB_FP32) swiglu_kernel<float><<<blocks, 256, 0, st>>>(g, u, (float*)h->act, n);
-    else swiglu_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(g, u, (__nv_bfloat16*)h->act, n);
+    const float* g = h->lane[ln].gu;
+    const float* u = h->lane[ln].gu + (size_t)h->lane[ln].rows_cap * h->cfg.F;
+    if (h->cfg.dtype == CDB_FP32) launch_pdl(swiglu_kernel<float>, dim3(blocks), dim3(256), 0, st, g, u, (float*)h->lane[ln].act, n);
+    else launch_pdl(swiglu_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, g, u, (__nv_bfloat16*)h->lane[ln].act, n);
 }
 
 // ------------------------------------------------------------------------------- embedding
@@ -137,6 +194,8 @@ __global__ void __launch_bounds__(256) embed_kernel(const T* __restrict__ table,
                                                     const int32_t* __restrict__ seq_id, float* __restrict__ out, int d,
                                                     int V, int max_seqs, float* gate_S, uint8_t* gate_fire, int reset,
                                                     int32_t* status) {
+    pdl_trigger();
+    pdl_wait();
     const int row = blockIdx.x;
     const int seq = seq_id ? seq_id[row] : 0;
     float* o = out + (size_t)row * d;
@@ -155,10 +214,10 @@ void launch_embed(const cdb* h, const int32_t* tokens, const RowsDev& rows, floa
     CDB_LAUNCH(h);
     if (rows.n_rows <= 0) return;
     if (h->cfg.dtype == CDB_FP32)
-        embed_kernel<float><<<rows.n_rows, 256, 0, st>>>((const float*)h->w.embed, tokens, rows.seq_id, out, h->cfg.d,
+        launch_pdl(embed_kernel<float>, dim3(rows.n_rows), dim3(256), 0, st, (const float*)h->w.embed, tokens, rows.seq_id, out, h->cfg.d,
             h->cfg.V, h->cfg.max_seqs, h->gate_S, h->gate_fire, reset_gate ? 1 : 0, h->status);
     else
-        embed_kernel<__nv_bfloat16><<<rows.n_rows, 256, 0, st>>>((const __nv_bfloat16*)h->w.embed, tokens, rows.seq_id, out,
+        launch_pdl(embed_kernel<__nv_bfloat16>, dim3(rows.n_rows), dim3(256), 0, st, (const __nv_bfloat16*)h->w.embed, tokens, rows.seq_id, out,
             h->cfg.d, h->cfg.V, h->cfg.max_seqs, h->gate_S, h->gate_fire, reset_gate ? 1 : 0, h->status);
 }
 
@@ -169,6 +228,8 @@ __global__ void __launch_bounds__(256) gate_kernel(const float* __restrict__ x, 
                                                    float eps, float b_gate, float q_or_eps, int max_seqs,
                                                    float* gate_S, uint8_t* gate_fire, float* gate_val_out,
                                                    uint8_t* fire_out) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float red[8];
     const int row = blockIdx.x;
     const int seq = rows.seq_id[row];
@@ -210,7 +271,7 @@ void launch_gate(const cdb* h, const RowsDev& rows, const float* x, const float*
                  uint8_t* fire_out, cudaStream_t st) {
     CDB_LAUNCH(h);
     if (rows.n_rows <= 0) return;
-    gate_kernel<<<rows.n_rows, 256, 0, st>>>(x, x_prev, h->w.w_gate, rows, h->cfg.d, h->cfg.gate_kind, h->cfg.eps,
+    launch_pdl(gate_kernel, dim3(rows.n_rows), dim3(256), 0, st, x, x_prev, h->w.w_gate, rows, h->cfg.d, h->cfg.gate_kind, h->cfg.eps,
                                              h->cfg.b_gate, h->cfg.q_or_eps, h->cfg.max_seqs, h->gate_S, h->gate_fire,
                                              gate_val_out, fire_out);
 }
@@ -223,6 +284,8 @@ __global__ void __launch_bounds__(1024) compact_kernel(RowsDev rows, const uint8
                                                        int max_seqs, int32_t* __restrict__ survivor_idx,
                                                        int32_t* __restrict__ exit_idx, int32_t* __restrict__ counts,
                                                        uint8_t* __restrict__ exit_flag) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ int warp_s[32], warp_e[32];
     __shared__ int base_s, base_e;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -275,7 +338,7 @@ __global__ void __launch_bounds__(1024) compact_kernel(RowsDev rows, const uint8
 void launch_compact(const cdb* h, const RowsDev& rows, const uint8_t* fire_prev, int32_t* survivor_idx,
                     int32_t* exit_idx, int32_t* counts, cudaStream_t st) {
     CDB_LAUNCH(h);
-    compact_kernel<<<1, 1024, 0, st>>>(rows, fire_prev, h->gate_fire, h->cfg.R, h->cfg.r_min, h->cfg.max_seqs,
+    launch_pdl(compact_kernel, dim3(1), dim3(1024), 0, st, rows, fire_prev, h->gate_fire, h->cfg.R, h->cfg.r_min, h->cfg.max_seqs,
                                        survivor_idx, exit_idx, counts, h->exit_flag);
 }
 
@@ -283,6 +346,8 @@ void launch_compact(const cdb* h, const RowsDev& rows, const uint8_t* fire_prev,
 __global__ void __launch_bounds__(256) gather_kernel(const float* __restrict__ src, const int32_t* __restrict__ idx,
                                                      const int32_t* __restrict__ count_dev, int max_count,
                                                      float* __restrict__ dst, int d) {
+    pdl_trigger();
+    pdl_wait();
     const int j = blockIdx.x;
     const int n = count_dev ? *count_dev : max_count;
     if (j >= n) return;
@@ -295,12 +360,14 @@ void launch_gather(const cdb* h, const float* src, const int32_t* idx, const int
                    float* dst, cudaStream_t st) {
     CDB_LAUNCH(h);
     if (max_count <= 0) return;
-    gather_kernel<<<max_count, 256, 0, st>>>(src, idx, count_dev, max_count, dst, h->cfg.d);
+    launch_pdl(gather_kernel, dim3(max_count), dim3(256), 0, st, src, idx, count_dev, max_count, dst, h->cfg.d);
 }
 
 // ------------------------------------------------------------------------------- greedy argmax
 // First maximum (lowest token id on ties) of each row of fp32 logits.
 __global__ void __launch_bounds__(256) argmax_kernel(const float* __restrict__ logits, int V, int32_t* __restrict__ out) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float bv[256];
     __shared__ int bi[256];
     const float* r = logits + (size_t)blockIdx.x * V;
@@ -326,7 +393,7 @@ __global__ void __launch_bounds__(256) argmax_kernel(const float* __restrict__ l
 void launch_argmax(const cdb* h, const float* logits, int n_rows, int32_t* token_out, cudaStream_t st) {
     CDB_LAUNCH(h);
     if (n_rows <= 0) return;
-    argmax_kernel<<<n_rows, 256, 0, st>>>(logits, h->cfg.V, token_out);
+    launch_pdl(argmax_kernel, dim3(n_rows), dim3(256), 0, st, logits, h->cfg.V, token_out);
 }
 
 // ------------------------------------------------------------------------------- copy-on-exit
@@ -334,6 +401,8 @@ void launch_argmax(const cdb* h, const float* logits, int n_rows, int32_t* token
 template <typename T>
 __global__ void __launch_bounds__(256) copy_on_exit_kernel(KvPool pool, RowsDev rows, const int32_t* __restrict__ exit_depth,
                                                            int layer0, int R, int max_seqs, int32_t* status) {
+    pdl_trigger();
+    pdl_wait();
     const int row = blockIdx.x, layer = layer0 + blockIdx.y;
     const int seq = rows.seq_id[row];
     if (seq < 0 || seq >= max_seqs) return;
@@ -361,9 +430,9 @@ void launch_copy_on_exit(const cdb* h, const RowsDev& rows, const int32_t* exit_
     if (rows.n_rows <= 0 || h->cfg.L_core <= 0) return;
     dim3 grid(rows.n_rows, h->cfg.L_core);
     if (h->cfg.dtype == CDB_FP32)
-        copy_on_exit_kernel<float><<<grid, 256, 0, st>>>(h->pool, rows, exit_depth, h->cfg.L_pre, h->cfg.R, h->cfg.max_seqs, h->status);
+        launch_pdl(copy_on_exit_kernel<float>, dim3(grid), dim3(256), 0, st, h->pool, rows, exit_depth, h->cfg.L_pre, h->cfg.R, h->cfg.max_seqs, h->status);
     else
-        copy_on_exit_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(h->pool, rows, exit_depth, h->cfg.L_pre, h->cfg.R, h->cfg.max_seqs, h->status);
+        launch_pdl(copy_on_exit_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, st, h->pool, rows, exit_depth, h->cfg.L_pre, h->cfg.R, h->cfg.max_seqs, h->status);
 }
 
 }  // namespace cdbk

@@ -266,6 +266,35 @@ def test_loop_step_rows_match_oracle(dims, gate_kind):
     assert near <= 1
 
 
+def test_two_stream_half_batches_equal_the_single_stream_step():
+    """With the two-stream flag a loop step of 64+ rows runs as two half-batches on two streams; rows are independent, so the
+    result must be bit-identical to the one-batch step (states, gate values, signals, KV pages)."""
+    binding = B()
+    dims = synth.Dims(V=64, d=256, H=2, Dh=128, F=320, L_pre=0, L_core=3, L_coda=0, R=4, dtype="bf16")
+    wd, _ = make_model(dims, 23, gate_std=0.1)
+    n = 101
+    rng = np.random.default_rng(10)
+    ctxs = rng.integers(1, 400, n)
+    table_np, n_pages = synth.make_page_table(ctxs, 16, seed=3)
+    pool_np = synth.to_bf16_grid(rng.standard_normal(synth.kv_pool_shape(dims, n_pages)).astype(np.float32))
+    h_np = rng.standard_normal((n, dims.d)).astype(np.float32)
+    outs = []
+    for flags in (binding.FLAG_TWO_STREAM, 0):
+        cdb = binding.Cdb(dims, wd, max_rows=n, max_seqs=n, max_position=table_np.shape[1] * 16, q_or_eps=0.5, flags=flags)
+        pool = dev(pool_np, torch.bfloat16)
+        cdb.kv_bind(pool)
+        rows = rows_of(binding, np.arange(n), ctxs - 1, dev(table_np), depth=rng.integers(1, 5, n) * 0 + 2, slot=np.zeros(n))
+        h, g, f = dev(h_np), torch.zeros(n, device="cuda"), torch.zeros(n, dtype=torch.uint8, device="cuda")
+        cdb.boundary_embed(dev(np.zeros(n, dtype=np.int32)), rows, torch.zeros((n, dims.d), device="cuda"))
+        cdb.loop_step(rows, h, g, f)
+        torch.cuda.synchronize()
+        assert cdb.poll_status() == 0
+        outs.append((h.clone(), g.clone(), f.clone(), pool.clone()))
+        cdb.destroy()
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
 # ------------------------------------------------------------------ boundary: embedding, coda + LM head + greedy
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
