@@ -1,0 +1,50 @@
+"""World-size-2 check of the multi-GPU plumbing on CPU (gloo): sequence sharding is a partition, the
+timing reduction returns the slowest rank's value on every rank, and ranks draw different workloads."""
+import os
+import socket
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank))
+    from paper_2608_09444_b200 import dist as D
+    from paper_2608_09444_b200 import synth
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    assert D.env_rank() == (rank, rank, world)
+    mine = D.shard(range(11), world, rank)
+    slow = D.max_over_ranks(10.0 + rank)
+    rows = synth.make_step_rows(8, 4, D.rank_seed(1, rank))
+    dist.barrier()
+    out.put((rank, mine, slow, rows["position"].tolist()))
+    dist.destroy_process_group()
+
+
+def test_two_ranks_shard_and_reduce():
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    shards = [r[1] for r in res]
+    assert sorted(shards[0] + shards[1]) == list(range(11)) and not set(shards[0]) & set(shards[1])
+    assert abs(len(shards[0]) - len(shards[1])) <= 1
+    assert [r[2] for r in res] == [11.0, 11.0]                 # both ranks see the slowest rank's time
+    assert res[0][3] != res[1][3]                              # weak scaling: each rank has its own rows

@@ -1,0 +1,99 @@
+"""Ouro-1.4B-shaped single loop step at full size (256 ragged rows, 24 layers, 55.9 GB paged KV pool),
+in exactly the launch configuration bench.py times, against the CPU oracle:
+  * survivor / exit index lists and counts of all 256 rows: bit-exact;
+  * for a sample of rows spanning every loop depth and the context extremes, computed one by one by the
+    oracle: hidden state after the step, gate value, the k, v the step wrote into the row's page
+    (max |gpu - oracle| / max |oracle| <= 2e-2, bf16), the exit signal (values within 1e-3 of the
+    threshold excluded and counted), and for sampled exit rows the greedy token (a mismatch is accepted
+    only when the oracle's own margin between the two candidates is below twice the measured logit error).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import cdb_oracle as O
+from paper_2608_09444_b200 import synth
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2
+
+
+def rel_err(a, b):
+    a, b = np.asarray(a, dtype=np.float64).ravel(), np.asarray(b, dtype=np.float64).ravel()
+    return float(np.max(np.abs(a - b)) / max(np.max(np.abs(b)), 1e-30))
+
+
+def test_c2_full_size_step_matches_oracle_on_sampled_rows():
+    from paper_2608_09444_b200.workloads import LoopStepWorkload
+    wl = LoopStepWorkload(synth.OURO_1P4B, n_rows=256, seed=1)
+    dm = wl.dims
+    r = wl.rows_np
+    # ---- sample: shortest and longest context, one row per loop depth, two exits, two survivors
+    flags = np.array([O.exit_now(int(r["loop_depth"][i]), dm.R, int(r["fire_prev"][i]), 0, 1) for i in range(256)])
+    sample = {int(np.argmin(wl.ctx)), int(np.argmax(wl.ctx))}
+    for d in range(1, dm.R + 1):
+        sample.add(int(np.flatnonzero(r["loop_depth"] == d)[0]))
+    sample.update(int(i) for i in np.flatnonzero(flags)[:2])
+    sample.update(int(i) for i in np.flatnonzero(~flags)[:2])
+    sample = sorted(sample)
+    items = wl.oracle_inputs(sample)                       # before the step: the step overwrites the rows' slots
+
+    wl.step_resident()
+    torch.cuda.synchronize()
+    assert wl.cdb.poll_status() == 0
+
+    # ---- integer outputs of all rows
+    want_s, want_e = O.stable_partition(list(flags), [True] * 256)
+    counts = wl.counts.cpu().numpy()
+    assert (int(counts[0]), int(counts[1])) == (len(want_s), len(want_e)) == (wl.n_surv, wl.n_exit)
+    assert np.array_equal(wl.surv_idx.cpu().numpy()[:len(want_s)], want_s)
+    assert np.array_equal(wl.exit_idx.cpu().numpy()[:len(want_e)], want_e)
+    h = wl.h.cpu().numpy()
+    assert np.array_equal(wl.h_next.cpu().numpy()[:len(want_s)], h[want_s])         # gathers are exact copies
+    assert np.array_equal(wl.h_exit.cpu().numpy()[:len(want_e)], h[want_e])
+
+    # ---- sampled rows against the oracle
+    wn = synth.weights_to_numpy(wl.weights)
+    orc = O.Oracle(dm, wn, gate_kind=O.GATE_SIGMOID_CDF, q_or_eps=0.5)
+    gate_val, fire = wl.gate_val.cpu().numpy(), wl.fire.cpu().numpy()
+    tokens = wl.tokens.cpu().numpy()
+    exit_pos = {int(row): j for j, row in enumerate(want_e)}
+    worst_h = worst_kv = worst_logit = 0.0
+    near_threshold = explained = 0
+    for it in items:
+        i, c = it["row"], it["ctx"]
+        kv = [O.gather_pages(it["pages"][l], it["table"], c) for l in range(dm.L_core)]
+        Ks, Vs = [k for k, _ in kv], [v for _, v in kv]
+        h_ref, g_ref, f_ref, _, new_kv = orc.loop_step_row(it["h"], c - 1, it["depth"], Ks, Vs)
+        worst_h = max(worst_h, rel_err(h[i], h_ref))
+        assert abs(gate_val[i] - g_ref) <= TOL
+        if abs(g_ref - 0.5) < 1e-3:
+            near_threshold += 1
+        else:
+            assert bool(fire[i]) == f_ref, i
+        page, off = int(wl.table_np[i, (c - 1) // 16]), (c - 1) % 16
+        got = wl.pool[:, page, :, :, off, :].float().cpu().numpy()                  # [L][2][H][Dh]
+        for l in range(dm.L_core):
+            worst_kv = max(worst_kv, rel_err(got[l, 0], new_kv[l][0]), rel_err(got[l, 1], new_kv[l][1]))
+        if i in exit_pos:
+            logits_ref = orc.round(O.rmsnorm(h_ref, orc.w["g_final"], dm.eps)) @ orc.w["W_lm"].T
+            # the GPU's own logits for this row (the bench path does not keep them): one more LM-head call
+            j = exit_pos[i]
+            lg = torch.zeros((1, dm.V), device="cuda")
+            tk = torch.zeros(1, dtype=torch.int32, device="cuda")
+            from paper_2608_09444_b200 import binding as B
+            one = B.Rows(wl.exit_seq[j:j + 1].contiguous(), wl.exit_pos[j:j + 1].contiguous(), wl.d_in["page_table"])
+            wl.cdb.boundary_coda_lmhead(one, wl.h_exit[j:j + 1].clone(), tk, lg)
+            torch.cuda.synchronize()
+            lg = lg[0].cpu().numpy()
+            assert int(tk[0]) == int(tokens[j])                                     # a row alone = the row in the batch
+            worst_logit = max(worst_logit, rel_err(lg, logits_ref))
+            want_tok = int(np.argmax(logits_ref))
+            if int(tokens[j]) != want_tok:
+                margin = logits_ref[want_tok] - logits_ref[int(tokens[j])]
+                assert margin < 2 * np.max(np.abs(lg - logits_ref)), (i, margin)
+                explained += 1
+    print(f"sampled rows {sample}: hidden {worst_h:.2e}, kv {worst_kv:.2e}, logits {worst_logit:.2e}; "
+          f"near-threshold gates excluded {near_threshold}, near-tie tokens {explained}")
+    assert worst_h <= TOL and worst_kv <= TOL and worst_logit <= TOL
+    assert near_threshold <= 1 and explained <= 1
