@@ -82,7 +82,7 @@ void layer_forward(cdb_t* h, int ln, int layer, const RowsDev& rows, float* x, c
     const size_t d = c.d, F = c.F;
     launch_rmsnorm(h, x, h->g_attn + (size_t)layer * d, L.xn, rows, st);
     launch_linear(h, L.xn, layer_ptr(h, h->w.W_qkv, layer, 3 * d * d), L.qkv, n, 3 * c.d, c.d, Epilogue::Store, st);
-    launch_rope_kv_write(h, ln, layer, rows, st);
+    launch_rope_kv_write(h, ln, layer, L.qkv, 1, 0, rows, st);
     if (attn_after) cudaStreamWaitEvent(st, attn_after, 0);      // the other half-batch's attention goes first
     h->attn_split_done = attn_done;
     launch_attention(h, ln, layer, rows, L.qrot, L.attn_o, st);
@@ -107,8 +107,13 @@ void layer_forward_tc(cdb_t* h, int ln, int layer, const RowsDev& rows, float* x
     const int n = rows.n_rows;
     const size_t d = c.d, F = c.F;
     if (!xn_ready) launch_rmsnorm(h, x, h->g_attn + (size_t)layer * d, L.xn, rows, st);
-    launch_linear(h, L.xn, layer_ptr(h, h->w.W_qkv, layer, 3 * d * d), L.qkv, n, 3 * c.d, c.d, Epilogue::Store, st);
-    launch_rope_kv_write(h, ln, layer, rows, st);
+    {
+        ProfScope ps(h, kProfLinear, st);
+        CDB_LAUNCH(h);
+        const int s = launch_linear_splitk_tc(h, L.xn, layer_ptr(h, h->w.W_qkv, layer, 3 * d * d), L.ws, kWsPerRow / 3, n, 3 * c.d, c.d, st);
+        if (!s) h->launch_error = 1;
+        launch_rope_kv_write(h, ln, layer, L.ws, s, (size_t)n * 3 * d, rows, st);      // sums the parts
+    }
     if (attn_after) cudaStreamWaitEvent(st, attn_after, 0);      // the other half-batch's attention goes first
     h->attn_split_done = attn_done;
     launch_attention(h, ln, layer, rows, L.qrot, L.attn_o, st);
@@ -171,6 +176,8 @@ void free_all(cdb_t* h) {
         void* lp[] = {L.xn, L.qrot, L.attn_o, L.act, L.qkv, L.gu, L.ws, L.attn_part, L.attn_item_start, L.attn_counters};
         for (void* p : lp) if (p) cudaFree(p);
     }
+    for (int i = 0; i < h->n_tiled; ++i) if (h->tiled[i].tiled) cudaFree(h->tiled[i].tiled);
+    h->n_tiled = 0;
     if (h->side) cudaStreamDestroy(h->side);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
@@ -248,7 +255,7 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
         CDB_ALLOC(L.act, char, r * F * h->elem_size);
         CDB_ALLOC(L.qkv, float, r * 3 * d);
         CDB_ALLOC(L.gu, float, r * 2 * F);
-        CDB_ALLOC(L.ws, float, (size_t)kMaxKSplits * r * d);
+        CDB_ALLOC(L.ws, float, (size_t)kWsPerRow * r * d);
         CDB_ALLOC(L.attn_part, float, r * c.H * h->max_splits * (size_t)(c.Dh + 2));
         CDB_ALLOC(L.attn_item_start, int32_t, r + 1);
         CDB_ALLOC(L.attn_counters, int32_t, n_layers);
@@ -275,6 +282,20 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
         }
         e = cudaMemcpy(h->rope_cos, cs.data(), cs.size() * sizeof(float), cudaMemcpyHostToDevice);
         if (e == cudaSuccess) e = cudaMemcpy(h->rope_sin, sn.data(), sn.size() * sizeof(float), cudaMemcpyHostToDevice);
+    }
+    if (e == cudaSuccess && c.dtype == CDB_BF16 && !(c.flags & CDB_FLAG_SIMT_GEMM)) {
+        // tile-major copies of the projection weights (the caller's row-major tensors stay borrowed)
+        struct { const void* p; int layers, N, K; } stacks[6] = {
+            {w->W_qkv, L, 3 * c.d, c.d}, {w->W_o, L, c.d, c.d}, {w->W_gate, L, c.F, c.d},
+            {w->W_up, L, c.F, c.d}, {w->W_down, L, c.d, c.F}, {w->W_lm, 1, c.V, c.d}};
+        for (int i = 0; i < 6 && e == cudaSuccess; ++i) {
+            TiledWeight& t = h->tiled[h->n_tiled];
+            t.orig = (const char*)stacks[i].p; t.layers = stacks[i].layers; t.N = stacks[i].N; t.K = stacks[i].K;
+            e = cudaMalloc((void**)&t.tiled, tiled_weight_bytes(t.layers, t.N, t.K));
+            if (e != cudaSuccess) { t.tiled = nullptr; break; }
+            ++h->n_tiled;
+            launch_repack_tiled(t.orig, t.tiled, t.layers, t.N, t.K, 0);
+        }
     }
     if (e == cudaSuccess) {
         gains_to_f32(h, w->g_attn, h->g_attn, (size_t)L * d);

@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
 
 #include "cdb.h"
 
@@ -11,7 +12,8 @@ namespace cdbk {
 
 constexpr int kPageSize = 16;        // tokens per KV page
 constexpr int kSplitTokens = 256;    // attention split length; depends on nothing but the row's own context
-constexpr int kMaxKSplits = 4;       // split-K parts of the residual projections
+constexpr int kMaxKSplits = 8;       // most split-K parts of a projection
+constexpr int kWsPerRow = 12;        // workspace floats per row, in units of d: 8 parts of [d] or 3 parts of [3d] fit
 constexpr int kStatusPage = 1, kStatusPosition = 2, kStatusSeq = 3;
 
 enum class Epilogue : int { Store = 0, ResidualAdd = 1 };
@@ -51,13 +53,21 @@ struct Lane {
     void* act;                      // [rows_cap][F] SwiGLU output (dtype)
     float* qkv;                     // [rows_cap][3d]
     float* gu;                      // [2][rows_cap][F] gate and up projections
-    float* ws;                      // [kMaxKSplits][rows_cap][d] split-K partial products
+    float* ws;                      // [rows_cap * kWsPerRow * d] split-K partial products [part][row][features]
     float* attn_part;               // [rows_cap*H*max_splits][Dh + 2] split partials (o, m, l)
     int32_t* attn_item_start;       // [rows_cap + 1] exclusive scan of splits per row
     int32_t* attn_counters;         // [L] work-fetch counters
 };
 
 }  // namespace cdbk
+
+// A weight stack and its tile-major copy: [layer][feature tile][k block][128 rows][64 columns] bf16, zero padded,
+// so that the [128 x 64] tile a projection CTA pulls per k-block is 16 KB of contiguous HBM.
+struct TiledWeight {
+    const char* orig;           // caller's row-major stack [layers][N][K]
+    char* tiled;                // library-owned copy
+    int layers, N, K;
+};
 
 struct cdb {
     cdb_config_t cfg;
@@ -74,6 +84,9 @@ struct cdb {
     float* g_final;                 // [d]
     float* gate_S;                  // [max_seqs] survival of the cumulative exit probability
     uint8_t* gate_fire;             // [max_seqs] stored exit signal
+    TiledWeight tiled[6];           // W_qkv, W_o, W_gate, W_up, W_down, W_lm (bf16 configs)
+    int n_tiled;
+
     // per-lane scratch: lane 0 holds max_rows rows, lane 1 half of that (second half-batch of a split step)
     cdbk::Lane lane[2];
     float* h_prev;                  // [max_rows][d] state at step entry (convergence gate)
@@ -116,7 +129,8 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
+    static const bool no_pdl = getenv("CDB_NO_PDL") != nullptr;      // tuning aid: plain stream-ordered launches
+    cfg.attrs = attr; cfg.numAttrs = no_pdl ? 0 : 1;
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 }  // namespace cdbk
@@ -142,7 +156,7 @@ namespace cdbk {
 
 // ---- launchers (each enqueues on `st`; none synchronises) -----------------------------------
 void launch_rmsnorm(const cdb* h, const float* x, const float* gain, void* out, const RowsDev& rows, cudaStream_t st);
-void launch_rope_kv_write(const cdb* h, int ln, int layer, const RowsDev& rows, cudaStream_t st);
+void launch_rope_kv_write(const cdb* h, int ln, int layer, const float* qkv_parts, int parts, size_t part_stride, const RowsDev& rows, cudaStream_t st);
 void launch_attention(const cdb* h, int ln, int layer, const RowsDev& rows, const void* q, void* o, cudaStream_t st);
 void launch_attention_plan(const cdb* h, int ln, const RowsDev& rows, cudaStream_t st);
 void launch_swiglu(const cdb* h, int ln, int n_rows, cudaStream_t st);
@@ -160,6 +174,8 @@ void launch_copy_on_exit(const cdb* h, const RowsDev& rows, const int32_t* exit_
 void launch_reduce_residual_norm(const cdb* h, const float* ws, int splits, size_t split_stride, float* x, const float* gain,
                                  void* out, const RowsDev& rows, cudaStream_t st);
 // bf16 tensor-core variants (gemm_tcgen05.cu)
+size_t tiled_weight_bytes(int layers, int N, int K);
+void launch_repack_tiled(const void* W, void* Wt, int layers, int N, int K, cudaStream_t st);
 bool linear_tc_supported(const cdb* h, int n, int N, int K);
 bool launch_gate_up_swiglu_tc(const cdb* h, const void* x, const void* Wg, const void* Wu, void* act, int n, int F, int K, cudaStream_t st);
 int launch_linear_splitk_tc(const cdb* h, const void* x, const void* W, float* ws, int max_splits, int n, int N, int K, cudaStream_t st);

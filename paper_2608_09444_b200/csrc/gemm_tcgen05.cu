@@ -35,6 +35,14 @@ constexpr int kMaxSmem = 225 * 1024;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// One lane of a converged warp (the warp stays converged, so addresses and descriptors computed by all
+// lanes remain warp-uniform for the compiler).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred = 0;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
+
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
@@ -116,15 +124,21 @@ struct GemmParams {
     int stages;
     int mode;
     int k_splits;               // the K range is cut into this many parts, each a tile of its own
+    int w_tiled;                // weights come from the tile-major copy: tile (ft, kb) starts at row (ft * n_kb + kb) * 128
     size_t split_stride;
     int32_t* status;
+    unsigned long long* dbg;    // tuning aid: per-CTA phase time stamps (NULL = off)
+    int dbg_mode;               // tuning aid: 1 skip MMAs, 2 skip activation loads, 4 skip weight loads (results wrong)
 };
+
+__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t) :: "memory"); return t; }
 
 // at most 72 registers per thread, so that a CTA fits on an SM beside four attention CTAs
 __global__ void __maxnreg__(72)
 gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w2,
                          const __grid_constant__ CUtensorMap map_x, GemmParams p) {
     pdl_trigger();
+    if (p.dbg && threadIdx.x == 0) p.dbg[blockIdx.x * 8 + 0] = gtime();
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2 * 8 + 4];          // full[stages], empty[stages], acc_full[2], acc_empty[2]
     __shared__ uint32_t tmem_base_slot;
@@ -159,6 +173,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_slot;
     volatile int* abortp = &abort_flag;
+    if (p.dbg && threadIdx.x == 0) p.dbg[blockIdx.x * 8 + 1] = gtime();
     pdl_wait();                 // set-up above overlaps the previous kernel's tail; operands are read only from here on
 
     const int n_ftiles = (p.N + BM - 1) / BM, n_rtiles = (p.n + BN - 1) / BN;
@@ -171,30 +186,45 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
         if (lane == 0) {
             int s = 0; uint32_t ph = 0;
             bool ok = true;
+            long long prod_wait = 0, prod_issue = 0;
             for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
                 const int f0 = (t % n_ftiles) * BM, r0 = (t / n_ftiles % n_rtiles) * BN;
-                for (int kb = kb_begin(t); kb < kb_end(t); ++kb) {
+                // Every CTA walks its k-blocks from a different starting point (a function of its feature
+                // tile only), so that the CTAs do not all pull the same activation lines from L2 at once.
+                const int kb0 = kb_begin(t), nk = kb_end(t) - kb0, rot = ((t % n_ftiles) * 7) % nk;
+                for (int j = 0; j < nk; ++j) {
+                    const int kb = kb0 + (j + rot) % nk;
+                    const long long c0 = clock64();
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abortp)) { ok = false; break; }
-                    mbar_expect_tx(full_bar(s), stage_bytes);
+                    const long long c1 = clock64();
+                    prod_wait += c1 - c0;
+                    mbar_expect_tx(full_bar(s), ((p.dbg_mode & 4) ? 0 : x_off) + ((p.dbg_mode & 2) ? 0 : x_bytes) + (p.dbg_mode == 6 ? 0 : 0));
                     const uint32_t dst = ring + (uint32_t)s * stage_bytes;
-                    tma_load_2d(dst, &map_w, full_bar(s), kb * BK, f0);
-                    if (dual) tma_load_2d(dst + w_bytes, &map_w2, full_bar(s), kb * BK, f0);
-                    tma_load_2d(dst + x_off, &map_x, full_bar(s), kb * BK, r0);
+                    const int wc = p.w_tiled ? 0 : kb * BK, wr = p.w_tiled ? ((f0 / BM) * n_kb + kb) * BM : f0;
+                    if (!(p.dbg_mode & 4)) {
+                        tma_load_2d(dst, &map_w, full_bar(s), wc, wr);
+                        if (dual) tma_load_2d(dst + w_bytes, &map_w2, full_bar(s), wc, wr);
+                    }
+                    if (!(p.dbg_mode & 2)) tma_load_2d(dst + x_off, &map_x, full_bar(s), kb * BK, r0);
+                    prod_issue += clock64() - c1;
                     if (++s == S) { s = 0; ph ^= 1u; }
                 }
             }
+            if (p.dbg) { p.dbg[blockIdx.x * 8 + 5] = prod_wait; p.dbg[blockIdx.x * 8 + 7] = prod_issue; }
             if (!ok || *abortp) {                        // give copies already in flight time to land
                 for (int i = 0; i < 64; ++i) __nanosleep(1000);
             }
         }
         __syncwarp();
     } else if (warp == 1) {
-        if (lane == 0) {
+        {
+            const bool leader = elect_one();
             // instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, N = BN, M = 128
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
             int s = 0; uint32_t ph = 0;
             int it = 0;
             bool ok = true;
+            long long mma_wait = 0, mma_t0 = clock64();
             for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
                 const int acc = it & 1;
                 const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
@@ -202,8 +232,10 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = tmem_base + (uint32_t)acc * acc_cols;
                 const int kb0 = kb_begin(t), kb1 = kb_end(t);
-                for (int kb = kb0; kb < kb1; ++kb) {
+                for (int kb = kb0; kb < kb1; ++kb) {        // arrival order of the stages; which k-block is in one does not matter here
+                    const long long m0 = clock64();
                     if (!mbar_wait(full_bar(s), ph, abortp)) { ok = false; break; }
+                    mma_wait += clock64() - m0;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a_addr = ring + (uint32_t)s * stage_bytes;
                     const uint64_t a_desc = smem_desc_sw128(a_addr), a2_desc = smem_desc_sw128(a_addr + w_bytes);
@@ -212,14 +244,16 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
                     for (int k = 0; k < BK / UMMA_K; ++k) { // advance 32 bytes inside the swizzle span per UMMA_K
                         const uint64_t adv = (uint64_t)(k * UMMA_K * 2 >> 4);
                         const uint32_t accum = (kb > kb0 || k > 0) ? 1u : 0u;
-                        umma_bf16(d_tmem, a_desc + adv, b_desc + adv, idesc, accum);
-                        if (dual) umma_bf16(d_tmem + (uint32_t)BN, a2_desc + adv, b_desc + adv, idesc, accum);
+                        if (leader && !(p.dbg_mode & 1)) umma_bf16(d_tmem, a_desc + adv, b_desc + adv, idesc, accum);
+                        if (leader && dual && !(p.dbg_mode & 1)) umma_bf16(d_tmem + (uint32_t)BN, a2_desc + adv, b_desc + adv, idesc, accum);
                     }
-                    umma_commit(empty_bar(s));              // stage is free once these MMAs have read it
+                    __syncwarp();
+                    if (leader) umma_commit(empty_bar(s));  // stage is free once these MMAs have read it
                     if (++s == S) { s = 0; ph ^= 1u; }
                 }
-                if (ok) umma_commit(acc_full_bar(acc));     // accumulator complete
+                if (ok && leader) umma_commit(acc_full_bar(acc));     // accumulator complete
             }
+            if (p.dbg && leader) { p.dbg[blockIdx.x * 8 + 3] = mma_wait; p.dbg[blockIdx.x * 8 + 2] = clock64() - mma_t0; }
         }
         __syncwarp();
     } else {
@@ -232,6 +266,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
             const int f = (t % n_ftiles) * BM + q * 32 + lane, r0 = (t / n_ftiles % n_rtiles) * BN;
             const int split = t / (n_ftiles * n_rtiles);
             if (!mbar_wait(acc_full_bar(acc), acc_ph, abortp)) { ok = false; break; }
+            if (p.dbg && it == 0 && warp == 2 && lane == 0) p.dbg[blockIdx.x * 8 + 4] = gtime();
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * acc_cols;
             // 16 columns (= 16 batch rows) of this thread's feature per pass keeps the epilogue's register
@@ -275,6 +310,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
+            if (p.dbg && warp == 2 && lane == 0) p.dbg[blockIdx.x * 8 + 6] = gtime();
             if (lane == 0) mbar_arrive(acc_empty_bar(acc));
         }
     }
@@ -322,6 +358,41 @@ bool linear_tc_supported(const cdb* h, int n, int N, int K) {
     return n >= 1 && N >= 1 && K % 8 == 0 && encode_fn() != nullptr;
 }
 
+// Tile-major weight copies ----------------------------------------------------------------------------
+size_t tiled_weight_bytes(int layers, int N, int K) {
+    return (size_t)layers * ((N + BM - 1) / BM) * ((K + BK - 1) / BK) * BM * BK * sizeof(__nv_bfloat16);
+}
+
+namespace {
+__global__ void repack_tiled_kernel(const __nv_bfloat16* __restrict__ W, __nv_bfloat16* __restrict__ Wt, int layers, int N, int K) {
+    const int n_ft = (N + BM - 1) / BM, n_kb = (K + BK - 1) / BK;
+    const size_t per_layer = (size_t)n_ft * n_kb * BM * BK, total = per_layer * layers;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t l = i / per_layer, r = i % per_layer;
+        const int c = (int)(r % BK), row = (int)(r / BK % BM), kb = (int)(r / (BK * BM) % n_kb), ft = (int)(r / ((size_t)BK * BM * n_kb));
+        const int f = ft * BM + row, k = kb * BK + c;
+        Wt[i] = (f < N && k < K) ? W[l * (size_t)N * K + (size_t)f * K + k] : __float2bfloat16_rn(0.f);
+    }
+}
+
+// the tile-major copy of the [N][K] matrix at W, or NULL when W is not (a layer of) a registered stack
+const void* find_tiled(const cdb* h, const void* W, int N, int K) {
+    for (int i = 0; i < h->n_tiled; ++i) {
+        const TiledWeight& t = h->tiled[i];
+        if (t.N != N || t.K != K || !t.tiled) continue;
+        const size_t layer_bytes = (size_t)N * K * 2;
+        const char* w = (const char*)W;
+        if (w < t.orig || w >= t.orig + layer_bytes * t.layers || (size_t)(w - t.orig) % layer_bytes) continue;
+        return t.tiled + (size_t)(w - t.orig) / layer_bytes * tiled_weight_bytes(1, N, K);
+    }
+    return nullptr;
+}
+}  // namespace
+
+void launch_repack_tiled(const void* W, void* Wt, int layers, int N, int K, cudaStream_t st) {
+    repack_tiled_kernel<<<148 * 8, 256, 0, st>>>((const __nv_bfloat16*)W, (__nv_bfloat16*)Wt, layers, N, K);
+}
+
 // Common launcher.  W2 / act only in SwiGLU mode.  k_splits > 1 only with kModeStore (y = workspace).
 static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* W2, float* y, __nv_bfloat16* act, int n,
                         int N, int K, int mode, int k_splits, size_t split_stride, cudaStream_t st) {
@@ -340,15 +411,9 @@ static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* 
     const int n_ft = (N + BM - 1) / BM;
     static const int forced_bn = getenv("CDB_GEMM_BN") ? atoi(getenv("CDB_GEMM_BN")) : 0;     // tuning aid
     const int bn_max = mode == kModeSwiGLU ? 128 : 256;
-    // Rows per tile: the width that minimises (waves of tiles over the SMs) x (bytes a tile pulls per k-block).
-    p.BN = 64;
-    long best = -1;
-    for (int bn = bn_max; bn >= 64; bn >>= 1) {
-        if (bn / 2 >= n && bn > 64) continue;                       // tile wider than needed for n rows
-        const int tiles = n_ft * ((n + bn - 1) / bn) * k_splits;
-        const long cost = (long)((tiles + sms - 1) / sms) * ((mode == kModeSwiGLU ? 2 : 1) * BM + bn);
-        if (best < 0 || cost < best) { best = cost; p.BN = bn; }
-    }
+    // Rows per tile (MMA N): the widest of 64 / 128 / 256 the batch can fill: one tcgen05.mma then does the
+    // most work per issue and each weight tile is pulled through L2 the fewest times.
+    p.BN = n <= 64 ? 64 : (n <= 128 || bn_max == 128) ? 128 : 256;
     if ((forced_bn == 64 || forced_bn == 128 || forced_bn == 256) && forced_bn <= bn_max) p.BN = forced_bn;
     const int stage_bytes = (mode == kModeSwiGLU ? 2 : 1) * BM * BK * 2 + p.BN * BK * 2;
     static const int smem_cap = getenv("CDB_GEMM_SMEM_KB") ? atoi(getenv("CDB_GEMM_SMEM_KB")) * 1024 : kMaxSmem;   // tuning aid
@@ -358,9 +423,19 @@ static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* 
     if (p.stages < 2) p.stages = 2;
     if (p.stages > 8) p.stages = 8;
     p.status = h->status;
+    p.dbg_mode = getenv("CDB_GEMM_DBGMODE") ? atoi(getenv("CDB_GEMM_DBGMODE")) : 0;
+    p.dbg = getenv("CDB_GEMM_DBG") ? (unsigned long long*)strtoull(getenv("CDB_GEMM_DBG"), nullptr, 0) : nullptr;
     CUtensorMap map_w, map_w2, map_x;
-    if (!make_map(&map_w, W, N, K, BM) || !make_map(&map_x, x, n, K, p.BN)) return false;
-    if (!make_map(&map_w2, W2 ? W2 : W, N, K, BM)) return false;
+    const int n_kb = (K + BK - 1) / BK;
+    const void* Wt = find_tiled(h, W, N, K);
+    const void* Wt2 = W2 ? find_tiled(h, W2, N, K) : Wt;
+    p.w_tiled = (Wt && Wt2) ? 1 : 0;
+    if (p.w_tiled) {
+        if (!make_map(&map_w, Wt, n_ft * n_kb * BM, BK, BM) || !make_map(&map_w2, Wt2, n_ft * n_kb * BM, BK, BM)) return false;
+    } else {
+        if (!make_map(&map_w, W, N, K, BM) || !make_map(&map_w2, W2 ? W2 : W, N, K, BM)) return false;
+    }
+    if (!make_map(&map_x, x, n, K, p.BN)) return false;
     const int n_tiles = n_ft * ((n + p.BN - 1) / p.BN) * k_splits;
     const int grid = n_tiles < sms ? n_tiles : sms;
     const size_t smem = (size_t)p.stages * stage_bytes + 1024;
@@ -380,10 +455,16 @@ bool launch_gate_up_swiglu_tc(const cdb* h, const void* x, const void* Wg, const
 // Split-K: partial products ws[s][n][N] (fp32), s < returned split count; the caller reduces them in
 // split order (deterministic).
 int launch_linear_splitk_tc(const cdb* h, const void* x, const void* W, float* ws, int max_splits, int n, int N, int K, cudaStream_t st) {
-    // The part count depends on K alone, never on the number of rows, so that a row's result does not
-    // depend on the batch it is computed in.
+    // The part count depends on the weight's shape alone, never on the number of rows, so that a row's
+    // result does not depend on the batch it is computed in: about one tile per SM for a batch that
+    // fills one row tile, and at least four k-blocks per part.
     (void)n;
-    int splits = (K + BK - 1) / BK / 8;                              // at least eight k-blocks per part
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int n_ft = (N + BM - 1) / BM, n_kb = (K + BK - 1) / BK;
+    int splits = (sms + n_ft / 2) / n_ft;
+    if (splits > n_kb / 4) splits = n_kb / 4;
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
     return launch_gemm(h, x, W, nullptr, ws, nullptr, n, N, K, kModeStore, splits, (size_t)n * N, st) ? splits : 0;

@@ -11,6 +11,18 @@ template <typename T> __device__ __forceinline__ T from_f32(float v);
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
+template <typename T> __device__ __forceinline__ void store4(T* p, float a, float b, float c, float d);
+template <> __device__ __forceinline__ void store4<float>(float* p, float a, float b, float c, float d) {
+    *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
+}
+template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16* p, float a, float b, float c, float d) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+    uint2 v;
+    v.x = *reinterpret_cast<uint32_t*>(&lo);
+    v.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(p) = v;
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -74,24 +86,28 @@ __global__ void __launch_bounds__(256) reduce_residual_norm_kernel(const float* 
     pdl_trigger();
     pdl_wait();
     __shared__ float red[8];
-    constexpr int MAXV = 24;
+    constexpr int MAXV = 6;                                    // float4 chunks per thread: d <= 6 * 4 * 256
     const int row = blockIdx.x;
+    const int d4 = d / 4;
     if (seq_id != nullptr && seq_id[row] < 0) {
-        if (gain) for (int i = threadIdx.x; i < d; i += 256) out[(size_t)row * d + i] = from_f32<T>(0.f);
+        if (gain) for (int i = threadIdx.x; i < d4; i += 256) store4<T>(out + (size_t)row * d + 4 * i, 0.f, 0.f, 0.f, 0.f);
         return;
     }
-    float v[MAXV];
+    float4 v[MAXV];
     float ss = 0.f;
 #pragma unroll
     for (int k = 0; k < MAXV; ++k) {
         const int i = threadIdx.x + 256 * k;
-        if (i < d) {
-            const size_t at = (size_t)row * d + i;
-            float a = x[at];
-            for (int s = 0; s < splits; ++s) a += ws[(size_t)s * split_stride + at];
-            x[at] = a;
+        if (i < d4) {
+            const size_t at = (size_t)row * d4 + i;
+            float4 a = reinterpret_cast<const float4*>(x)[at];
+            for (int s = 0; s < splits; ++s) {                 // fixed order: part 0, 1, ...
+                const float4 b = __ldcg(reinterpret_cast<const float4*>(ws + (size_t)s * split_stride) + at);
+                a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+            }
+            reinterpret_cast<float4*>(x)[at] = a;
             v[k] = a;
-            ss = fmaf(a, a, ss);
+            ss = fmaf(a.x, a.x, fmaf(a.y, a.y, fmaf(a.z, a.z, fmaf(a.w, a.w, ss))));
         }
     }
     if (!gain) return;
@@ -100,7 +116,10 @@ __global__ void __launch_bounds__(256) reduce_residual_norm_kernel(const float* 
 #pragma unroll
     for (int k = 0; k < MAXV; ++k) {
         const int i = threadIdx.x + 256 * k;
-        if (i < d) out[(size_t)row * d + i] = from_f32<T>(v[k] * inv * gain[i]);
+        if (i < d4) {
+            const float4 g = reinterpret_cast<const float4*>(gain)[i];
+            store4<T>(out + (size_t)row * d + 4 * i, v[k].x * inv * g.x, v[k].y * inv * g.y, v[k].z * inv * g.z, v[k].w * inv * g.w);
+        }
     }
 }
 
@@ -117,9 +136,10 @@ void launch_reduce_residual_norm(const cdb* h, const float* ws, int splits, size
 // ------------------------------------------------------------------------------- RoPE + KV write
 // Rotates q and k of every row at its position (rotate-half pairing), rounds q, k, v to T, stores
 // q to qrot and k, v into the page of (seq, layer, slot) that holds the position.
+// qkv arrives as `parts` split-K partial products [part][row][3d] that are summed here in part order.
 template <typename T>
-__global__ void __launch_bounds__(256) rope_kv_write_kernel(const float* __restrict__ qkv, T* __restrict__ qrot,
-                                                            KvPool pool, RowsDev rows, int layer,
+__global__ void __launch_bounds__(256) rope_kv_write_kernel(const float* __restrict__ qkv, int parts, size_t part_stride,
+                                                            T* __restrict__ qrot, KvPool pool, RowsDev rows, int layer,
                                                             const float* __restrict__ rope_cos,
                                                             const float* __restrict__ rope_sin, int d,
                                                             int max_position, int max_seqs, int32_t* status) {
@@ -134,35 +154,48 @@ __global__ void __launch_bounds__(256) rope_kv_write_kernel(const float* __restr
     if (pos < 0 || pos >= max_position) { if (threadIdx.x == 0) atomicCAS(status, 0, kStatusPosition); return; }
     const int page = rows.page_table[((size_t)seq * rows.n_slots + slot) * rows.page_table_stride + pos / kPageSize];
     if (page < 0 || page >= pool.n_phys_pages) { if (threadIdx.x == 0) atomicCAS(status, 0, kStatusPage); return; }
-    const int Dh = pool.Dh, half = Dh / 2;
+    // four consecutive pair indices per thread: float4 loads of each split-K part, 8- or 16-byte stores
+    const int Dh = pool.Dh, half = Dh / 2, q4 = half / 4;
     const float* r = qkv + (size_t)row * 3 * d;
+    auto val4 = [&](int i) {
+        float4 a = __ldcg(reinterpret_cast<const float4*>(r + i));
+        for (int s = 1; s < parts; ++s) {
+            const float4 b = __ldcg(reinterpret_cast<const float4*>(r + (size_t)s * part_stride + i));
+            a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+        }
+        return a;
+    };
     T* base = (T*)pool.base;
-    for (int idx = threadIdx.x; idx < pool.H * half; idx += 256) {
-        const int hd = idx / half, i = idx % half;
-        const float c = rope_cos[(size_t)pos * half + i], s = rope_sin[(size_t)pos * half + i];
+    for (int idx = threadIdx.x; idx < pool.H * q4; idx += 256) {
+        const int hd = idx / q4, i = (idx % q4) * 4;
+        const float4 c = *reinterpret_cast<const float4*>(rope_cos + (size_t)pos * half + i);
+        const float4 s = *reinterpret_cast<const float4*>(rope_sin + (size_t)pos * half + i);
         const int e = hd * Dh + i;
-        const float q1 = r[e], q2 = r[e + half];
-        const float k1 = r[d + e], k2 = r[d + e + half];
-        qrot[(size_t)row * d + e] = from_f32<T>(q1 * c - q2 * s);
-        qrot[(size_t)row * d + e + half] = from_f32<T>(q2 * c + q1 * s);
+        const float4 q1 = val4(e), q2 = val4(e + half), k1 = val4(d + e), k2 = val4(d + e + half);
+        const float4 v1 = val4(2 * d + e), v2 = val4(2 * d + e + half);
+        store4<T>(qrot + (size_t)row * d + e, q1.x * c.x - q2.x * s.x, q1.y * c.y - q2.y * s.y, q1.z * c.z - q2.z * s.z, q1.w * c.w - q2.w * s.w);
+        store4<T>(qrot + (size_t)row * d + e + half, q2.x * c.x + q1.x * s.x, q2.y * c.y + q1.y * s.y, q2.z * c.z + q1.z * s.z, q2.w * c.w + q1.w * s.w);
         T* kt = base + pool.tile_offset(layer, page, 0, hd) + (size_t)(pos % kPageSize) * Dh;
         T* vt = base + pool.tile_offset(layer, page, 1, hd) + (size_t)(pos % kPageSize) * Dh;
-        kt[i] = from_f32<T>(k1 * c - k2 * s);
-        kt[i + half] = from_f32<T>(k2 * c + k1 * s);
-        vt[i] = from_f32<T>(r[2 * d + e]);
-        vt[i + half] = from_f32<T>(r[2 * d + e + half]);
+        store4<T>(kt + i, k1.x * c.x - k2.x * s.x, k1.y * c.y - k2.y * s.y, k1.z * c.z - k2.z * s.z, k1.w * c.w - k2.w * s.w);
+        store4<T>(kt + i + half, k2.x * c.x + k1.x * s.x, k2.y * c.y + k1.y * s.y, k2.z * c.z + k1.z * s.z, k2.w * c.w + k1.w * s.w);
+        store4<T>(vt + i, v1.x, v1.y, v1.z, v1.w);
+        store4<T>(vt + i + half, v2.x, v2.y, v2.z, v2.w);
     }
 }
 
-void launch_rope_kv_write(const cdb* h, int ln, int layer, const RowsDev& rows, cudaStream_t st) {
+void launch_rope_kv_write(const cdb* h, int ln, int layer, const float* qkv_parts, int parts, size_t part_stride,
+                          const RowsDev& rows, cudaStream_t st) {
     CDB_LAUNCH(h);
     if (rows.n_rows <= 0) return;
     if (h->cfg.dtype == CDB_FP32)
-        launch_pdl(rope_kv_write_kernel<float>, dim3(rows.n_rows), dim3(256), 0, st, h->lane[ln].qkv, (float*)h->lane[ln].qrot, h->pool, rows, layer,
-            h->rope_cos, h->rope_sin, h->cfg.d, h->cfg.max_position, h->cfg.max_seqs, h->status);
+        launch_pdl(rope_kv_write_kernel<float>, dim3(rows.n_rows), dim3(256), 0, st, qkv_parts, parts, part_stride,
+                   (float*)h->lane[ln].qrot, h->pool, rows, layer, h->rope_cos, h->rope_sin, h->cfg.d, h->cfg.max_position,
+                   h->cfg.max_seqs, h->status);
     else
-        launch_pdl(rope_kv_write_kernel<__nv_bfloat16>, dim3(rows.n_rows), dim3(256), 0, st, h->lane[ln].qkv, (__nv_bfloat16*)h->lane[ln].qrot, h->pool, rows,
-            layer, h->rope_cos, h->rope_sin, h->cfg.d, h->cfg.max_position, h->cfg.max_seqs, h->status);
+        launch_pdl(rope_kv_write_kernel<__nv_bfloat16>, dim3(rows.n_rows), dim3(256), 0, st, qkv_parts, parts, part_stride,
+                   (__nv_bfloat16*)h->lane[ln].qrot, h->pool, rows, layer, h->rope_cos, h->rope_sin, h->cfg.d,
+                   h->cfg.max_position, h->cfg.max_seqs, h->status);
 }
 
 // ------------------------------------------------------------------------------- SwiGLU
