@@ -28,6 +28,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
              "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
         flags += ["-Xptxas", "-v"]
+    flags += os.environ.get("CDB_NVCC_FLAGS", "").split()
     for src in SOURCES:
         s = os.path.join(CSRC, src)
         o = os.path.join(CSRC, src[:-3] + ".o")

@@ -60,6 +60,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait: false when the limit ran out or another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;            // the common case costs one probe
     const long long t0 = clock64();
     for (uint32_t it = 0;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -128,13 +129,11 @@ struct GemmParams {
     size_t split_stride;
     int32_t* status;
     unsigned long long* dbg;    // tuning aid: per-CTA phase time stamps (NULL = off)
-    int dbg_mode;               // tuning aid: 1 skip MMAs, 2 skip activation loads, 4 skip weight loads (results wrong)
 };
 
 __device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t) :: "memory"); return t; }
 
-// at most 72 registers per thread, so that a CTA fits on an SM beside four attention CTAs
-__global__ void __maxnreg__(72)
+__global__ void __launch_bounds__(kThreads, 1)
 gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w2,
                          const __grid_constant__ CUtensorMap map_x, GemmParams p) {
     pdl_trigger();
@@ -183,10 +182,10 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
     auto kb_end = [&](int t) { return (int)((long long)(t / (n_ftiles * n_rtiles) + 1) * n_kb / p.k_splits); };
 
     if (warp == 0) {
-        if (lane == 0) {
+        {
+            const bool leader = elect_one();
             int s = 0; uint32_t ph = 0;
             bool ok = true;
-            long long prod_wait = 0, prod_issue = 0;
             for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
                 const int f0 = (t % n_ftiles) * BM, r0 = (t / n_ftiles % n_rtiles) * BN;
                 // Every CTA walks its k-blocks from a different starting point (a function of its feature
@@ -194,23 +193,19 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
                 const int kb0 = kb_begin(t), nk = kb_end(t) - kb0, rot = ((t % n_ftiles) * 7) % nk;
                 for (int j = 0; j < nk; ++j) {
                     const int kb = kb0 + (j + rot) % nk;
-                    const long long c0 = clock64();
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abortp)) { ok = false; break; }
-                    const long long c1 = clock64();
-                    prod_wait += c1 - c0;
-                    mbar_expect_tx(full_bar(s), ((p.dbg_mode & 4) ? 0 : x_off) + ((p.dbg_mode & 2) ? 0 : x_bytes) + (p.dbg_mode == 6 ? 0 : 0));
                     const uint32_t dst = ring + (uint32_t)s * stage_bytes;
                     const int wc = p.w_tiled ? 0 : kb * BK, wr = p.w_tiled ? ((f0 / BM) * n_kb + kb) * BM : f0;
-                    if (!(p.dbg_mode & 4)) {
+                    if (leader) {
+                        mbar_expect_tx(full_bar(s), stage_bytes);
                         tma_load_2d(dst, &map_w, full_bar(s), wc, wr);
                         if (dual) tma_load_2d(dst + w_bytes, &map_w2, full_bar(s), wc, wr);
+                        tma_load_2d(dst + x_off, &map_x, full_bar(s), kb * BK, r0);
                     }
-                    if (!(p.dbg_mode & 2)) tma_load_2d(dst + x_off, &map_x, full_bar(s), kb * BK, r0);
-                    prod_issue += clock64() - c1;
+                    __syncwarp();
                     if (++s == S) { s = 0; ph ^= 1u; }
                 }
             }
-            if (p.dbg) { p.dbg[blockIdx.x * 8 + 5] = prod_wait; p.dbg[blockIdx.x * 8 + 7] = prod_issue; }
             if (!ok || *abortp) {                        // give copies already in flight time to land
                 for (int i = 0; i < 64; ++i) __nanosleep(1000);
             }
@@ -224,7 +219,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
             int s = 0; uint32_t ph = 0;
             int it = 0;
             bool ok = true;
-            long long mma_wait = 0, mma_t0 = clock64();
+            const long long mma_t0 = clock64();
             for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
                 const int acc = it & 1;
                 const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
@@ -233,9 +228,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
                 const uint32_t d_tmem = tmem_base + (uint32_t)acc * acc_cols;
                 const int kb0 = kb_begin(t), kb1 = kb_end(t);
                 for (int kb = kb0; kb < kb1; ++kb) {        // arrival order of the stages; which k-block is in one does not matter here
-                    const long long m0 = clock64();
                     if (!mbar_wait(full_bar(s), ph, abortp)) { ok = false; break; }
-                    mma_wait += clock64() - m0;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a_addr = ring + (uint32_t)s * stage_bytes;
                     const uint64_t a_desc = smem_desc_sw128(a_addr), a2_desc = smem_desc_sw128(a_addr + w_bytes);
@@ -244,8 +237,8 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
                     for (int k = 0; k < BK / UMMA_K; ++k) { // advance 32 bytes inside the swizzle span per UMMA_K
                         const uint64_t adv = (uint64_t)(k * UMMA_K * 2 >> 4);
                         const uint32_t accum = (kb > kb0 || k > 0) ? 1u : 0u;
-                        if (leader && !(p.dbg_mode & 1)) umma_bf16(d_tmem, a_desc + adv, b_desc + adv, idesc, accum);
-                        if (leader && dual && !(p.dbg_mode & 1)) umma_bf16(d_tmem + (uint32_t)BN, a2_desc + adv, b_desc + adv, idesc, accum);
+                        if (leader) umma_bf16(d_tmem, a_desc + adv, b_desc + adv, idesc, accum);
+                        if (leader && dual) umma_bf16(d_tmem + (uint32_t)BN, a2_desc + adv, b_desc + adv, idesc, accum);
                     }
                     __syncwarp();
                     if (leader) umma_commit(empty_bar(s));  // stage is free once these MMAs have read it
@@ -253,7 +246,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
                 }
                 if (ok && leader) umma_commit(acc_full_bar(acc));     // accumulator complete
             }
-            if (p.dbg && leader) { p.dbg[blockIdx.x * 8 + 3] = mma_wait; p.dbg[blockIdx.x * 8 + 2] = clock64() - mma_t0; }
+            if (p.dbg && leader) p.dbg[blockIdx.x * 8 + 2] = clock64() - mma_t0;
         }
         __syncwarp();
     } else {
@@ -269,44 +262,55 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
             if (p.dbg && it == 0 && warp == 2 && lane == 0) p.dbg[blockIdx.x * 8 + 4] = gtime();
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * acc_cols;
-            // 16 columns (= 16 batch rows) of this thread's feature per pass keeps the epilogue's register
-            // footprint small enough for the CTA to share an SM with the attention kernel
-            for (int c0 = 0; c0 < BN; c0 += 16) {
-                if (r0 + c0 >= p.n) break;                  // warp-uniform: nothing but padding rows left
-                uint32_t v[16];
-                tmem_ld16(t_addr + (uint32_t)c0, v);
-                if (dual) {
-                    uint32_t u[16];
+            // 16 columns (= 16 batch rows) of this thread's feature per pass: a small register footprint
+            const int n_cols = min(BN, p.n - r0);               // columns holding real rows (warp-uniform)
+            if (dual) {
+                for (int c0 = 0; c0 < n_cols; c0 += 16) {
+                    uint32_t v[16], u[16];
+                    tmem_ld16(t_addr + (uint32_t)c0, v);
                     tmem_ld16(t_addr + (uint32_t)(BN + c0), u);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                     if (f < p.N) {
                         __nv_bfloat16* dst = p.act + (size_t)(r0 + c0) * p.N + f;
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
-                            if (r0 + c0 + j < p.n) {
+                            if (c0 + j < n_cols) {
                                 const float g = __uint_as_float(v[j]);
-                                dst[(size_t)j * p.N] = __float2bfloat16_rn(g / (1.f + expf(-g)) * __uint_as_float(u[j]));
+                                dst[(size_t)j * p.N] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * __uint_as_float(u[j]));
                             }
                         }
                     }
-                    continue;
                 }
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (f < p.N) {
-                    float* dst = p.y + (size_t)split * p.split_stride + (size_t)(r0 + c0) * p.N + f;
-                    if (p.mode == kModeAccumulate) {
-                        float prev[16];                      // all residual loads in flight before the first add
+            } else {
+                // software pipeline: the TMEM load of the next 16 columns is in flight while these are stored
+                uint32_t v[2][16];
+                tmem_ld16(t_addr, v[0]);
+#pragma unroll 1
+                for (int c0 = 0; c0 < n_cols; c0 += 32) {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) prev[j] = (r0 + c0 + j < p.n) ? __ldcg(dst + (size_t)j * p.N) : 0.f;
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const int c = c0 + 16 * hh;
+                        if (c >= n_cols) break;
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                        if (c + 16 < n_cols) tmem_ld16(t_addr + (uint32_t)(c + 16), v[hh ^ 1]);
+                        if (f < p.N) {
+                            float* dst = p.y + (size_t)split * p.split_stride + (size_t)(r0 + c) * p.N + f;
+                            if (p.mode == kModeAccumulate) {
+                                float prev[16];                  // all residual loads in flight before the first add
 #pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (r0 + c0 + j < p.n) dst[(size_t)j * p.N] = prev[j] + __uint_as_float(v[j]);
-                    } else {
+                                for (int j = 0; j < 16; ++j) prev[j] = (c + j < n_cols) ? __ldcg(dst + (size_t)j * p.N) : 0.f;
 #pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (r0 + c0 + j < p.n) dst[(size_t)j * p.N] = __uint_as_float(v[j]);
+                                for (int j = 0; j < 16; ++j)
+                                    if (c + j < n_cols) dst[(size_t)j * p.N] = prev[j] + __uint_as_float(v[hh][j]);
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 16; ++j)
+                                    if (c + j < n_cols) __stcg(dst + (size_t)j * p.N, __uint_as_float(v[hh][j]));
+                            }
+                        }
                     }
                 }
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
@@ -423,7 +427,6 @@ static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* 
     if (p.stages < 2) p.stages = 2;
     if (p.stages > 8) p.stages = 8;
     p.status = h->status;
-    p.dbg_mode = getenv("CDB_GEMM_DBGMODE") ? atoi(getenv("CDB_GEMM_DBGMODE")) : 0;
     p.dbg = getenv("CDB_GEMM_DBG") ? (unsigned long long*)strtoull(getenv("CDB_GEMM_DBG"), nullptr, 0) : nullptr;
     CUtensorMap map_w, map_w2, map_x;
     const int n_kb = (K + BK - 1) / BK;
