@@ -43,12 +43,12 @@ def oracle_runs():
     return out
 
 
-def run_engine(mode="refill", lookahead=True, max_batch=8, max_live=8, gate=True, **kw):
+def run_engine(mode="refill", lookahead=True, max_batch=8, max_live=8, gate=True, n_slots=1, **kw):
     from paper_2608_09444_b200 import binding as B
     from paper_2608_09444_b200.engine import Engine
     dims, w, prompts = c1_inputs()
     wd = {k: v.cuda() for k, v in w.items()}
-    eng = Engine(dims, wd, max_batch=max_batch, max_live=max_live, max_len=48, n_pages=3 * max_live,
+    eng = Engine(dims, wd, max_batch=max_batch, max_live=max_live, max_len=48, n_pages=3 * max_live * n_slots,
                  gate_kind=B.GATE_SIGMOID_CDF if gate else B.GATE_NONE, q_or_eps=0.5, lookahead=lookahead,
                  mode=mode, max_prefill_rows=256, record_states=True, record_logits=True, **kw)
     res = eng.generate(list(prompts), 16)
@@ -117,3 +117,18 @@ def test_c1_exits_disabled_equals_fixed_depth(oracle_runs):
     eng, res = run_engine("refill", gate=False)
     compare(eng, res, ref)
     assert all(np.all(d == 4) for d in res["depths"])
+
+
+@pytest.mark.parametrize("layout", ["depth_indexed", "first_then_shared"])
+def test_c1_depth_aware_kv_layouts(layout):
+    """Last-exited cache (depth-indexed slots + copy-on-exit of the last state into the skipped slots,
+    section 4.2) and the first-then-shared layout (appendix C.1), end to end against the oracle."""
+    from paper_2608_09444_b200 import binding as B
+    dims, w, prompts = c1_inputs()
+    wn = synth.weights_to_numpy(w)
+    o_layout = {"depth_indexed": O.DEPTH_INDEXED, "first_then_shared": O.FIRST_THEN_SHARED}[layout]
+    b_layout = {"depth_indexed": B.KV_DEPTH_INDEXED, "first_then_shared": B.KV_FIRST_THEN_SHARED}[layout]
+    orc = O.Oracle(dims, wn, kv_layout=o_layout, gate_kind=O.GATE_SIGMOID_CDF, q_or_eps=0.5, lookahead=True)
+    ref = [orc.generate(p, 16, keep_states=True) for p in prompts]
+    eng, res = run_engine("refill", n_slots=O.n_slots(o_layout, dims.R), kv_layout=b_layout)
+    compare(eng, res, ref)
