@@ -14,8 +14,9 @@
  *  - "device" pointers are CUDA device memory owned by the CALLER; they must stay valid until
  *    the stream work that uses them has finished.  "host" values are plain C values.
  *  - The library owns only what cdb_create() allocates (scratch buffers, per-sequence gate
- *    state, RoPE table) and frees it in cdb_destroy().  The weights are BORROWED: the pointers
- *    in cdb_weights_t must outlive the handle.
+ *    state, RoPE table, tile-major copies of bf16 projection weights) and frees it in
+ *    cdb_destroy().  The weights are BORROWED: the pointers in cdb_weights_t must outlive the
+ *    handle and their contents must not change after cdb_create().
  *  - All work is enqueued on the given stream (a cudaStream_t passed as void*) and no call
  *    synchronises, except cdb_create, cdb_destroy and cdb_poll_status.
  *  - Argument checks that can be made on the host happen before anything is launched.
