@@ -130,13 +130,6 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     static const bool no_pdl = getenv("CDB_NO_PDL") != nullptr;      // tuning aid: plain stream-ordered launches
-    static const int carve = getenv("CDB_ALL_CARVEOUT") ? atoi(getenv("CDB_ALL_CARVEOUT")) : -2;      // tuning aid
-    if (carve > -2) {
-        static const void* seen[64]; static int n_seen = 0;
-        bool have = false;
-        for (int i = 0; i < n_seen; ++i) have |= seen[i] == (const void*)kernel;
-        if (!have && n_seen < 64) { seen[n_seen++] = (const void*)kernel; cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve); }
-    }
     cfg.attrs = attr; cfg.numAttrs = no_pdl ? 0 : 1;
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }

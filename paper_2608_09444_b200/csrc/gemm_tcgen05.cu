@@ -31,7 +31,7 @@ constexpr int UMMA_K = 16;
 constexpr int kThreads = 192;
 constexpr long long kWaitCycles = 1500000000LL;     // about a second of SM clocks
 constexpr int kStatusTimeout = 4;
-constexpr int kMaxSmem = 225 * 1024;
+constexpr int kMaxSmem = 196 * 1024;    // every launch then asks for the same shared-memory carve-out (no SM reconfiguration between projections)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -127,6 +127,7 @@ struct GemmParams {
     int k_splits;               // the K range is cut into this many parts, each a tile of its own
     int w_tiled;                // weights come from the tile-major copy: tile (ft, kb) starts at row (ft * n_kb + kb) * 128
     size_t split_stride;
+    uint32_t stage_out_off;     // SwiGLU mode: byte offset (from the ring base) of a [BN][128] bf16 output staging tile
     int32_t* status;
     unsigned long long* dbg;    // tuning aid: per-CTA phase time stamps (NULL = off)
 };
@@ -265,22 +266,55 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
             // 16 columns (= 16 batch rows) of this thread's feature per pass: a small register footprint
             const int n_cols = min(BN, p.n - r0);               // columns holding real rows (warp-uniform)
             if (dual) {
-                for (int c0 = 0; c0 < n_cols; c0 += 16) {
-                    uint32_t v[16], u[16];
-                    tmem_ld16(t_addr + (uint32_t)c0, v);
-                    tmem_ld16(t_addr + (uint32_t)(BN + c0), u);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    if (f < p.N) {
-                        __nv_bfloat16* dst = p.act + (size_t)(r0 + c0) * p.N + f;
+                // gate and up accumulators side by side; loads of the next 16 columns fly while these are finished
+                uint32_t v[2][16], u[2][16];
+                tmem_ld16(t_addr, v[0]);
+                tmem_ld16(t_addr + (uint32_t)BN, u[0]);
+#pragma unroll 1
+                for (int c0 = 0; c0 < n_cols; c0 += 32) {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            if (c0 + j < n_cols) {
-                                const float g = __uint_as_float(v[j]);
-                                dst[(size_t)j * p.N] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * __uint_as_float(u[j]));
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const int c = c0 + 16 * hh;
+                        if (c >= n_cols) break;
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                        if (c + 16 < n_cols) {
+                            tmem_ld16(t_addr + (uint32_t)(c + 16), v[hh ^ 1]);
+                            tmem_ld16(t_addr + (uint32_t)(BN + c + 16), u[hh ^ 1]);
+                        }
+                        // SwiGLU, rounded to bf16, into the staging tile [row][feature of this tile] (2-byte global
+                        // stores straight from here cost 7 us per tile; staged rows leave as 16-byte stores)
+                        {
+                            const uint32_t srow = ring + p.stage_out_off + (uint32_t)c * (BM * 2) + (uint32_t)(q * 32 + lane) * 2;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const float g = __uint_as_float(v[hh][j]);
+                                const __nv_bfloat16 r = __float2bfloat16_rn(__fdividef(g, 1.f + __expf(-g)) * __uint_as_float(u[hh][j]));
+                                asm volatile("st.shared.b16 [%0], %1;" ::"r"(srow + (uint32_t)j * (BM * 2)), "h"(*reinterpret_cast<const uint16_t*>(&r)) : "memory");
                             }
                         }
                     }
                 }
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                asm volatile("bar.sync 1, 128;" ::: "memory");              // the four epilogue warps: tile staged
+                {
+                    const int et = threadIdx.x - 64;                         // 0..127 among the epilogue warps
+                    const int f0t = (t % n_ftiles) * BM;
+                    for (int idx = et; idx < n_cols * 16; idx += 128) {      // 16 chunks of 8 features per row
+                        const int row = idx >> 4, ch = idx & 15;
+                        const int fc = f0t + ch * 8;
+                        uint4 val;
+                        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
+                                     : "r"(ring + p.stage_out_off + (uint32_t)row * (BM * 2) + (uint32_t)ch * 16));
+                        __nv_bfloat16* dst = p.act + (size_t)(r0 + row) * p.N + fc;
+                        if (fc + 8 <= p.N) {
+                            *reinterpret_cast<uint4*>(dst) = val;
+                        } else {
+                            const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&val);
+                            for (int k = 0; k < 8; ++k) if (fc + k < p.N) dst[k] = e[k];
+                        }
+                    }
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");              // staging tile free for the next tile
             } else {
                 // software pipeline: the TMEM load of the next 16 columns is in flight while these are stored
                 uint32_t v[2][16];
@@ -423,11 +457,14 @@ static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* 
     static const int smem_cap = getenv("CDB_GEMM_SMEM_KB") ? atoi(getenv("CDB_GEMM_SMEM_KB")) * 1024 : kMaxSmem;   // tuning aid
     int budget = smem_cap < kMaxSmem ? smem_cap : kMaxSmem;
     if (h->gemm_smem_cap > 0 && h->gemm_smem_cap < budget) budget = h->gemm_smem_cap;
-    p.stages = (budget - 1024) / stage_bytes;
+    const int stage_out = mode == kModeSwiGLU ? p.BN * BM * 2 : 0;   // output staging tile of the SwiGLU epilogue
+    p.stages = (budget - 1024 - stage_out) / stage_bytes;
     if (p.stages < 2) p.stages = 2;
     if (p.stages > 8) p.stages = 8;
+    p.stage_out_off = (uint32_t)(p.stages * stage_bytes);
     p.status = h->status;
     p.dbg = getenv("CDB_GEMM_DBG") ? (unsigned long long*)strtoull(getenv("CDB_GEMM_DBG"), nullptr, 0) : nullptr;
+    if (getenv("CDB_GEMM_DBG_ONLY") && atoi(getenv("CDB_GEMM_DBG_ONLY")) != mode * 100000 + N) p.dbg = nullptr;   // tuning aid: one launch kind
     CUtensorMap map_w, map_w2, map_x;
     const int n_kb = (K + BK - 1) / BK;
     const void* Wt = find_tiled(h, W, N, K);
@@ -441,7 +478,7 @@ static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* 
     if (!make_map(&map_x, x, n, K, p.BN)) return false;
     const int n_tiles = n_ft * ((n + p.BN - 1) / p.BN) * k_splits;
     const int grid = n_tiles < sms ? n_tiles : sms;
-    const size_t smem = (size_t)p.stages * stage_bytes + 1024;
+    const size_t smem = (size_t)p.stages * stage_bytes + stage_out + 1024;
     launch_pdl(gemm_bf16_tcgen05_kernel, dim3(grid), dim3(kThreads), smem, st, map_w, map_w2, map_x, p);
     return true;
 }
