@@ -437,3 +437,185 @@ extern "C" int cdb_paged_attention_static(const void* q, void* o, const void* po
     }
     return cudaGetLastError() == cudaSuccess ? CDB_OK : CDB_ERR_CUDA;
 }
+
+// =====================================================================================================
+// Query-tiled causal attention for prompt processing.  The rows of a prompt are consecutive positions of
+// one sequence, so a tile of 32 query rows shares every K/V page it reads: a CTA of 128 threads (4 per
+// query, each owning a quarter of the head dimension) stages a page's K and V tile in shared memory once
+// and all 32 queries consume it.  Against one-query-per-warp decode attention this cuts the KV traffic of
+// a prompt of P tokens from ~P^2/2 to ~P^2/64 tokens.  Same rounding points as the decode kernel: K, V
+// and q in the pool's dtype, scores / softmax / P.V in fp32 FMAs.
+// =====================================================================================================
+namespace cdbk {
+namespace {
+
+constexpr int kPfTile = 32;                 // query rows per tile
+
+// Cuts the batch into tiles: maximal runs of rows with the same sequence and consecutive positions, in
+// pieces of at most kPfTile rows.  tiles[i] = first row, tile_rows[i] = rows in it.  One thread: n_rows is small.
+__global__ void prefill_plan_kernel(RowsDev rows, int32_t* __restrict__ tiles, int32_t* __restrict__ tile_rows,
+                                    int32_t* __restrict__ n_tiles) {
+    pdl_trigger();
+    pdl_wait();
+    if (blockIdx.x != 0 || threadIdx.x != 0) return;
+    int nt = 0, r = 0;
+    while (r < rows.n_rows) {
+        if (rows.seq_id[r] < 0) { ++r; continue; }
+        int len = 1;
+        while (r + len < rows.n_rows && len < kPfTile && rows.seq_id[r + len] == rows.seq_id[r] &&
+               rows.position[r + len] == rows.position[r] + len)
+            ++len;
+        tiles[nt] = r; tile_rows[nt] = len; ++nt;
+        r += len;
+    }
+    *n_tiles = nt;
+}
+
+template <typename T, int DH>
+__global__ void __launch_bounds__(128) attn_prefill_kernel(AttnParams p, const int32_t* __restrict__ tiles,
+                                                           const int32_t* __restrict__ tile_rows,
+                                                           const int32_t* __restrict__ n_tiles, T* __restrict__ out) {
+    pdl_trigger();
+    pdl_wait();
+    constexpr int EPC = Chunk<T>::EPC;
+    constexpr int DQ = DH / 4;               // dims per thread
+    constexpr int CH = DQ / EPC;             // 16-byte chunks per thread per token
+    static_assert(DQ % EPC == 0, "a thread's dims must be whole 16-byte chunks");
+    __shared__ __align__(16) unsigned char k_s[kPageSize * DH * sizeof(T)];
+    __shared__ __align__(16) unsigned char v_s[kPageSize * DH * sizeof(T)];
+    const int H = p.pool.H;
+    const int tile = blockIdx.x, head = blockIdx.y;
+    if (tile >= *n_tiles) return;
+    const int row0 = tiles[tile], nq = tile_rows[tile];
+    const int qi = threadIdx.x >> 2, part = threadIdx.x & 3;           // query in tile, quarter of the head dim
+    const bool active = qi < nq;
+    const int row = row0 + (active ? qi : 0);
+    const int seq = p.rows.seq_id[row0];
+    const int slot = p.rows.slot_of(row0);
+    const int pos = p.rows.position[row];
+    const int pos_last = p.rows.position[row0 + nq - 1];
+    if (seq < 0 || seq >= p.max_seqs || slot < 0 || slot >= p.rows.n_slots || pos_last < 0) {
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, kStatusSeq);
+        return;
+    }
+    const int32_t* table = p.rows.page_table + ((size_t)seq * p.rows.n_slots + slot) * p.rows.page_table_stride;
+    const T* pool_base = (const T*)p.pool.base;
+
+    float qf[DQ], o[DQ];
+    {
+        const uint4* qp = (const uint4*)((const T*)p.q + (size_t)row * H * DH + (size_t)head * DH + part * DQ);
+#pragma unroll
+        for (int j = 0; j < CH; ++j) {
+            const uint4 v = qp[j];
+            Chunk<T>::unpack(v, qf + j * EPC);
+        }
+#pragma unroll
+        for (int e = 0; e < DQ; ++e) { qf[e] *= p.scale_log2; o[e] = 0.f; }
+    }
+    float m = -INFINITY, l = 0.f;
+    constexpr int TILE_CHUNKS = kPageSize * DH * (int)sizeof(T) / 16;
+    for (int pi = 0; pi <= pos_last / kPageSize; ++pi) {
+        const int page = table[pi];
+        const bool page_ok = page >= 0 && page < p.pool.n_phys_pages;
+        __syncthreads();                                               // previous page fully consumed
+        if (page_ok) {
+            const uint4* kt = (const uint4*)(pool_base + p.pool.tile_offset(p.layer, page, 0, head));
+            const uint4* vt = (const uint4*)(pool_base + p.pool.tile_offset(p.layer, page, 1, head));
+            for (int i = threadIdx.x; i < TILE_CHUNKS; i += 128) {
+                ((uint4*)k_s)[i] = kt[i];
+                ((uint4*)v_s)[i] = vt[i];
+            }
+        } else if (threadIdx.x == 0) {
+            atomicCAS(p.status, 0, kStatusPage);
+        }
+        __syncthreads();
+        if (!page_ok) continue;
+        // tokens of this page the query may see (none for idle threads and for pages past the query's position;
+        // such threads still run the score loop, whose shuffles need the whole warp)
+        const int t_hi = active ? min(kPageSize, pos - pi * kPageSize + 1) : 0;
+        float s[kPageSize];
+        float pmax = -INFINITY;
+#pragma unroll
+        for (int t = 0; t < kPageSize; ++t) {
+            float acc = 0.f;
+            const uint4* kr = (const uint4*)(k_s + ((size_t)t * DH + part * DQ) * sizeof(T));
+#pragma unroll
+            for (int j = 0; j < CH; ++j) {
+                float kf[EPC];
+                Chunk<T>::unpack(kr[j], kf);
+#pragma unroll
+                for (int e = 0; e < EPC; ++e) acc = fmaf(qf[j * EPC + e], kf[e], acc);
+            }
+            acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+            acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+            s[t] = t < t_hi ? acc : -INFINITY;
+            pmax = fmaxf(pmax, s[t]);
+        }
+        if (t_hi <= 0) continue;                                       // (the loop's barriers are at its top)
+        const float m_new = fmaxf(m, pmax);
+        const float corr = exp2f(m - m_new);
+        l *= corr;
+#pragma unroll
+        for (int e = 0; e < DQ; ++e) o[e] *= corr;
+#pragma unroll
+        for (int t = 0; t < kPageSize; ++t) {
+            if (t < t_hi) {
+                const float pr = exp2f(s[t] - m_new);
+                l += pr;
+                const uint4* vr = (const uint4*)(v_s + ((size_t)t * DH + part * DQ) * sizeof(T));
+#pragma unroll
+                for (int j = 0; j < CH; ++j) {
+                    float vf[EPC];
+                    Chunk<T>::unpack(vr[j], vf);
+#pragma unroll
+                    for (int e = 0; e < EPC; ++e) o[j * EPC + e] = fmaf(pr, vf[e], o[j * EPC + e]);
+                }
+            }
+        }
+        m = m_new;
+    }
+    if (active) {
+        const float inv = 1.f / l;
+        T* orow = out + (size_t)row * H * DH + (size_t)head * DH + part * DQ;
+#pragma unroll
+        for (int e = 0; e < DQ; ++e) orow[e] = T(o[e] * inv);
+    }
+}
+
+template <typename T, int DH>
+void launch_prefill_t(const cdb* h, const AttnParams& p, int ln, void* o, cudaStream_t st) {
+    const Lane& L = h->lane[ln];
+    // pads first: rows the tiles do not cover keep a zero output
+    cudaMemsetAsync(o, 0, (size_t)p.rows.n_rows * p.pool.H * DH * sizeof(T), st);
+    CDB_LAUNCH(h);
+    launch_pdl(prefill_plan_kernel, dim3(1), dim3(32), 0, st, p.rows, L.attn_item_start, L.pf_tile_rows, L.pf_n_tiles);
+    CDB_LAUNCH(h);
+    dim3 grid(p.rows.n_rows, p.pool.H);                                // upper bound on tiles; surplus CTAs exit at once
+    launch_pdl(attn_prefill_kernel<T, DH>, grid, dim3(128), 0, st, p, (const int32_t*)L.attn_item_start,
+               (const int32_t*)L.pf_tile_rows, (const int32_t*)L.pf_n_tiles, (T*)o);
+}
+
+}  // namespace
+
+// Causal attention of prompt rows (consecutive positions of each sequence adjacent in the batch) over the
+// pages their own call has just written.  Uses the lane's split-scan buffer for its tile list.
+void launch_attention_prefill(const cdb* h, int ln, int layer, const RowsDev& rows, const void* q, void* o, cudaStream_t st) {
+    if (rows.n_rows <= 0) return;
+    AttnParams p;
+    p.q = q; p.pool = h->pool; p.rows = rows; p.layer = layer; p.max_splits = h->max_splits;
+    p.max_seqs = h->cfg.max_seqs;
+    p.scale_log2 = 1.4426950408889634f / sqrtf((float)h->cfg.Dh);
+    p.part = nullptr; p.item_start = nullptr; p.counter = nullptr; p.status = h->status;
+    const int Dh = h->cfg.Dh;
+    if (h->cfg.dtype == CDB_BF16) {
+        if (Dh == 128) launch_prefill_t<__nv_bfloat16, 128>(h, p, ln, o, st);
+        else if (Dh == 96) launch_prefill_t<__nv_bfloat16, 96>(h, p, ln, o, st);
+        else launch_prefill_t<__nv_bfloat16, 64>(h, p, ln, o, st);
+    } else {
+        if (Dh == 128) launch_prefill_t<float, 128>(h, p, ln, o, st);
+        else if (Dh == 96) launch_prefill_t<float, 96>(h, p, ln, o, st);
+        else launch_prefill_t<float, 64>(h, p, ln, o, st);
+    }
+}
+
+}  // namespace cdbk

@@ -85,7 +85,8 @@ void layer_forward(cdb_t* h, int ln, int layer, const RowsDev& rows, float* x, c
     launch_rope_kv_write(h, ln, layer, L.qkv, 1, 0, rows, st);
     if (attn_after) cudaStreamWaitEvent(st, attn_after, 0);      // the other half-batch's attention goes first
     h->attn_split_done = attn_done;
-    launch_attention(h, ln, layer, rows, L.qrot, L.attn_o, st);
+    if (h->prefill_attention) launch_attention_prefill(h, ln, layer, rows, L.qrot, L.attn_o, st);
+    else launch_attention(h, ln, layer, rows, L.qrot, L.attn_o, st);
     h->attn_split_done = nullptr;
     launch_linear(h, L.attn_o, layer_ptr(h, h->w.W_o, layer, d * d), x, n, c.d, c.d, Epilogue::ResidualAdd, st);
     launch_rmsnorm(h, x, h->g_mlp + (size_t)layer * d, L.xn, rows, st);
@@ -116,7 +117,8 @@ void layer_forward_tc(cdb_t* h, int ln, int layer, const RowsDev& rows, float* x
     }
     if (attn_after) cudaStreamWaitEvent(st, attn_after, 0);      // the other half-batch's attention goes first
     h->attn_split_done = attn_done;
-    launch_attention(h, ln, layer, rows, L.qrot, L.attn_o, st);
+    if (h->prefill_attention) launch_attention_prefill(h, ln, layer, rows, L.qrot, L.attn_o, st);
+    else launch_attention(h, ln, layer, rows, L.qrot, L.attn_o, st);
     h->attn_split_done = nullptr;
     {
         ProfScope ps(h, kProfLinear, st);
@@ -173,7 +175,7 @@ void free_all(cdb_t* h) {
                     h->h_prev, h->h_work, h->logits, h->exit_flag, h->status, h->emit_tmp};
     for (void* p : ptrs) if (p) cudaFree(p);
     for (Lane& L : h->lane) {
-        void* lp[] = {L.xn, L.qrot, L.attn_o, L.act, L.qkv, L.gu, L.ws, L.attn_part, L.attn_item_start, L.attn_counters};
+        void* lp[] = {L.xn, L.qrot, L.attn_o, L.act, L.qkv, L.gu, L.ws, L.attn_part, L.attn_item_start, L.attn_counters, L.pf_tile_rows, L.pf_n_tiles};
         for (void* p : lp) if (p) cudaFree(p);
     }
     for (int i = 0; i < h->n_tiled; ++i) if (h->tiled[i].tiled) cudaFree(h->tiled[i].tiled);
@@ -259,6 +261,8 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
         CDB_ALLOC(L.attn_part, float, r * c.H * h->max_splits * (size_t)(c.Dh + 2));
         CDB_ALLOC(L.attn_item_start, int32_t, r + 1);
         CDB_ALLOC(L.attn_counters, int32_t, n_layers);
+        CDB_ALLOC(L.pf_tile_rows, int32_t, r);
+        CDB_ALLOC(L.pf_n_tiles, int32_t, 1);
     }
     CDB_ALLOC(h->h_prev, float, R_ * d);
     CDB_ALLOC(h->h_work, float, R_ * d);
@@ -480,6 +484,7 @@ int cdb_prefill(cdb_t* h, const int32_t* token_ids, const cdb_rows_t* rows, cons
     cudaStream_t st = (cudaStream_t)stream;
     const cdb_config_t& c = h->cfg;
     float* x = h->h_work;
+    h->prefill_attention = 1;
     launch_embed(h, token_ids, rd, x, true, st);
     launch_attention_plan(h, 0, rd, st);
     rd.slot_override = 0;
@@ -490,6 +495,7 @@ int cdb_prefill(cdb_t* h, const int32_t* token_ids, const cdb_rows_t* rows, cons
     }
     rd.slot_override = 0;
     for (int l = c.L_pre + c.L_core; l < c.L_pre + c.L_core + c.L_coda; ++l) layer_forward(h, 0, l, rd, x, st);
+    h->prefill_attention = 0;
     if (n_emit > 0) {
         // gather the emitting rows to the front of h_prev (free during prefill), then LM head on them
         launch_gather(h, x, emit_idx, nullptr, n_emit, h->h_prev, st);

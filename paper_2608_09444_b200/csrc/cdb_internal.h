@@ -57,6 +57,8 @@ struct Lane {
     float* attn_part;               // [rows_cap*H*max_splits][Dh + 2] split partials (o, m, l)
     int32_t* attn_item_start;       // [rows_cap + 1] exclusive scan of splits per row
     int32_t* attn_counters;         // [L] work-fetch counters
+    int32_t* pf_tile_rows;          // [rows_cap] rows per prefill tile (tile starts reuse attn_item_start)
+    int32_t* pf_n_tiles;            // [1]
 };
 
 }  // namespace cdbk
@@ -103,6 +105,7 @@ struct cdb {
     cudaEvent_t ev_fork, ev_join, ev_attn[2];
     mutable cudaEvent_t attn_split_done; // recorded right after the next attention split kernel when set
     mutable int attn_ctas_per_sm_cap;
+    mutable int prefill_attention;      // 1 while cdb_prefill runs: layers use the query-tiled causal attention
     mutable int gemm_smem_cap;          // > 0: projection kernels keep their shared-memory ring below this many bytes   // > 0: leave room on every SM for the other half-batch's kernels
 
     mutable uint64_t launches;
@@ -159,6 +162,7 @@ void launch_rmsnorm(const cdb* h, const float* x, const float* gain, void* out, 
 void launch_rope_kv_write(const cdb* h, int ln, int layer, const float* qkv_parts, int parts, size_t part_stride, const RowsDev& rows, cudaStream_t st);
 void launch_attention(const cdb* h, int ln, int layer, const RowsDev& rows, const void* q, void* o, cudaStream_t st);
 void launch_attention_plan(const cdb* h, int ln, const RowsDev& rows, cudaStream_t st);
+void launch_attention_prefill(const cdb* h, int ln, int layer, const RowsDev& rows, const void* q, void* o, cudaStream_t st);
 void launch_swiglu(const cdb* h, int ln, int n_rows, cudaStream_t st);
 void launch_embed(const cdb* h, const int32_t* tokens, const RowsDev& rows, float* out, bool reset_gate, cudaStream_t st);
 void launch_gate(const cdb* h, const RowsDev& rows, const float* x, const float* x_prev, float* gate_val_out,

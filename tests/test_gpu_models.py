@@ -122,3 +122,44 @@ def test_lockstep_replay_of_adaptive_decode_bf16():
           f"near-tie tokens {explained}/{tokens}")
     assert worst_state <= TOL and worst_logit <= TOL and worst_gate <= TOL
     assert explained <= max(2, tokens // 20) and near_gate <= max(2, decisions // 50)
+
+
+@pytest.mark.parametrize("H,Dh,dtype", [(2, 128, "bf16"), (3, 96, "bf16"), (2, 64, "bf16"), (4, 64, "fp32")])
+def test_prefill_matches_oracle(H, Dh, dtype):
+    """Lock-step prompt processing (query-tiled causal attention over the pages the call itself writes),
+    several prompts of ragged length in one call with a pad row, against the oracle's prefill."""
+    from paper_2608_09444_b200 import binding as B
+    dims = synth.Dims(V=300, d=H * Dh, H=H, Dh=Dh, F=192, L_pre=1, L_core=2, L_coda=1, R=3, dtype=dtype)
+    w = synth.make_weights(dims, 8, std=0.05, gain_jitter=0.1)
+    wn = synth.weights_to_numpy(w)
+    lens = [1, 33, 70, 16, 47]
+    prompts = [synth.make_prompts(1, n, dims.V, 20 + i)[0] for i, n in enumerate(lens)]
+    table_np, n_pages = synth.make_page_table(np.asarray(lens), 16, seed=2, extra_pages=1)
+    n = sum(lens) + 1
+    cdb = B.Cdb(dims, {k: v.cuda() for k, v in w.items()}, max_rows=n, max_seqs=len(lens), max_position=table_np.shape[1] * 16,
+                gate_kind=B.GATE_NONE)
+    tdt = torch.float32 if dtype == "fp32" else torch.bfloat16
+    pool = torch.full(synth.kv_pool_shape(dims, n_pages), float("nan"), dtype=tdt, device="cuda")   # nothing is read before written
+    cdb.kv_bind(pool)
+    seq = np.concatenate([np.full(m, i) for i, m in enumerate(lens)] + [[-1]])
+    pos = np.concatenate([np.arange(m) for m in lens] + [[0]])
+    tok = np.concatenate(prompts + [[0]])
+    ends = np.cumsum(lens) - 1
+    rows = B.Rows(i32(seq), i32(pos), i32(table_np))
+    token, logits = torch.zeros(len(lens), dtype=torch.int32, device="cuda"), torch.zeros((len(lens), dims.V), device="cuda")
+    cdb.prefill(i32(tok), rows, i32(ends), token, logits)
+    torch.cuda.synchronize()
+    assert cdb.poll_status() == 0
+    orc = O.Oracle(dims, wn, gate_kind=O.GATE_NONE)
+    tol = 1e-4 if dtype == "fp32" else TOL
+    for i, pr in enumerate(prompts):
+        cache = orc.new_cache(len(pr))
+        ref = orc.prefill(pr, cache)
+        assert rel_err(logits[i].cpu().numpy(), ref) <= tol, (i, rel_err(logits[i].cpu().numpy(), ref))
+        if int(token[i]) != int(np.argmax(ref)):
+            assert ref.max() - ref[int(token[i])] < 2 * np.max(np.abs(logits[i].cpu().numpy() - ref))
+        # the KV the prompt left behind (last core layer, shared slot): what decode will attend to
+        l = dims.L_pre + dims.L_core - 1
+        page, off = table_np[i, (len(pr) - 1) // 16], (len(pr) - 1) % 16
+        got = pool[l, page, 0, :, off, :].float().cpu().numpy()
+        assert rel_err(got, cache[l][0][0][len(pr) - 1]) <= tol
