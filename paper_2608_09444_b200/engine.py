@@ -10,6 +10,7 @@ that per-tick row lists and page tables are reproducible bit for bit.
 from __future__ import annotations
 
 import dataclasses
+import time
 
 import numpy as np
 import torch
@@ -34,7 +35,7 @@ class Engine:
                  kv_layout: int = B.KV_SHARED, gate_kind: int = B.GATE_SIGMOID_CDF, q_or_eps: float = 0.5,
                  r_min: int = 1, lookahead: bool = True, mode: str = "refill", min_coda_batch: int = 1,
                  max_prefill_rows: int | None = None, flags: int = 0, record_states: bool = False,
-                 record_logits: bool = False, device: str = "cuda:0"):
+                 record_logits: bool = False, record_ticks: bool = True, device: str = "cuda:0"):
         self.dims, self.mode, self.lookahead = dims, mode, lookahead
         self.max_batch, self.max_live, self.min_coda_batch = max_batch, max_live, min_coda_batch
         self.dev = torch.device(device)
@@ -68,7 +69,7 @@ class Engine:
         self.counts = torch.zeros(2, **i32)
         self.tok_out = torch.zeros(max_rows, **i32)
         self.logits = torch.zeros((max_rows, dims.V), **f32) if record_logits else None
-        self.record_states, self.record_logits = record_states, record_logits
+        self.record_states, self.record_logits, self.record_ticks = record_states, record_logits, record_ticks
         self.stats = {"recurrent_steps": 0, "row_steps": 0, "coda_calls": 0, "prefill_calls": 0, "tick_rows": []}
         self.trace_states = {}                                        # (sid, token index) -> exit state
         self.trace_logits = {}
@@ -118,6 +119,7 @@ class Engine:
         Ts = [T] * n if np.isscalar(T) else list(T)
         seqs = [_Seq(i, np.asarray(prompts[i], dtype=np.int32), Ts[i], [], [], [], []) for i in range(n)]
         waiting = list(range(n))
+        self.stats["start"] = time.perf_counter()
         live_slot = {}                       # sid -> live slot id (index into gate state / page table)
         free_slots = list(range(self.max_live - 1, -1, -1))
         ready = []                           # [(sid, h row index in h_ready)] awaiting the recurrent batch (FIFO)
@@ -155,10 +157,9 @@ class Engine:
                 cdb.boundary_prelude(tok_t, rows, out)
             else:
                 cdb.boundary_embed(tok_t, rows, out)
-            for k, s in enumerate(sids):
-                slot = ready_free.pop()
-                self.h_ready[slot].copy_(out[k])
-                ready.append((s, slot))
+            slots = [ready_free.pop() for _ in sids]
+            self.h_ready.index_copy_(0, torch.tensor(slots, dtype=torch.int64, device=self.dev), out)
+            ready.extend(zip(sids, slots))
 
         def finish_or_continue(s, token):
             sq = seqs[s]
@@ -249,12 +250,20 @@ class Engine:
 
         def run_recurrent(allow_refill):
             nonlocal rec
+            if "decode_start" not in self.stats and not waiting:          # every prompt processed: decode phase begins
+                torch.cuda.synchronize(self.dev)
+                self.stats["decode_start"] = time.perf_counter()
             # survivors are already at the front of h_rec in stable order; append refills (FIFO)
+            n_keep = len(rec)
+            take = []
             while allow_refill and ready and len(rec) < self.max_batch:
                 s, slot = ready.pop(0)
-                self.h_rec[len(rec)].copy_(self.h_ready[slot])
+                take.append(slot)
                 ready_free.append(slot)
                 rec.append([s, 1])
+            if take:
+                cdb.gather_rows(self.h_ready, torch.tensor(take, dtype=torch.int32, device=self.dev), None, len(take),
+                                self.h_rec[n_keep:n_keep + len(take)])
             k = len(rec)
             if k == 0:
                 return False
@@ -279,14 +288,16 @@ class Engine:
             gv = self.gate_val[:k].cpu().numpy()
             self.stats["recurrent_steps"] += 1
             self.stats["row_steps"] += k
-            self.stats["tick_rows"].append([(s, len(seqs[s].tokens), r) for s, r in rec])
+            if self.record_ticks:
+                self.stats["tick_rows"].append([(s, len(seqs[s].tokens), r) for s, r in rec])
             for i, (s, r) in enumerate(rec):
                 seqs[s].cur_gates.append(float(gv[i]))
-            for j, i in enumerate(ex):
-                s, r = rec[int(i)]
-                slot = coda_free.pop()
-                self.h_coda[slot].copy_(self.h_exit[j])
-                coda_q.append((s, r, slot))
+            if ne:
+                slots = [coda_free.pop() for _ in range(ne)]
+                self.h_coda.index_copy_(0, torch.tensor(slots, dtype=torch.int64, device=self.dev), self.h_exit[:ne])
+                for j, i in enumerate(ex):
+                    s, r = rec[int(i)]
+                    coda_q.append((s, r, slots[j]))
             self.h_rec, self.h_tmp = self.h_tmp, self.h_rec        # survivors become the front of the next batch
             rec = [[rec[int(i)][0], rec[int(i)][1] + 1] for i in surv]
             self.last_lists = (surv.copy(), ex.copy())
@@ -318,6 +329,7 @@ class Engine:
                     while waiting and free_slots and run_prefill():
                         pass
         torch.cuda.synchronize(self.dev)
+        self.stats["end"] = time.perf_counter()
         return {"tokens": [np.asarray(s.tokens, dtype=np.int32) for s in seqs],
                 "depths": [np.asarray(s.depths, dtype=np.int32) for s in seqs],
                 "gates": [s.gates for s in seqs]}
