@@ -35,7 +35,8 @@ class Engine:
                  kv_layout: int = B.KV_SHARED, gate_kind: int = B.GATE_SIGMOID_CDF, q_or_eps: float = 0.5,
                  r_min: int = 1, lookahead: bool = True, mode: str = "refill", min_coda_batch: int = 1,
                  max_prefill_rows: int | None = None, flags: int = 0, record_states: bool = False,
-                 record_logits: bool = False, record_ticks: bool = True, device: str = "cuda:0"):
+                 record_logits: bool = False, record_ticks: bool = True, use_graphs: bool = True,
+                 device: str = "cuda:0"):
         self.dims, self.mode, self.lookahead = dims, mode, lookahead
         self.max_batch, self.max_live, self.min_coda_batch = max_batch, max_live, min_coda_batch
         self.dev = torch.device(device)
@@ -73,6 +74,12 @@ class Engine:
         self.stats = {"recurrent_steps": 0, "row_steps": 0, "coda_calls": 0, "prefill_calls": 0, "tick_rows": []}
         self.trace_states = {}                                        # (sid, token index) -> exit state
         self.trace_logits = {}
+        # Recurrent step as a CUDA graph per row-count bucket (rows padded with seq_id = -1 to a multiple of 32):
+        # the descriptor lives in fixed device arrays refreshed by one host-to-device copy per step.
+        self.use_graphs = use_graphs
+        self.desc_host = torch.zeros((5, max_rows), dtype=torch.int32).pin_memory()
+        self.desc_dev = torch.zeros((5, max_rows), **i32)
+        self.graphs = {}
 
     # ------------------------------------------------------------------ descriptor helpers
     def _rows(self, seq_ids, positions, depths=None, slots=None, forced=None):
@@ -270,17 +277,7 @@ class Engine:
             sl = [live_slot[s] for s, _ in rec]
             pos = [position_of(seqs[s]) for s, _ in rec]
             dep = [r for _, r in rec]
-            rows = self._rows(sl, pos, depths=dep, slots=[self._slot(r) for r in dep],
-                              forced=[forced_for(seqs[s]) for s, _ in rec])
-            hx = self.h_rec[:k]
-            if self.lookahead:               # the stored signal is the previous step's: lists before the step
-                cdb.compact(rows, self.surv_idx, self.exit_idx, self.counts)
-                cdb.loop_step(rows, hx, self.gate_val, self.fire)
-                cdb.gather_rows(hx, self.surv_idx, self.counts[0:1], k, self.h_tmp)
-                cdb.gather_rows(hx, self.exit_idx, self.counts[1:2], k, self.h_exit)
-            else:
-                cdb.loop_step(rows, hx, self.gate_val, self.fire)
-                cdb.compact(rows, self.surv_idx, self.exit_idx, self.counts, h_src=hx, h_next=self.h_tmp, h_exit=self.h_exit)
+            _run_step(self, k, sl, dep, pos, [self._slot(r) for r in dep], [forced_for(seqs[s]) for s, _ in rec])
             cnt = self.counts.cpu().numpy()
             ns, ne = int(cnt[0]), int(cnt[1])
             surv = self.surv_idx[:ns].cpu().numpy()
@@ -298,7 +295,6 @@ class Engine:
                 for j, i in enumerate(ex):
                     s, r = rec[int(i)]
                     coda_q.append((s, r, slots[j]))
-            self.h_rec, self.h_tmp = self.h_tmp, self.h_rec        # survivors become the front of the next batch
             rec = [[rec[int(i)][0], rec[int(i)][1] + 1] for i in surv]
             self.last_lists = (surv.copy(), ex.copy())
             return True
@@ -333,3 +329,55 @@ class Engine:
         return {"tokens": [np.asarray(s.tokens, dtype=np.int32) for s in seqs],
                 "depths": [np.asarray(s.depths, dtype=np.int32) for s in seqs],
                 "gates": [s.gates for s in seqs]}
+
+
+def _bucket(k: int, cap: int) -> int:
+    return min(cap, (k + 31) // 32 * 32)
+
+
+def _static_rows(eng: "Engine", nb: int) -> B.Rows:
+    d = eng.desc_dev
+    return B.Rows(d[0, :nb], d[2, :nb], eng.page_table, loop_depth=d[1, :nb], kv_slot=d[3, :nb], forced_exit=d[4, :nb])
+
+
+def _step_body(eng: "Engine", rows: B.Rows, nb: int):
+    """compaction lists, loop step, survivor / exit gathers; survivors end up at the front of h_rec"""
+    c, hx = eng.cdb, eng.h_rec[:nb]
+    if eng.lookahead:                        # the stored signal is the previous step's: lists before the step
+        c.compact(rows, eng.surv_idx, eng.exit_idx, eng.counts)
+        c.loop_step(rows, hx, eng.gate_val, eng.fire)
+        c.gather_rows(hx, eng.surv_idx, eng.counts[0:1], nb, eng.h_tmp)
+        c.gather_rows(hx, eng.exit_idx, eng.counts[1:2], nb, eng.h_exit)
+    else:
+        c.loop_step(rows, hx, eng.gate_val, eng.fire)
+        c.compact(rows, eng.surv_idx, eng.exit_idx, eng.counts, h_src=hx, h_next=eng.h_tmp, h_exit=eng.h_exit)
+    hx.copy_(eng.h_tmp[:nb])
+
+
+def _run_step(eng: "Engine", k: int, seq, depth, pos, slot, forced):
+    """One recurrent step over the first k rows of h_rec (descriptor given as host sequences)."""
+    nb = _bucket(k, eng.max_rows) if eng.use_graphs else k
+    dh = eng.desc_host
+    dh[0, :k] = torch.as_tensor(np.asarray(seq, dtype=np.int32))
+    dh[1, :k] = torch.as_tensor(np.asarray(depth, dtype=np.int32))
+    dh[2, :k] = torch.as_tensor(np.asarray(pos, dtype=np.int32))
+    dh[3, :k] = torch.as_tensor(np.asarray(slot, dtype=np.int32))
+    dh[4, :k] = torch.as_tensor(np.asarray(forced, dtype=np.int32))
+    dh[0, k:nb] = -1
+    dh[1:, k:nb] = 0
+    if not eng.use_graphs:
+        eng.desc_dev.copy_(dh, non_blocking=True)
+        _step_body(eng, _static_rows(eng, nb), nb)
+        return
+    if nb not in eng.graphs:
+        # warm-up on an all-pad descriptor (touches no state), then capture
+        eng.desc_dev[0, :nb].fill_(-1)
+        rows = _static_rows(eng, nb)
+        _step_body(eng, rows, nb)
+        torch.cuda.synchronize(eng.dev)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            _step_body(eng, rows, nb)
+        eng.graphs[nb] = (g, rows)
+    eng.desc_dev.copy_(dh, non_blocking=True)
+    eng.graphs[nb][0].replay()

@@ -132,3 +132,16 @@ def test_c1_depth_aware_kv_layouts(layout):
     ref = [orc.generate(p, 16, keep_states=True) for p in prompts]
     eng, res = run_engine("refill", n_slots=O.n_slots(o_layout, dims.R), kv_layout=b_layout)
     compare(eng, res, ref)
+
+
+def test_c1_graph_replay_equals_direct_launches(oracle_runs):
+    """The engine replays the recurrent step as a CUDA graph per row-count bucket (rows padded with pads);
+    launching the same calls directly must give the same tokens, depths and states."""
+    eng_g, res_g = run_engine("refill", max_batch=5, max_live=8, use_graphs=True)
+    eng_d, res_d = run_engine("refill", max_batch=5, max_live=8, use_graphs=False)
+    compare(eng_g, res_g, oracle_runs["adaptive"])
+    compare(eng_d, res_d, oracle_runs["adaptive"])
+    for s in range(8):
+        for j in range(1, 16):
+            assert np.array_equal(eng_g.trace_states[(s, j)], eng_d.trace_states[(s, j)])
+    assert eng_g.graphs and not eng_d.graphs
