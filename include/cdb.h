@@ -24,7 +24,10 @@
  *    GEMM A-operands are of the configured dtype (fp32 or bf16); accumulation is fp32.
  *  - A row with seq_id < 0 is a pad: it computes nothing that is visible, writes no KV and
  *    appears in neither compaction list.
- *  - Scratch is per handle: two calls on the same handle must not overlap on the GPU.
+ *  - Scratch is per handle: two calls on the same handle must not overlap on the GPU, with one
+ *    exception: a boundary call (cdb_boundary_embed / _prelude / _coda_lmhead) may run on another
+ *    stream while cdb_loop_step / cdb_compact / cdb_gather_rows run, for rows of other sequences
+ *    (the coda and prelude of exited tokens overlap the next loop step, Fig. 3 of the paper).
  */
 #ifndef CDB_H
 #define CDB_H

@@ -11,6 +11,10 @@
 
 using namespace cdbk;
 
+// The boundary stages (embedding / prelude, coda / LM head) use scratch lane 1 and the loop step lane 0, so a
+// boundary call on one stream may overlap a loop step on another (the two-stream half-batch mode also uses
+// lane 1 and must not be combined with that).
+constexpr int kBoundaryLane = 1;
 constexpr int kMinSplitRows = 64;          // below this a loop step runs as one batch on one stream
 constexpr int kSplitGemmSmemBytes = 0;            // no cap: a projection CTA co-resides with attention only when its ring is large
 constexpr int kSplitAttnCtasPerSm = 3;     // attention CTAs per SM when two half-batches share the GPU
@@ -162,11 +166,11 @@ void core_layers(cdb_t* h, int ln, const RowsDev& rows, float* x, cudaStream_t s
 }
 
 // final RMSNorm + LM head + greedy argmax on n rows of x
-void lm_head(cdb_t* h, const RowsDev& rows, const float* x, int32_t* token_out, float* logits_out, cudaStream_t st) {
+void lm_head(cdb_t* h, int ln, const RowsDev& rows, const float* x, int32_t* token_out, float* logits_out, cudaStream_t st) {
     const cdb_config_t& c = h->cfg;
     float* logits = logits_out ? logits_out : h->logits;
-    launch_rmsnorm(h, x, h->g_final, h->lane[0].xn, rows, st);
-    launch_linear(h, h->lane[0].xn, h->w.W_lm, logits, rows.n_rows, c.V, c.d, Epilogue::Store, st);
+    launch_rmsnorm(h, x, h->g_final, h->lane[ln].xn, rows, st);
+    launch_linear(h, h->lane[ln].xn, h->w.W_lm, logits, rows.n_rows, c.V, c.d, Epilogue::Store, st);
     launch_argmax(h, logits, rows.n_rows, token_out, st);
 }
 
@@ -249,7 +253,7 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
     CDB_ALLOC(h->gate_fire, uint8_t, c.max_seqs);
     for (int ln = 0; ln < 2; ++ln) {
         Lane& L = h->lane[ln];
-        L.rows_cap = ln == 0 ? c.max_rows : (c.max_rows + 1) / 2;
+        L.rows_cap = c.max_rows;
         const size_t r = L.rows_cap;
         CDB_ALLOC(L.xn, char, r * wide * h->elem_size);
         CDB_ALLOC(L.qrot, char, r * d * h->elem_size);
@@ -361,8 +365,8 @@ static int boundary_in(cdb_t* h, const int32_t* token_ids, const cdb_rows_t* row
     if (prelude && h->cfg.L_pre > 0) {
         if (!h->pool.base) return fail(h, CDB_ERR_STATE, "no KV pool bound");
         rd.slot_override = 0;
-        launch_attention_plan(h, 0, rd, st);
-        for (int l = 0; l < h->cfg.L_pre; ++l) layer_forward(h, 0, l, rd, h_out, st);
+        launch_attention_plan(h, kBoundaryLane, rd, st);
+        for (int l = 0; l < h->cfg.L_pre; ++l) layer_forward(h, kBoundaryLane, l, rd, h_out, st);
     }
     return check_launch(h, "cdb_boundary_embed/prelude");
 }
@@ -464,10 +468,10 @@ int cdb_boundary_coda_lmhead(cdb_t* h, const cdb_rows_t* rows, float* h_exit, in
     if (c.L_coda > 0) {
         if (!h->pool.base) return fail(h, CDB_ERR_STATE, "no KV pool bound");
         rd.slot_override = 0;
-        launch_attention_plan(h, 0, rd, st);
-        for (int l = c.L_pre + c.L_core; l < c.L_pre + c.L_core + c.L_coda; ++l) layer_forward(h, 0, l, rd, h_exit, st);
+        launch_attention_plan(h, kBoundaryLane, rd, st);
+        for (int l = c.L_pre + c.L_core; l < c.L_pre + c.L_core + c.L_coda; ++l) layer_forward(h, kBoundaryLane, l, rd, h_exit, st);
     }
-    lm_head(h, rd, h_exit, token_out, logits_out, st);
+    lm_head(h, kBoundaryLane, rd, h_exit, token_out, logits_out, st);
     return check_launch(h, "cdb_boundary_coda_lmhead");
 }
 
@@ -502,7 +506,7 @@ int cdb_prefill(cdb_t* h, const int32_t* token_ids, const cdb_rows_t* rows, cons
         RowsDev re = rd;
         re.n_rows = n_emit;
         re.seq_id = nullptr;
-        lm_head(h, re, h->h_prev, token_out, logits_out, st);
+        lm_head(h, 0, re, h->h_prev, token_out, logits_out, st);
     }
     return check_launch(h, "cdb_prefill");
 }

@@ -1,0 +1,303 @@
+"""Pipelined (asynchronous) driver of the CDB hot path, refill mode with the lookahead gate.
+
+What the paper's section 4.3 / Fig. 3 describes: while the GPU runs loop step N, the host already knows
+which rows leave after it (the exit flag of step N depends only on the signal stored by step N-1, so the
+compaction lists are computed at the START of step N), prepares the descriptor of step N+1 and enqueues
+it; the coda + sampling + prelude of the rows that left after step N-1 run on a second stream beside loop
+step N, and their tokens rejoin the recurrent batch at step N+1.  The main stream therefore never waits
+for the host or for a boundary stage.
+
+Streams and buffers
+  main  H2D descriptor -> cdb_compact (lists) -> [event] -> CUDA graph (loop step, survivor gather to the
+        front of h_rec, exit gather to h_exit[parity]) -> refill gather
+  side  D2H lists; copy of exited rows into the coda queue; cdb_boundary_coda_lmhead; D2H tokens;
+        cdb_boundary_embed / _prelude of the sampled tokens into h_ready
+Results (tokens, exit depths) are those of the synchronous engine and of the CPU oracle: scheduling
+changes when work runs, never what is computed.
+"""
+from __future__ import annotations
+
+import time
+
+import numpy as np
+import torch
+
+from . import binding as B
+from .engine import Engine, _bucket, _static_rows
+
+
+class PipelinedEngine(Engine):
+    def __init__(self, *a, **kw):
+        kw.setdefault("mode", "refill")
+        kw.setdefault("lookahead", True)
+        super().__init__(*a, **kw)
+        if self.mode != "refill" or not self.lookahead:
+            raise ValueError("the pipelined engine implements refill mode with the lookahead gate")
+        self.side = torch.cuda.Stream(device=self.dev)
+        d = self.dims.d
+        self.h_exit2 = [torch.zeros((self.max_rows, d), dtype=torch.float32, device=self.dev) for _ in range(2)]
+        self.h_coda_in = torch.zeros((self.cap, d), dtype=torch.float32, device=self.dev)
+        self.h_pre_out = torch.zeros((self.cap, d), dtype=torch.float32, device=self.dev)
+        self.lists_host = torch.zeros((2 * self.max_rows + 2,), dtype=torch.int32).pin_memory()
+        self.lists_dev = torch.zeros((2 * self.max_rows + 2,), dtype=torch.int32, device=self.dev)
+        self.pgraphs = {}
+
+    # ---- graph of one step body for (bucket, parity): loop step + gathers; compaction runs before it
+    def _body(self, rows, nb, parity):
+        c, hx = self.cdb, self.h_rec[:nb]
+        c.loop_step(rows, hx, self.gate_val, self.fire)
+        c.gather_rows(hx, self.surv_idx, self.counts[0:1], nb, self.h_tmp)
+        c.gather_rows(hx, self.exit_idx, self.counts[1:2], nb, self.h_exit2[parity])
+        hx.copy_(self.h_tmp[:nb])
+
+    def _capture_all(self):
+        """Graphs for every row-count bucket and both parities, captured before any live row exists (the
+        warm-up run of a capture scribbles over h_rec)."""
+        nb = 32
+        while True:
+            nb = min(nb, self.max_rows)
+            for parity in (0, 1):
+                if (nb, parity) in self.pgraphs:
+                    continue
+                self.desc_dev[0, :nb].fill_(-1)                   # all pads: the warm-up touches no model state
+                rows = _static_rows(self, nb)
+                self.cdb.compact(rows, self.surv_idx, self.exit_idx, self.counts)
+                self._body(rows, nb, parity)
+                torch.cuda.synchronize(self.dev)
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    self._body(rows, nb, parity)
+                self.pgraphs[(nb, parity)] = (g, rows)
+            if nb >= _bucket(self.max_batch, self.max_rows):
+                break
+            nb += 32
+        torch.cuda.synchronize(self.dev)
+
+    # ------------------------------------------------------------------ generation
+    def generate(self, prompts, T, forced_depths=None, teacher_tokens=None):
+        """Same contract as Engine.generate (teacher tokens are not supported: sampled tokens stay on the
+        device and feed the prelude directly).  Gate values are not read back."""
+        if teacher_tokens is not None:
+            raise ValueError("lock-step replay needs the synchronous engine")
+        dims, cdb, dev = self.dims, self.cdb, self.dev
+        main, side = torch.cuda.current_stream(dev), self.side
+        n = len(prompts)
+        Ts = [T] * n if np.isscalar(T) else list(T)
+        P = [len(p) for p in prompts]
+        tokens = [[None] * Ts[i] for i in range(n)]
+        depths = [[] for _ in range(n)]
+        gen = [0] * n                                   # tokens sampled so far (values may still be in flight)
+        waiting, live_slot = list(range(n)), {}
+        free_slots = list(range(self.max_live - 1, -1, -1))
+        ready, ready_free = [], list(range(self.cap - 1, -1, -1))     # (sid, slot in h_ready, event, iteration)
+        coda_q, coda_free = [], list(range(self.cap - 1, -1, -1))     # (sid, depth, slot in h_coda)
+        pending_tokens, pending_release = [], []
+        ring = [torch.zeros((5, self.max_rows), dtype=torch.int32).pin_memory() for _ in range(4)]
+        tok_ring = [torch.zeros(self.cap, dtype=torch.int32).pin_memory() for _ in range(16)]
+        tok_dev = torch.zeros(self.cap, dtype=torch.int32, device=dev)
+        counts_h = torch.zeros(2, dtype=torch.int32).pin_memory()
+        surv_h = torch.zeros(self.max_rows, dtype=torch.int32).pin_memory()
+        exit_h = torch.zeros(self.max_rows, dtype=torch.int32).pin_memory()
+        i64 = lambda a: torch.tensor(a, dtype=torch.int64, device=dev)
+        i32 = lambda a: torch.tensor(np.asarray(a, dtype=np.int32), dtype=torch.int32, device=dev)
+        self._capture_all()
+        self.stats["start"] = time.perf_counter()
+        x_done = [None, None]                           # h_exit2[parity] copied out (event on the side stream)
+        gather_done = None                              # last refill gather on the main stream
+        tok_calls = 0
+
+        def forced_for(s):
+            if forced_depths is not None and forced_depths[s] is not None:
+                return int(forced_depths[s][gen[s] - 1])
+            return 0
+
+        def drain_tokens(block):
+            while pending_tokens and (block or pending_tokens[0][0].query()):
+                ev, buf, items = pending_tokens.pop(0)
+                ev.synchronize()
+                vals = buf.numpy()
+                for j, (s, idx) in enumerate(items):
+                    tokens[s][idx] = int(vals[j])
+            while pending_release and (block or pending_release[0][0].query()):
+                ev, s = pending_release.pop(0)
+                ev.synchronize()
+                self._release_pages(live_slot[s])
+                free_slots.append(live_slot.pop(s))
+
+        def enqueue_prelude(sids, tok_t, stream, it):
+            """prelude of the device-resident input tokens tok_t of sequences sids -> h_ready; on `stream`"""
+            sl = [live_slot[s] for s in sids]
+            pos = [P[s] + gen[s] - 1 for s in sids]
+            rows = B.Rows(i32(sl), i32(pos), self.page_table)
+            out = self.h_pre_out[:len(sids)]
+            (cdb.boundary_prelude if dims.L_pre > 0 else cdb.boundary_embed)(tok_t, rows, out, stream=stream)
+            slots = [ready_free.pop() for _ in sids]
+            if gather_done is not None:
+                stream.wait_event(gather_done)          # a freed h_ready slot may still be read by the last refill gather
+            self.h_ready.index_copy_(0, i64(slots), out)
+            ev = torch.cuda.Event()
+            ev.record(stream)
+            ready.extend((s, slot, ev, it) for s, slot in zip(sids, slots))
+
+        def admit():
+            """prompt processing of waiting requests while live slots and pages are free (drains the pipeline)"""
+            side.synchronize()
+            drain_tokens(True)
+            while waiting and free_slots:
+                batch, rows_total = [], 0
+                while waiting and free_slots and rows_total + P[waiting[0]] <= self.max_rows:
+                    s = waiting[0]
+                    if not self._reserve_pages(free_slots[-1], P[s] + Ts[s]):
+                        break
+                    live_slot[s] = free_slots.pop()
+                    waiting.pop(0)
+                    batch.append(s)
+                    rows_total += P[s]
+                if not batch:
+                    break
+                toks = np.concatenate([np.asarray(prompts[s], dtype=np.int32) for s in batch])
+                sl = np.concatenate([np.full(P[s], live_slot[s]) for s in batch])
+                pos = np.concatenate([np.arange(P[s]) for s in batch])
+                ends = np.cumsum([P[s] for s in batch]) - 1
+                m = len(batch)
+                cdb.prefill(i32(toks), B.Rows(i32(sl), i32(pos), self.page_table), i32(ends), tok_dev[:m])
+                vals = tok_dev[:m].cpu().numpy()
+                self.stats["prefill_calls"] += 1
+                cont = []
+                for j, s in enumerate(batch):
+                    tokens[s][0] = int(vals[j])
+                    gen[s] = 1
+                    if gen[s] >= Ts[s]:
+                        self._release_pages(live_slot[s])
+                        free_slots.append(live_slot.pop(s))
+                    else:
+                        cont.append(j)
+                if cont:
+                    enqueue_prelude([batch[j] for j in cont], tok_dev[:m][i64(cont)].contiguous(), main, -1)
+            torch.cuda.synchronize(dev)
+
+        def boundary_for(prev, it, force):
+            """side stream: queue the rows that left after the previous step, run the coda (+ sampling) when
+            enough have gathered, and the prelude of the sampled tokens"""
+            nonlocal tok_calls
+            with torch.cuda.stream(side):
+                if prev is not None and prev["ne"]:
+                    side.wait_event(prev["G"])
+                    slots = [coda_free.pop() for _ in range(prev["ne"])]
+                    self.h_coda.index_copy_(0, i64(slots), self.h_exit2[prev["parity"]][:prev["ne"]])
+                    ev = torch.cuda.Event()
+                    ev.record(side)
+                    x_done[prev["parity"]] = ev
+                    coda_q.extend((s, r, slot) for (s, r), slot in zip(prev["exits"], slots))
+                if not coda_q or (len(coda_q) < self.min_coda_batch and not force):
+                    return
+                items = list(coda_q)
+                coda_q.clear()
+                m = len(items)
+                hin = self.h_coda_in[:m]
+                cdb.gather_rows(self.h_coda, i32([it_[2] for it_ in items]), None, m, hin, stream=side)
+                sids = [it_[0] for it_ in items]
+                rows = B.Rows(i32([live_slot[s] for s in sids]), i32([P[s] + gen[s] - 1 for s in sids]), self.page_table)
+                if self.kv_layout == B.KV_DEPTH_INDEXED:
+                    cdb.kv_copy_on_exit(rows, i32([it_[1] for it_ in items]), stream=side)
+                cdb.boundary_coda_lmhead(rows, hin, tok_dev[:m], stream=side)
+                buf = tok_ring[tok_calls % len(tok_ring)][:m]
+                tok_calls += 1
+                buf.copy_(tok_dev[:m], non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(side)
+                pending_tokens.append((ev, buf, [(s, gen[s]) for s in sids]))
+                self.stats["coda_calls"] += 1
+                cont = []
+                for j, (s, r, slot) in enumerate(items):
+                    coda_free.append(slot)
+                    gen[s] += 1
+                    if gen[s] >= Ts[s]:
+                        pending_release.append((ev, s))
+                    else:
+                        cont.append(j)
+                if cont:
+                    enqueue_prelude([sids[j] for j in cont], tok_dev[:m][i64(cont)].contiguous(), side, it)
+
+        rec, prev, it = [], None, 0
+        while True:
+            drain_tokens(False)
+            if waiting and free_slots:
+                admit()
+            if "decode_start" not in self.stats and not waiting:
+                torch.cuda.synchronize(dev)
+                self.stats["decode_start"] = time.perf_counter()
+            # ---- refills whose prelude was enqueued in an earlier iteration join this step
+            take = []
+            while ready and len(rec) + len(take) < self.max_batch and ready[0][3] < it:
+                take.append(ready.pop(0))
+            if take:
+                for _, _, ev, _ in take:
+                    if ev is not None:
+                        main.wait_event(ev)
+                cdb.gather_rows(self.h_ready, i32([t[1] for t in take]), None, len(take),
+                                self.h_rec[len(rec):len(rec) + len(take)])
+                gather_done = torch.cuda.Event()
+                gather_done.record(main)
+                for s, slot, _, _ in take:
+                    ready_free.append(slot)
+                    rec.append([s, 1])
+            k = len(rec)
+            step = None
+            if k:
+                parity = it & 1
+                nb = _bucket(k, self.max_rows)
+                dh = ring[it % len(ring)]
+                dh[0, :k] = torch.as_tensor(np.asarray([live_slot[s] for s, _ in rec], dtype=np.int32))
+                dh[1, :k] = torch.as_tensor(np.asarray([r for _, r in rec], dtype=np.int32))
+                dh[2, :k] = torch.as_tensor(np.asarray([P[s] + gen[s] - 1 for s, _ in rec], dtype=np.int32))
+                dh[3, :k] = torch.as_tensor(np.asarray([self._slot(r) for _, r in rec], dtype=np.int32))
+                dh[4, :k] = torch.as_tensor(np.asarray([forced_for(s) for s, _ in rec], dtype=np.int32))
+                dh[0, k:nb] = -1
+                dh[1:, k:nb] = 0
+                self.desc_dev.copy_(dh, non_blocking=True)
+                g, rows = self.pgraphs[(nb, parity)]
+                cdb.compact(rows, self.surv_idx, self.exit_idx, self.counts)
+                lists_ready = torch.cuda.Event()
+                lists_ready.record(main)
+                if x_done[parity] is not None:
+                    main.wait_event(x_done[parity])         # the exits of two steps ago have left h_exit2[parity]
+                g.replay()
+                G = torch.cuda.Event()
+                G.record(main)
+                with torch.cuda.stream(side):
+                    side.wait_event(lists_ready)
+                    counts_h.copy_(self.counts, non_blocking=True)
+                    surv_h[:nb].copy_(self.surv_idx[:nb], non_blocking=True)
+                    exit_h[:nb].copy_(self.exit_idx[:nb], non_blocking=True)
+                    lists_copied = torch.cuda.Event()
+                    lists_copied.record(side)
+                step = (parity, G, lists_copied)
+            # ---- boundary stages of the rows that left after the previous step, beside this step
+            idle = not k and not ready
+            boundary_for(prev, it, force=idle or self.min_coda_batch <= 1)
+            prev = None
+            if step is not None:
+                parity, G, lists_copied = step
+                lists_copied.synchronize()
+                ns, ne = int(counts_h[0]), int(counts_h[1])
+                surv, ex = surv_h[:ns].numpy().copy(), exit_h[:ne].numpy().copy()
+                exits = [(rec[int(i)][0], rec[int(i)][1]) for i in ex]
+                for s, r in exits:
+                    depths[s].append(r)
+                self.stats["recurrent_steps"] += 1
+                self.stats["row_steps"] += k
+                prev = {"parity": parity, "ne": ne, "exits": exits, "G": G}
+                rec = [[rec[int(i)][0], rec[int(i)][1] + 1] for i in surv]
+            it += 1
+            if not rec and prev is None and not ready and not coda_q and not waiting:
+                if all(gen[s] >= Ts[s] for s in range(n)):
+                    break
+                if not pending_tokens and not pending_release:
+                    raise RuntimeError("pipelined scheduler stalled")
+                drain_tokens(True)
+        torch.cuda.synchronize(dev)
+        drain_tokens(True)
+        self.stats["end"] = time.perf_counter()
+        return {"tokens": [np.asarray(t, dtype=np.int32) for t in tokens],
+                "depths": [np.asarray(d, dtype=np.int32) for d in depths], "gates": None}

@@ -16,6 +16,7 @@ import torch
 from . import binding as B
 from . import synth
 from .engine import Engine
+from .engine_async import PipelinedEngine
 
 
 def flop_bound(dims, mean_depth):
@@ -26,18 +27,18 @@ def flop_bound(dims, mean_depth):
 
 
 def run(dims, weights, prompts, T, *, mode, gate_kind, q_or_eps=0.5, forced_depths=None, max_batch=None, max_live=None,
-        min_coda_batch=1, max_prefill_rows=4096):
+        min_coda_batch=1, max_prefill_rows=4096, pipelined=False):
     n, P = len(prompts), max(len(p) for p in prompts)
     live = min(n, max_live or n)
     pages = live * ((P + T + dims.page_size - 1) // dims.page_size)
-    eng = Engine(dims, weights, max_batch=min(max_batch or n, live), max_live=live, max_len=P + T, n_pages=pages, gate_kind=gate_kind,
+    eng = (PipelinedEngine if pipelined else Engine)(dims, weights, max_batch=min(max_batch or n, live), max_live=live, max_len=P + T, n_pages=pages, gate_kind=gate_kind,
                  q_or_eps=q_or_eps, lookahead=True, mode=mode, min_coda_batch=min_coda_batch,
                  max_prefill_rows=max_prefill_rows, record_ticks=False)
     res = eng.generate(prompts, T, forced_depths=forced_depths)
     st = eng.stats
     depths = np.concatenate(res["depths"])
     decode_s = st["end"] - st["decode_start"]
-    out = {"mode": mode, "max_batch": eng.max_batch, "max_live": live, "total_s": st["end"] - st["start"],
+    out = {"mode": mode + ("_pipelined" if pipelined else ""), "max_batch": eng.max_batch, "max_live": live, "total_s": st["end"] - st["start"],
            "generated_tokens_per_s_end_to_end": sum(len(t) for t in res["tokens"]) / (st["end"] - st["start"]),
            "decode_s": decode_s, "prefill_s": st["decode_start"] - st["start"],
            "decode_tokens_per_s": len(depths) / decode_s, "token_loop_steps_per_s": st["row_steps"] / decode_s,
@@ -77,7 +78,7 @@ def main():
     ap.add_argument("--max-batch", type=int, default=0)
     ap.add_argument("--min-coda-batch", type=int, default=0)
     ap.add_argument("--max-live", type=int, default=0, help="sequences resident at once (0 = all); fewer than --seqs queues the rest")
-    ap.add_argument("--modes", default="cb,refill,no_refill")
+    ap.add_argument("--modes", default="cb,refill,no_refill", help="cb, refill, no_refill, refill_pipelined")
     args = ap.parse_args()
     torch.cuda.set_device(0)
     if args.model == "ouro":
@@ -101,13 +102,15 @@ def main():
         forced = [list(r) for r in synth.forced_exit_depths((args.seqs, args.tokens - 1), seed, 12.0, dims.R)]
         min_coda = args.min_coda_batch or 32
     for mode in args.modes.split(","):
-        out, _ = run(dims, w, prompts, args.tokens, mode=mode, gate_kind=gate_kind, forced_depths=None if mode == "cb" else forced,
+        pipelined = mode.endswith("_pipelined")
+        mode = mode.replace("_pipelined", "")
+        out, _ = run(dims, w, prompts, args.tokens, mode=mode, pipelined=pipelined, gate_kind=gate_kind, forced_depths=None if mode == "cb" else forced,
                      max_batch=args.max_batch or None, max_live=args.max_live or None, min_coda_batch=min_coda)
         report["runs"].append(out)
         print(json.dumps(out), flush=True)
     by = {r["mode"]: r for r in report["runs"]}
     if "cb" in by:
-        for m in ("refill", "no_refill"):
+        for m in ("refill", "no_refill", "refill_pipelined"):
             if m in by:
                 key = "decode_tokens_per_s" if not args.max_live else "generated_tokens_per_s_end_to_end"
                 by[m]["speedup_vs_fixed_depth"] = by[m][key] / by["cb"][key]

@@ -145,3 +145,24 @@ def test_c1_graph_replay_equals_direct_launches(oracle_runs):
         for j in range(1, 16):
             assert np.array_equal(eng_g.trace_states[(s, j)], eng_d.trace_states[(s, j)])
     assert eng_g.graphs and not eng_d.graphs
+
+
+@pytest.mark.parametrize("max_batch,max_live", [(8, 8), (3, 4)])
+def test_c1_pipelined_engine_gives_the_same_tokens(oracle_runs, max_batch, max_live):
+    """Asynchronous pipeline (compaction lists read at the start of a step, coda + prelude of exited rows on
+    a second stream beside the next step, refills one step later): scheduling changes when work runs, not
+    what is computed, so tokens and exit depths must equal the oracle's."""
+    from paper_2608_09444_b200 import binding as B
+    from paper_2608_09444_b200.engine_async import PipelinedEngine
+    dims, w, prompts = c1_inputs()
+    wd = {k: v.cuda() for k, v in w.items()}
+    eng = PipelinedEngine(dims, wd, max_batch=max_batch, max_live=max_live, max_len=48, n_pages=3 * max_live,
+                          gate_kind=B.GATE_SIGMOID_CDF, q_or_eps=0.5, max_prefill_rows=256)
+    res = eng.generate(list(prompts), 16)
+    assert eng.cdb.poll_status() == 0
+    ref = oracle_runs["adaptive"]
+    for s in range(8):
+        assert np.array_equal(res["tokens"][s], ref[s]["tokens"]), s
+        assert np.array_equal(res["depths"][s], ref[s]["depths"]), s
+    assert eng.stats["row_steps"] == int(sum(r["depths"].sum() for r in ref))
+    assert not [p for row in eng.page_table_host for p in row if p >= 0]
