@@ -134,6 +134,8 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     static const bool no_pdl = getenv("CDB_NO_PDL") != nullptr;      // tuning aid: plain stream-ordered launches
     cfg.attrs = attr; cfg.numAttrs = no_pdl ? 0 : 1;
+    static const int carve = getenv("CDB_MISC_CARVEOUT") ? atoi(getenv("CDB_MISC_CARVEOUT")) : -2;   // tuning aid
+    if (carve > -2) cudaFuncSetAttribute((const void*)kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve);
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 }  // namespace cdbk

@@ -174,7 +174,9 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
     const uint32_t tmem_base = tmem_base_slot;
     volatile int* abortp = &abort_flag;
     if (p.dbg && threadIdx.x == 0) p.dbg[blockIdx.x * 8 + 1] = gtime();
-    pdl_wait();                 // set-up above overlaps the previous kernel's tail; operands are read only from here on
+    // Set-up above overlaps the previous kernel's tail.  The weights do not depend on that kernel, so the
+    // producer warp starts their copies before it waits (below); every other warp waits here.
+    if (warp != 0) pdl_wait();
 
     const int n_ftiles = (p.N + BM - 1) / BM, n_rtiles = (p.n + BN - 1) / BN;
     const int n_tiles = n_ftiles * n_rtiles * p.k_splits;                   // tile t = (split, row tile, feature tile)
@@ -187,24 +189,51 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
             const bool leader = elect_one();
             int s = 0; uint32_t ph = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-                const int f0 = (t % n_ftiles) * BM, r0 = (t / n_ftiles % n_rtiles) * BN;
-                // Every CTA walks its k-blocks from a different starting point (a function of its feature
-                // tile only), so that the CTAs do not all pull the same activation lines from L2 at once.
-                const int kb0 = kb_begin(t), nk = kb_end(t) - kb0, rot = ((t % n_ftiles) * 7) % nk;
-                for (int j = 0; j < nk; ++j) {
-                    const int kb = kb0 + (j + rot) % nk;
-                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abortp)) { ok = false; break; }
-                    const uint32_t dst = ring + (uint32_t)s * stage_bytes;
-                    const int wc = p.w_tiled ? 0 : kb * BK, wr = p.w_tiled ? ((f0 / BM) * n_kb + kb) * BM : f0;
-                    if (leader) {
-                        mbar_expect_tx(full_bar(s), stage_bytes);
-                        tma_load_2d(dst, &map_w, full_bar(s), wc, wr);
-                        if (dual) tma_load_2d(dst + w_bytes, &map_w2, full_bar(s), wc, wr);
-                        tma_load_2d(dst + x_off, &map_x, full_bar(s), kb * BK, r0);
+            // The first fill of the ring runs in two passes over the same (tile, k-block) sequence: pass 0
+            // arms the stage barriers and starts the weight copies, then the warp waits for the previous
+            // kernel, and pass 1 adds the activation copies.  Later stages take both copies at once.
+            int n_pre = 0;                                   // stages filled by pass 0
+            for (int pass = 0; pass < 2; ++pass) {
+                if (pass == 1) pdl_wait();
+                int g = 0;                                   // position in this CTA's (tile, k-block) sequence
+                for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+                    const int f0 = (t % n_ftiles) * BM, r0 = (t / n_ftiles % n_rtiles) * BN;
+                    // Every CTA walks its k-blocks from a different starting point (a function of its feature
+                    // tile only), so that the CTAs do not all pull the same activation lines from L2 at once.
+                    const int kb0 = kb_begin(t), nk = kb_end(t) - kb0, rot = ((t % n_ftiles) * 7) % nk;
+                    if (pass == 0 && g >= S) break;
+                    for (int j = 0; j < nk; ++j, ++g) {
+                        if (pass == 0 && g >= S) break;
+                        const int kb = kb0 + (j + rot) % nk;
+                        const int wc = p.w_tiled ? 0 : kb * BK, wr = p.w_tiled ? ((f0 / BM) * n_kb + kb) * BM : f0;
+                        if (pass == 0) {                     // ring is empty: stage g is free
+                            const uint32_t dst = ring + (uint32_t)g * stage_bytes;
+                            if (leader) {
+                                mbar_expect_tx(full_bar(g), stage_bytes);
+                                tma_load_2d(dst, &map_w, full_bar(g), wc, wr);
+                                if (dual) tma_load_2d(dst + w_bytes, &map_w2, full_bar(g), wc, wr);
+                            }
+                            __syncwarp();
+                            n_pre = g + 1;
+                            continue;
+                        }
+                        if (g < n_pre) {
+                            if (leader) tma_load_2d(ring + (uint32_t)g * stage_bytes + x_off, &map_x, full_bar(g), kb * BK, r0);
+                            __syncwarp();
+                            if (++s == S) { s = 0; ph ^= 1u; }
+                            continue;
+                        }
+                        if (!mbar_wait(empty_bar(s), ph ^ 1u, abortp)) { ok = false; break; }
+                        const uint32_t dst = ring + (uint32_t)s * stage_bytes;
+                        if (leader) {
+                            mbar_expect_tx(full_bar(s), stage_bytes);
+                            tma_load_2d(dst, &map_w, full_bar(s), wc, wr);
+                            if (dual) tma_load_2d(dst + w_bytes, &map_w2, full_bar(s), wc, wr);
+                            tma_load_2d(dst + x_off, &map_x, full_bar(s), kb * BK, r0);
+                        }
+                        __syncwarp();
+                        if (++s == S) { s = 0; ph ^= 1u; }
                     }
-                    __syncwarp();
-                    if (++s == S) { s = 0; ph ^= 1u; }
                 }
             }
             if (!ok || *abortp) {                        // give copies already in flight time to land

@@ -48,3 +48,14 @@ def test_two_ranks_shard_and_reduce():
     assert abs(len(shards[0]) - len(shards[1])) <= 1
     assert [r[2] for r in res] == [11.0, 11.0]                 # both ranks see the slowest rank's time
     assert res[0][3] != res[1][3]                              # weak scaling: each rank has its own rows
+
+
+def test_latency_model_fit_recovers_its_coefficients():
+    """The least-squares fit of t = delta + gamma N_b + alpha N_c (section 5) returns the coefficients
+    that generated exact synthetic points, and B* follows delta / (gamma + alpha L)."""
+    from paper_2608_09444_b200.sweep import fit
+    d, g, a = 1.7, 2.5e-3, 3.1e-5
+    pts = [[nb, L, d + g * nb + a * nb * L] for nb in (1, 8, 64, 256) for L in (128, 2048, 8192)]
+    f = fit(pts)
+    assert abs(f["delta_ms"] - d) < 1e-9 and abs(f["gamma_ms_per_row"] - g) < 1e-11 and abs(f["alpha_ms_per_token"] - a) < 1e-13
+    assert f["r2"] > 1 - 1e-12 and f["max_rel_residual"] < 1e-9
