@@ -24,6 +24,7 @@ GATE_NONE, GATE_SIGMOID_CDF, GATE_L2_CONVERGENCE = 0, 1, 2
 FLAG_SIMT_GEMM = 1
 FLAG_TWO_STREAM = 2
 FLAG_UNFUSED_LAYER = 4
+FLAG_SIMT_PREFILL = 8
 
 EXPORTS = ["cdb_create", "cdb_destroy", "cdb_last_error", "cdb_kv_bind", "cdb_set_gate", "cdb_boundary_embed",
            "cdb_boundary_prelude", "cdb_loop_step", "cdb_compact", "cdb_gather_rows", "cdb_boundary_coda_lmhead",

@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libcdb.so")
-SOURCES = ["cdb_api.cu", "kernels_misc.cu", "attention.cu", "gemm_simt.cu", "gemm_tcgen05.cu"]
+SOURCES = ["cdb_api.cu", "kernels_misc.cu", "attention.cu", "attention_prefill_tc.cu", "gemm_simt.cu", "gemm_tcgen05.cu"]
 
 
 def _stale(target: str, deps: list[str]) -> bool:

@@ -452,23 +452,57 @@ namespace {
 constexpr int kPfTile = 32;                 // query rows per tile
 
 // Cuts the batch into tiles: maximal runs of rows with the same sequence and consecutive positions, in
-// pieces of at most kPfTile rows.  tiles[i] = first row, tile_rows[i] = rows in it.  One thread: n_rows is small.
-__global__ void prefill_plan_kernel(RowsDev rows, int32_t* __restrict__ tiles, int32_t* __restrict__ tile_rows,
-                                    int32_t* __restrict__ n_tiles) {
+// pieces of at most `tile` rows.  tiles[i] = first row, tile_rows[i] = rows in it, in row order.  One CTA of
+// 1024 threads walks the rows in chunks: a max-scan finds each row's run start, a sum-scan numbers the tiles.
+__global__ void __launch_bounds__(1024) prefill_plan_kernel(RowsDev rows, int tile, int32_t* __restrict__ tiles,
+                                                            int32_t* __restrict__ tile_rows, int32_t* __restrict__ n_tiles) {
     pdl_trigger();
     pdl_wait();
-    if (blockIdx.x != 0 || threadIdx.x != 0) return;
-    int nt = 0, r = 0;
-    while (r < rows.n_rows) {
-        if (rows.seq_id[r] < 0) { ++r; continue; }
-        int len = 1;
-        while (r + len < rows.n_rows && len < kPfTile && rows.seq_id[r + len] == rows.seq_id[r] &&
-               rows.position[r + len] == rows.position[r] + len)
-            ++len;
-        tiles[nt] = r; tile_rows[nt] = len; ++nt;
-        r += len;
+    __shared__ int w_max[32], w_sum[32];
+    __shared__ int carry_run, carry_cnt;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int r = tid; r < rows.n_rows; r += 1024) tile_rows[r] = 0;
+    if (tid == 0) { carry_run = -1; carry_cnt = 0; }
+    __syncthreads();
+    for (int base = 0; base < rows.n_rows; base += 1024) {
+        const int r = base + tid;
+        bool valid = false, start = false;
+        if (r < rows.n_rows) {
+            const int sq = rows.seq_id[r];
+            valid = sq >= 0;
+            if (valid) {
+                start = r == 0;
+                if (!start) {
+                    const int sp = rows.seq_id[r - 1];
+                    start = sp != sq || rows.position[r] != rows.position[r - 1] + 1;
+                }
+            }
+        }
+        // inclusive max-scan of (start ? r : -1), seeded with the run start carried from the previous chunk
+        int rs = start ? r : -1;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) { const int o = __shfl_up_sync(0xffffffffu, rs, d); if (lane >= d) rs = max(rs, o); }
+        if (lane == 31) w_max[warp] = rs;
+        __syncthreads();
+        int pre = carry_run;
+        for (int w = 0; w < warp; ++w) pre = max(pre, w_max[w]);
+        rs = max(rs, pre);
+        const bool ts = valid && ((r - rs) % tile == 0);
+        int cnt = ts ? 1 : 0;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) { const int o = __shfl_up_sync(0xffffffffu, cnt, d); if (lane >= d) cnt += o; }
+        if (lane == 31) w_sum[warp] = cnt;
+        __syncthreads();
+        int pre_c = carry_cnt;
+        for (int w = 0; w < warp; ++w) pre_c += w_sum[w];
+        cnt += pre_c;                                                   // tiles started at or before this row
+        if (ts) tiles[cnt - 1] = r;
+        if (valid) atomicAdd(&tile_rows[cnt - 1], 1);
+        __syncthreads();
+        if (tid == 1023) { carry_run = rs; carry_cnt = cnt; }
+        __syncthreads();
     }
-    *n_tiles = nt;
+    if (tid == 0) *n_tiles = carry_cnt;
 }
 
 template <typename T, int DH>
@@ -582,13 +616,23 @@ __global__ void __launch_bounds__(128) attn_prefill_kernel(AttnParams p, const i
     }
 }
 
+}  // namespace
+
+// Tile list of a prompt batch into the lane's split-scan buffer (first rows), pf_tile_rows and pf_n_tiles.
+void launch_prefill_plan(const cdb* h, int ln, const RowsDev& rows, int tile, cudaStream_t st) {
+    const Lane& L = h->lane[ln];
+    CDB_LAUNCH(h);
+    launch_pdl(prefill_plan_kernel, dim3(1), dim3(1024), 0, st, rows, tile, L.attn_item_start, L.pf_tile_rows, L.pf_n_tiles);
+}
+
+namespace {
+
 template <typename T, int DH>
 void launch_prefill_t(const cdb* h, const AttnParams& p, int ln, void* o, cudaStream_t st) {
     const Lane& L = h->lane[ln];
     // pads first: rows the tiles do not cover keep a zero output
     cudaMemsetAsync(o, 0, (size_t)p.rows.n_rows * p.pool.H * DH * sizeof(T), st);
-    CDB_LAUNCH(h);
-    launch_pdl(prefill_plan_kernel, dim3(1), dim3(32), 0, st, p.rows, L.attn_item_start, L.pf_tile_rows, L.pf_n_tiles);
+    launch_prefill_plan(h, ln, p.rows, kPfTile, st);
     CDB_LAUNCH(h);
     dim3 grid(p.rows.n_rows, p.pool.H);                                // upper bound on tiles; surplus CTAs exit at once
     launch_pdl(attn_prefill_kernel<T, DH>, grid, dim3(128), 0, st, p, (const int32_t*)L.attn_item_start,
@@ -601,6 +645,7 @@ void launch_prefill_t(const cdb* h, const AttnParams& p, int ln, void* o, cudaSt
 // pages their own call has just written.  Uses the lane's split-scan buffer for its tile list.
 void launch_attention_prefill(const cdb* h, int ln, int layer, const RowsDev& rows, const void* q, void* o, cudaStream_t st) {
     if (rows.n_rows <= 0) return;
+    if (!(h->cfg.flags & CDB_FLAG_SIMT_PREFILL) && launch_attention_prefill_tc(h, ln, layer, rows, q, o, st)) return;
     AttnParams p;
     p.q = q; p.pool = h->pool; p.rows = rows; p.layer = layer; p.max_splits = h->max_splits;
     p.max_seqs = h->cfg.max_seqs;

@@ -165,6 +165,8 @@ void launch_rope_kv_write(const cdb* h, int ln, int layer, const float* qkv_part
 void launch_attention(const cdb* h, int ln, int layer, const RowsDev& rows, const void* q, void* o, cudaStream_t st);
 void launch_attention_plan(const cdb* h, int ln, const RowsDev& rows, cudaStream_t st);
 void launch_attention_prefill(const cdb* h, int ln, int layer, const RowsDev& rows, const void* q, void* o, cudaStream_t st);
+void launch_prefill_plan(const cdb* h, int ln, const RowsDev& rows, int tile, cudaStream_t st);
+bool launch_attention_prefill_tc(const cdb* h, int ln, int layer, const RowsDev& rows, const void* q, void* o, cudaStream_t st);
 void launch_swiglu(const cdb* h, int ln, int n_rows, cudaStream_t st);
 void launch_embed(const cdb* h, const int32_t* tokens, const RowsDev& rows, float* out, bool reset_gate, cudaStream_t st);
 void launch_gate(const cdb* h, const RowsDev& rows, const float* x, const float* x_prev, float* gate_val_out,

@@ -124,20 +124,27 @@ def test_lockstep_replay_of_adaptive_decode_bf16():
     assert explained <= max(2, tokens // 20) and near_gate <= max(2, decisions // 50)
 
 
-@pytest.mark.parametrize("H,Dh,dtype", [(2, 128, "bf16"), (3, 96, "bf16"), (2, 64, "bf16"), (4, 64, "fp32")])
-def test_prefill_matches_oracle(H, Dh, dtype):
+SHORT, LONG = [1, 33, 70, 16, 47], [130, 5, 300, 128, 257]
+
+
+@pytest.mark.parametrize("H,Dh,dtype,lens,simt", [
+    (2, 128, "bf16", SHORT, False), (3, 96, "bf16", SHORT, False), (2, 64, "bf16", SHORT, False), (4, 64, "fp32", SHORT, False),
+    (2, 128, "bf16", LONG, False), (3, 96, "bf16", LONG, False), (2, 64, "bf16", LONG, False),
+    (2, 128, "bf16", LONG, True), (4, 64, "fp32", LONG, False)])
+def test_prefill_matches_oracle(H, Dh, dtype, lens, simt):
     """Lock-step prompt processing (query-tiled causal attention over the pages the call itself writes),
-    several prompts of ragged length in one call with a pad row, against the oracle's prefill."""
+    several prompts of ragged length in one call with a pad row, against the oracle's prefill.  The long
+    set spans several query tiles and key tiles of the tensor-core kernel with ragged tails; `simt` runs
+    the plain-FMA kernel on the same bf16 input.  The pool starts as NaN: nothing may be read before written."""
     from paper_2608_09444_b200 import binding as B
     dims = synth.Dims(V=300, d=H * Dh, H=H, Dh=Dh, F=192, L_pre=1, L_core=2, L_coda=1, R=3, dtype=dtype)
     w = synth.make_weights(dims, 8, std=0.05, gain_jitter=0.1)
     wn = synth.weights_to_numpy(w)
-    lens = [1, 33, 70, 16, 47]
     prompts = [synth.make_prompts(1, n, dims.V, 20 + i)[0] for i, n in enumerate(lens)]
     table_np, n_pages = synth.make_page_table(np.asarray(lens), 16, seed=2, extra_pages=1)
     n = sum(lens) + 1
     cdb = B.Cdb(dims, {k: v.cuda() for k, v in w.items()}, max_rows=n, max_seqs=len(lens), max_position=table_np.shape[1] * 16,
-                gate_kind=B.GATE_NONE)
+                gate_kind=B.GATE_NONE, flags=B.FLAG_SIMT_PREFILL if simt else 0)
     tdt = torch.float32 if dtype == "fp32" else torch.bfloat16
     pool = torch.full(synth.kv_pool_shape(dims, n_pages), float("nan"), dtype=tdt, device="cuda")   # nothing is read before written
     cdb.kv_bind(pool)
