@@ -372,6 +372,7 @@ bool launch_attention_prefill_tc(const cdb* h, int ln, int layer, const RowsDev&
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
         attr_set[ki] = true;
     }
+    ProfScope prof(h, kProfAttention, st);
     CDB_LAUNCH(h);
     return launch_pdl(kern, dim3(grid), dim3(kPfThreads), smem, st, map_q, map_kv, p) == cudaSuccess;
 }
