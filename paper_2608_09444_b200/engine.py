@@ -117,16 +117,28 @@ class Engine:
             self.page_table_host[row] = -1
 
     # ------------------------------------------------------------------ generation
-    def generate(self, prompts, T, forced_depths=None, teacher_tokens=None):
+    def generate(self, prompts, T, forced_depths=None, teacher_tokens=None, arrivals=None):
         """prompts: list of int arrays; T: generated tokens per sequence (int or list).  forced_depths[s][j]
         replays the exit depth of adaptive pass j of sequence s (0 / None = decided by the gate);
-        teacher_tokens[s][j] replaces the token fed back after generated token j (lock-step replay)."""
+        teacher_tokens[s][j] replaces the token fed back after generated token j (lock-step replay).
+        arrivals[s] (seconds after the call starts, non-decreasing) makes request s visible to the scheduler
+        only from that wall-clock time on (online serving); stats["first_token_s"] / ["finish_s"] then hold
+        the times at which the host saw each request's first and last token."""
         dims, cdb = self.dims, self.cdb
         n = len(prompts)
         Ts = [T] * n if np.isscalar(T) else list(T)
         seqs = [_Seq(i, np.asarray(prompts[i], dtype=np.int32), Ts[i], [], [], [], []) for i in range(n)]
-        waiting = list(range(n))
+        waiting = list(range(n)) if arrivals is None else []
+        future = [] if arrivals is None else list(range(n))
         self.stats["start"] = time.perf_counter()
+        self.stats["first_token_s"], self.stats["finish_s"] = [None] * n, [None] * n
+        now = lambda: time.perf_counter() - self.stats["start"]
+
+        def poll_arrivals():
+            t = now()
+            while future and arrivals[future[0]] <= t:
+                waiting.append(future.pop(0))
+
         live_slot = {}                       # sid -> live slot id (index into gate state / page table)
         free_slots = list(range(self.max_live - 1, -1, -1))
         ready = []                           # [(sid, h row index in h_ready)] awaiting the recurrent batch (FIFO)
@@ -171,7 +183,10 @@ class Engine:
         def finish_or_continue(s, token):
             sq = seqs[s]
             sq.tokens.append(int(token))
+            if len(sq.tokens) == 1:
+                self.stats["first_token_s"][s] = now()
             if len(sq.tokens) >= sq.T:
+                self.stats["finish_s"][s] = now()
                 self._release_pages(live_slot[s])
                 free_slots.append(live_slot.pop(s))
                 return None
@@ -257,7 +272,7 @@ class Engine:
 
         def run_recurrent(allow_refill):
             nonlocal rec
-            if "decode_start" not in self.stats and not waiting:          # every prompt processed: decode phase begins
+            if "decode_start" not in self.stats and not waiting and not future:   # every prompt processed: decode phase begins
                 torch.cuda.synchronize(self.dev)
                 self.stats["decode_start"] = time.perf_counter()
             # survivors are already at the front of h_rec in stable order; append refills (FIFO)
@@ -299,7 +314,12 @@ class Engine:
             self.last_lists = (surv.copy(), ex.copy())
             return True
 
-        while waiting or live_slot:
+        while waiting or live_slot or future:
+            if future:
+                poll_arrivals()
+                if not waiting and not live_slot:
+                    time.sleep(min(1e-3, max(0.0, arrivals[future[0]] - now())))
+                    continue
             if self.mode == "refill":
                 runnable_other = bool(rec) or bool(ready) or (bool(waiting) and bool(free_slots))
                 if coda_q and (len(coda_q) >= self.min_coda_batch or not runnable_other):

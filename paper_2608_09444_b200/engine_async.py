@@ -74,7 +74,7 @@ class PipelinedEngine(Engine):
         torch.cuda.synchronize(self.dev)
 
     # ------------------------------------------------------------------ generation
-    def generate(self, prompts, T, forced_depths=None, teacher_tokens=None):
+    def generate(self, prompts, T, forced_depths=None, teacher_tokens=None, arrivals=None):
         """Same contract as Engine.generate (teacher tokens are not supported: sampled tokens stay on the
         device and feed the prelude directly).  Gate values are not read back."""
         if teacher_tokens is not None:
@@ -87,7 +87,8 @@ class PipelinedEngine(Engine):
         tokens = [[None] * Ts[i] for i in range(n)]
         depths = [[] for _ in range(n)]
         gen = [0] * n                                   # tokens sampled so far (values may still be in flight)
-        waiting, live_slot = list(range(n)), {}
+        waiting, live_slot = (list(range(n)) if arrivals is None else []), {}
+        future = [] if arrivals is None else list(range(n))
         free_slots = list(range(self.max_live - 1, -1, -1))
         ready, ready_free = [], list(range(self.cap - 1, -1, -1))     # (sid, slot in h_ready, event, iteration)
         coda_q, coda_free = [], list(range(self.cap - 1, -1, -1))     # (sid, depth, slot in h_coda)
@@ -102,6 +103,8 @@ class PipelinedEngine(Engine):
         i32 = lambda a: torch.tensor(np.asarray(a, dtype=np.int32), dtype=torch.int32, device=dev)
         self._capture_all()
         self.stats["start"] = time.perf_counter()
+        self.stats["first_token_s"], self.stats["finish_s"] = [None] * n, [None] * n
+        now = lambda: time.perf_counter() - self.stats["start"]
         x_done = [None, None]                           # h_exit2[parity] copied out (event on the side stream)
         gather_done = None                              # last refill gather on the main stream
         tok_calls = 0
@@ -118,6 +121,8 @@ class PipelinedEngine(Engine):
                 vals = buf.numpy()
                 for j, (s, idx) in enumerate(items):
                     tokens[s][idx] = int(vals[j])
+                    if idx == Ts[s] - 1:
+                        self.stats["finish_s"][s] = now()
             while pending_release and (block or pending_release[0][0].query()):
                 ev, s = pending_release.pop(0)
                 ev.synchronize()
@@ -167,6 +172,9 @@ class PipelinedEngine(Engine):
                 for j, s in enumerate(batch):
                     tokens[s][0] = int(vals[j])
                     gen[s] = 1
+                    self.stats["first_token_s"][s] = now()
+                    if Ts[s] == 1:
+                        self.stats["finish_s"][s] = now()
                     if gen[s] >= Ts[s]:
                         self._release_pages(live_slot[s])
                         free_slots.append(live_slot.pop(s))
@@ -222,9 +230,13 @@ class PipelinedEngine(Engine):
         rec, prev, it = [], None, 0
         while True:
             drain_tokens(False)
+            if future:
+                t_now = now()
+                while future and arrivals[future[0]] <= t_now:
+                    waiting.append(future.pop(0))
             if waiting and free_slots:
                 admit()
-            if "decode_start" not in self.stats and not waiting:
+            if "decode_start" not in self.stats and not waiting and not future:
                 torch.cuda.synchronize(dev)
                 self.stats["decode_start"] = time.perf_counter()
             # ---- refills whose prelude was enqueued in an earlier iteration join this step
@@ -291,7 +303,10 @@ class PipelinedEngine(Engine):
                 rec = [[rec[int(i)][0], rec[int(i)][1] + 1] for i in surv]
             it += 1
             if not rec and prev is None and not ready and not coda_q and not waiting:
-                if all(gen[s] >= Ts[s] for s in range(n)):
+                if future and not pending_tokens and not pending_release:
+                    time.sleep(min(1e-3, max(0.0, arrivals[future[0]] - now())))
+                    continue
+                if not future and all(gen[s] >= Ts[s] for s in range(n)):
                     break
                 if not pending_tokens and not pending_release:
                     raise RuntimeError("pipelined scheduler stalled")

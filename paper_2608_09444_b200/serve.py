@@ -1,0 +1,109 @@
+"""Online serving on synthetic traffic (the config-5 analogue of the paper's section 6 serving experiment).
+
+Requests arrive as a Poisson process; prompt and output lengths are log-normal (median 512 / 256 tokens,
+sigma 0.8, clipped to [4, 4096] / [4, 2048]), standing in for the ShareGPT / Alpaca replays the paper
+uses.  Each request's normalised latency is (time its last token reached the host - arrival time) /
+output length; the report gives its mean, p50 and p99 per arrival rate, next to throughput, for standard
+continuous batching (every token loops r_max times) and continuous depth batching with refill.
+
+    python -m paper_2608_09444_b200.serve --model ouro --rates 4,8,16 --requests 300
+
+The engines run against the wall clock, so a run lasts requests / rate seconds plus the drain.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import synth
+from .engine import Engine
+from .engine_async import PipelinedEngine
+from .offline import calibrate_gate_bias
+
+
+def make_requests(n, rate, seed, vocab, prompt_median=512, prompt_cap=4096, out_median=256, out_cap=2048):
+    """Seeded request trace: arrival times (s), prompts (token ids), output lengths."""
+    arrivals = synth.poisson_arrivals(n, rate, seed)
+    p_len = synth.lognormal_lengths(n, seed + 1, prompt_median, prompt_cap)
+    t_len = synth.lognormal_lengths(n, seed + 2, out_median, out_cap)
+    rng = np.random.default_rng(seed + 3)
+    prompts = [rng.integers(0, vocab, size=int(m), dtype=np.int32) for m in p_len]
+    return arrivals, prompts, [int(t) for t in t_len]
+
+
+def summarize(arrivals, out_lens, stats):
+    fin = np.asarray(stats["finish_s"], dtype=np.float64)
+    first = np.asarray(stats["first_token_s"], dtype=np.float64)
+    lat = (fin - arrivals) / np.asarray(out_lens, dtype=np.float64)
+    span = float(fin.max() - arrivals[0])
+    return {"normalized_latency_s_per_token": {"mean": float(lat.mean()), "p50": float(np.percentile(lat, 50)),
+                                               "p99": float(np.percentile(lat, 99))},
+            "time_to_first_token_s": {"mean": float((first - arrivals).mean()), "p99": float(np.percentile(first - arrivals, 99))},
+            "generated_tokens_per_s": float(np.sum(out_lens) / span), "span_s": span,
+            "recurrent_steps": stats["recurrent_steps"], "row_steps": stats["row_steps"],
+            "prefill_calls": stats["prefill_calls"], "coda_calls": stats["coda_calls"]}
+
+
+def run(dims, weights, arrivals, prompts, out_lens, *, mode, pipelined, gate_kind, q_or_eps=0.5, forced_depths=None,
+        max_batch=256, max_live=320, pool_tokens=400000, min_coda_batch=1, max_prefill_rows=4096):
+    max_len = max(len(p) + t for p, t in zip(prompts, out_lens))
+    pages = (pool_tokens + dims.page_size - 1) // dims.page_size
+    eng = (PipelinedEngine if pipelined else Engine)(
+        dims, weights, max_batch=max_batch, max_live=max_live, max_len=max_len, n_pages=pages, gate_kind=gate_kind,
+        q_or_eps=q_or_eps, lookahead=True, mode=mode, min_coda_batch=min_coda_batch,
+        max_prefill_rows=max(max_prefill_rows, max(len(p) for p in prompts)), record_ticks=False)
+    res = eng.generate(prompts, out_lens, forced_depths=forced_depths, arrivals=arrivals)
+    out = summarize(arrivals, out_lens, eng.stats)
+    out["mode"] = mode + ("_pipelined" if pipelined else "")
+    out["status"] = eng.cdb.poll_status()
+    d = np.concatenate([x for x in res["depths"] if len(x)]) if any(len(x) for x in res["depths"]) else np.zeros(0)
+    out["mean_depth"] = float(d.mean()) if d.size else float(dims.R)
+    eng.cdb.destroy()
+    del eng
+    torch.cuda.empty_cache()
+    return out, res
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--model", default="ouro", choices=["ouro", "huginn"])
+    ap.add_argument("--rates", default="4,8,16")
+    ap.add_argument("--requests", type=int, default=300)
+    ap.add_argument("--max-batch", type=int, default=256)
+    ap.add_argument("--max-live", type=int, default=320)
+    ap.add_argument("--pool-tokens", type=int, default=400000)
+    ap.add_argument("--modes", default="cb,refill_pipelined")
+    args = ap.parse_args()
+    torch.cuda.set_device(0)
+    dims, seed = (synth.OURO_1P4B, 4) if args.model == "ouro" else (synth.HUGINN_3P5B, 5)
+    w = synth.make_weights(dims, seed, device="cuda:0", gate_std=2.0 / np.sqrt(dims.d))
+    report = {"model": args.model, "requests": args.requests, "runs": []}
+    if args.model == "ouro":
+        gate_kind = B.GATE_SIGMOID_CDF
+        cal = list(synth.make_prompts(16, 256, dims.V, seed))
+        report["b_gate"] = calibrate_gate_bias(dims, w, cal, 24, 2.5)
+    else:
+        gate_kind = B.GATE_NONE
+    for ri, rate in enumerate(float(x) for x in args.rates.split(",")):
+        arrivals, prompts, out_lens = make_requests(args.requests, rate, seed + 10 * ri, dims.V)
+        forced = None
+        if args.model == "huginn":       # replayed exit depths: truncated geometric, mean 12
+            forced = [list(synth.forced_exit_depths((1, max(t - 1, 1)), seed + 100 + i, 12.0, dims.R)[0]) for i, t in enumerate(out_lens)]
+        for mode in args.modes.split(","):
+            pipelined = mode.endswith("_pipelined")
+            m = mode.replace("_pipelined", "")
+            out, _ = run(dims, w, arrivals, prompts, out_lens, mode=m, pipelined=pipelined, gate_kind=gate_kind,
+                         forced_depths=None if m == "cb" else forced, max_batch=args.max_batch, max_live=args.max_live,
+                         pool_tokens=args.pool_tokens, min_coda_batch=1 if args.model == "ouro" else 32)
+            out["rate_req_per_s"] = rate
+            report["runs"].append(out)
+            print(json.dumps(out), flush=True)
+    print(json.dumps(report))
+
+
+if __name__ == "__main__":
+    main()

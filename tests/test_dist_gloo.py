@@ -4,6 +4,7 @@ import os
 import socket
 import sys
 
+import numpy as np
 import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
@@ -59,3 +60,22 @@ def test_latency_model_fit_recovers_its_coefficients():
     f = fit(pts)
     assert abs(f["delta_ms"] - d) < 1e-9 and abs(f["gamma_ms_per_row"] - g) < 1e-11 and abs(f["alpha_ms_per_token"] - a) < 1e-13
     assert f["r2"] > 1 - 1e-12 and f["max_rel_residual"] < 1e-9
+
+
+def test_serving_trace_and_latency_summary():
+    """The request trace is seeded and within its clipping bounds; the summary computes per-request
+    (finish - arrival) / output length and its percentiles."""
+    from paper_2608_09444_b200.serve import make_requests, summarize
+    a1, p1, t1 = make_requests(50, 8.0, 3, 1000)
+    a2, p2, t2 = make_requests(50, 8.0, 3, 1000)
+    assert np.array_equal(a1, a2) and t1 == t2 and all(np.array_equal(x, y) for x, y in zip(p1, p2))
+    assert np.all(np.diff(a1) > 0) and 4 <= min(len(p) for p in p1) and max(len(p) for p in p1) <= 4096
+    assert 4 <= min(t1) and max(t1) <= 2048 and max(int(p.max()) for p in p1) < 1000
+    arr = np.array([0.0, 1.0, 2.0])
+    stats = {"finish_s": [2.0, 5.0, 2.5], "first_token_s": [0.5, 1.5, 2.25], "recurrent_steps": 7, "row_steps": 9,
+             "prefill_calls": 3, "coda_calls": 4}
+    s = summarize(arr, [4, 8, 1], stats)
+    lat = np.array([0.5, 0.5, 0.5])
+    assert abs(s["normalized_latency_s_per_token"]["mean"] - lat.mean()) < 1e-12
+    assert abs(s["normalized_latency_s_per_token"]["p99"] - 0.5) < 1e-12
+    assert abs(s["generated_tokens_per_s"] - 13 / 5.0) < 1e-12 and abs(s["time_to_first_token_s"]["mean"] - (0.5 + 0.5 + 0.25) / 3) < 1e-12

@@ -166,3 +166,28 @@ def test_c1_pipelined_engine_gives_the_same_tokens(oracle_runs, max_batch, max_l
         assert np.array_equal(res["depths"][s], ref[s]["depths"]), s
     assert eng.stats["row_steps"] == int(sum(r["depths"].sum() for r in ref))
     assert not [p for row in eng.page_table_host for p in row if p >= 0]
+
+
+@pytest.mark.parametrize("pipelined", [False, True])
+def test_c1_requests_arriving_over_time_give_the_same_tokens(oracle_runs, pipelined):
+    """Online serving: requests become visible at their (seeded Poisson) arrival times and carry their own
+    output lengths; what a request generates does not depend on when it arrives or what it is batched with,
+    so tokens and exit depths equal the oracle's prefix of the same length, and every request gets its
+    first-token and finish time stamps in order."""
+    from paper_2608_09444_b200 import binding as B
+    from paper_2608_09444_b200.engine import Engine
+    from paper_2608_09444_b200.engine_async import PipelinedEngine
+    dims, w, prompts = c1_inputs()
+    wd = {k: v.cuda() for k, v in w.items()}
+    arrivals = synth.poisson_arrivals(8, 200.0, 11)
+    lens = [16, 3, 9, 1, 16, 12, 5, 7]
+    eng = (PipelinedEngine if pipelined else Engine)(dims, wd, max_batch=4, max_live=5, max_len=48, n_pages=15,
+                                                      gate_kind=B.GATE_SIGMOID_CDF, q_or_eps=0.5, max_prefill_rows=256)
+    res = eng.generate(list(prompts), lens, arrivals=arrivals)
+    assert eng.cdb.poll_status() == 0
+    ref = oracle_runs["adaptive"]
+    for s in range(8):
+        assert np.array_equal(res["tokens"][s], ref[s]["tokens"][:lens[s]]), s
+        assert np.array_equal(res["depths"][s], ref[s]["depths"][:lens[s] - 1]), s
+        assert arrivals[s] <= eng.stats["first_token_s"][s] <= eng.stats["finish_s"][s]
+    assert not [p for row in eng.page_table_host for p in row if p >= 0]
