@@ -36,7 +36,7 @@ class Engine:
                  r_min: int = 1, lookahead: bool = True, mode: str = "refill", min_coda_batch: int = 1,
                  max_prefill_rows: int | None = None, flags: int = 0, record_states: bool = False,
                  record_logits: bool = False, record_ticks: bool = True, use_graphs: bool = True,
-                 device: str = "cuda:0"):
+                 time_device: bool = False, admit_min: int = 1, admit_wait_s: float = 0.0, device: str = "cuda:0"):
         self.dims, self.mode, self.lookahead = dims, mode, lookahead
         self.max_batch, self.max_live, self.min_coda_batch = max_batch, max_live, min_coda_batch
         self.dev = torch.device(device)
@@ -80,6 +80,40 @@ class Engine:
         self.desc_host = torch.zeros((5, max_rows), dtype=torch.int32).pin_memory()
         self.desc_dev = torch.zeros((5, max_rows), **i32)
         self.graphs = {}
+        # optional accounting of device time: CUDA-event pairs around every GPU phase the engine enqueues
+        self.time_device = time_device
+        # online serving: hold arrived requests until admit_min of them wait or the oldest has waited admit_wait_s,
+        # so that prompts are processed several at a time (one prompt alone re-reads every weight per loop)
+        self.admit_min, self.admit_wait_s = admit_min, admit_wait_s
+        self._dev_events = []
+
+    class _Phase:
+        def __init__(self, eng, name):
+            self.eng, self.name = eng, name
+
+        def __enter__(self):
+            if self.eng.time_device:
+                self.a = torch.cuda.Event(enable_timing=True)
+                self.a.record()
+
+        def __exit__(self, *exc):
+            if self.eng.time_device:
+                b = torch.cuda.Event(enable_timing=True)
+                b.record()
+                self.eng._dev_events.append((self.name, self.a, b))
+            return False
+
+    def _phase(self, name):
+        """Brackets the GPU work enqueued inside with an event pair (no-op unless time_device)."""
+        return Engine._Phase(self, name)
+
+    def _collect_device_time(self):
+        """stats["device_ms"][phase] = summed event time of that phase's brackets (after a synchronize)."""
+        out = {}
+        for name, a, b in self._dev_events:
+            out[name] = out.get(name, 0.0) + a.elapsed_time(b)
+        self._dev_events = []
+        self.stats["device_ms"] = out
 
     # ------------------------------------------------------------------ descriptor helpers
     def _rows(self, seq_ids, positions, depths=None, slots=None, forced=None):
@@ -172,12 +206,13 @@ class Engine:
             rows = self._rows(sl, pos)
             tok_t = torch.tensor(toks, dtype=torch.int32, device=self.dev)
             out = self.h_tmp[:len(sids)]
-            if dims.L_pre > 0:
-                cdb.boundary_prelude(tok_t, rows, out)
-            else:
-                cdb.boundary_embed(tok_t, rows, out)
             slots = [ready_free.pop() for _ in sids]
-            self.h_ready.index_copy_(0, torch.tensor(slots, dtype=torch.int64, device=self.dev), out)
+            with self._phase("prelude"):
+                if dims.L_pre > 0:
+                    cdb.boundary_prelude(tok_t, rows, out)
+                else:
+                    cdb.boundary_embed(tok_t, rows, out)
+                self.h_ready.index_copy_(0, torch.tensor(slots, dtype=torch.int64, device=self.dev), out)
             ready.extend(zip(sids, slots))
 
         def finish_or_continue(s, token):
@@ -194,7 +229,16 @@ class Engine:
             sq.next_input = int(teacher_tokens[s][j]) if teacher_tokens is not None else int(token)
             return s
 
+        def admission_due():
+            if not waiting or not free_slots:
+                return False
+            if arrivals is None or len(waiting) >= self.admit_min or not live_slot:
+                return True
+            return now() - arrivals[waiting[0]] >= self.admit_wait_s
+
         def run_prefill():
+            if not admission_due():
+                return False
             admitted = []
             rows_total = 0
             while waiting and free_slots:
@@ -223,7 +267,8 @@ class Engine:
             emit = torch.tensor(ends, dtype=torch.int32, device=self.dev)
             tok_t = torch.tensor(toks, dtype=torch.int32, device=self.dev)
             lg = self.logits[:len(admitted)] if self.record_logits else None
-            cdb.prefill(tok_t, rows, emit, self.tok_out[:len(admitted)], lg)
+            with self._phase("prefill"):
+                cdb.prefill(tok_t, rows, emit, self.tok_out[:len(admitted)], lg)
             out = self.tok_out[:len(admitted)].cpu().numpy()
             self.stats["prefill_calls"] += 1
             cont = []
@@ -251,7 +296,8 @@ class Engine:
             if self.kv_layout == B.KV_DEPTH_INDEXED:
                 cdb.kv_copy_on_exit(rows, torch.tensor([it[1] for it in items], dtype=torch.int32, device=self.dev))
             lg = self.logits[:k] if self.record_logits else None
-            cdb.boundary_coda_lmhead(rows, hin, self.tok_out[:k], lg)
+            with self._phase("coda"):
+                cdb.boundary_coda_lmhead(rows, hin, self.tok_out[:k], lg)
             out = self.tok_out[:k].cpu().numpy()
             self.stats["coda_calls"] += 1
             cont = []
@@ -292,7 +338,8 @@ class Engine:
             sl = [live_slot[s] for s, _ in rec]
             pos = [position_of(seqs[s]) for s, _ in rec]
             dep = [r for _, r in rec]
-            _run_step(self, k, sl, dep, pos, [self._slot(r) for r in dep], [forced_for(seqs[s]) for s, _ in rec])
+            with self._phase("recurrent"):
+                _run_step(self, k, sl, dep, pos, [self._slot(r) for r in dep], [forced_for(seqs[s]) for s, _ in rec])
             cnt = self.counts.cpu().numpy()
             ns, ne = int(cnt[0]), int(cnt[1])
             surv = self.surv_idx[:ns].cpu().numpy()
@@ -346,6 +393,8 @@ class Engine:
                         pass
         torch.cuda.synchronize(self.dev)
         self.stats["end"] = time.perf_counter()
+        if self.time_device:
+            self._collect_device_time()
         return {"tokens": [np.asarray(s.tokens, dtype=np.int32) for s in seqs],
                 "depths": [np.asarray(s.depths, dtype=np.int32) for s in seqs],
                 "gates": [s.gates for s in seqs]}

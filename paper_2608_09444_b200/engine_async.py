@@ -234,7 +234,8 @@ class PipelinedEngine(Engine):
                 t_now = now()
                 while future and arrivals[future[0]] <= t_now:
                     waiting.append(future.pop(0))
-            if waiting and free_slots:
+            if waiting and free_slots and (arrivals is None or len(waiting) >= self.admit_min or not live_slot
+                                           or now() - arrivals[waiting[0]] >= self.admit_wait_s):
                 admit()
             if "decode_start" not in self.stats and not waiting and not future:
                 torch.cuda.synchronize(dev)
@@ -267,14 +268,15 @@ class PipelinedEngine(Engine):
                 dh[4, :k] = torch.as_tensor(np.asarray([forced_for(s) for s, _ in rec], dtype=np.int32))
                 dh[0, k:nb] = -1
                 dh[1:, k:nb] = 0
-                self.desc_dev.copy_(dh, non_blocking=True)
-                g, rows = self.pgraphs[(nb, parity)]
-                cdb.compact(rows, self.surv_idx, self.exit_idx, self.counts)
-                lists_ready = torch.cuda.Event()
-                lists_ready.record(main)
-                if x_done[parity] is not None:
-                    main.wait_event(x_done[parity])         # the exits of two steps ago have left h_exit2[parity]
-                g.replay()
+                with self._phase("recurrent"):
+                    self.desc_dev.copy_(dh, non_blocking=True)
+                    g, rows = self.pgraphs[(nb, parity)]
+                    cdb.compact(rows, self.surv_idx, self.exit_idx, self.counts)
+                    lists_ready = torch.cuda.Event()
+                    lists_ready.record(main)
+                    if x_done[parity] is not None:
+                        main.wait_event(x_done[parity])     # the exits of two steps ago have left h_exit2[parity]
+                    g.replay()
                 G = torch.cuda.Event()
                 G.record(main)
                 with torch.cuda.stream(side):
@@ -314,5 +316,7 @@ class PipelinedEngine(Engine):
         torch.cuda.synchronize(dev)
         drain_tokens(True)
         self.stats["end"] = time.perf_counter()
+        if self.time_device:
+            self._collect_device_time()
         return {"tokens": [np.asarray(t, dtype=np.int32) for t in tokens],
                 "depths": [np.asarray(d, dtype=np.int32) for d in depths], "gates": None}

@@ -27,21 +27,22 @@ def flop_bound(dims, mean_depth):
 
 
 def run(dims, weights, prompts, T, *, mode, gate_kind, q_or_eps=0.5, forced_depths=None, max_batch=None, max_live=None,
-        min_coda_batch=1, max_prefill_rows=4096, pipelined=False):
+        min_coda_batch=1, max_prefill_rows=4096, pipelined=False, use_graphs=True, time_device=False):
     n, P = len(prompts), max(len(p) for p in prompts)
     live = min(n, max_live or n)
     pages = live * ((P + T + dims.page_size - 1) // dims.page_size)
     eng = (PipelinedEngine if pipelined else Engine)(dims, weights, max_batch=min(max_batch or n, live), max_live=live, max_len=P + T, n_pages=pages, gate_kind=gate_kind,
                  q_or_eps=q_or_eps, lookahead=True, mode=mode, min_coda_batch=min_coda_batch,
-                 max_prefill_rows=max_prefill_rows, record_ticks=False)
+                 max_prefill_rows=max_prefill_rows, record_ticks=False, use_graphs=use_graphs, time_device=time_device)
     res = eng.generate(prompts, T, forced_depths=forced_depths)
     st = eng.stats
     depths = np.concatenate(res["depths"])
     decode_s = st["end"] - st["decode_start"]
-    out = {"mode": mode + ("_pipelined" if pipelined else ""), "max_batch": eng.max_batch, "max_live": live, "total_s": st["end"] - st["start"],
+    out = {"mode": mode + ("_pipelined" if pipelined else "") + ("" if use_graphs else "_nographs"), "max_batch": eng.max_batch, "max_live": live, "total_s": st["end"] - st["start"],
            "generated_tokens_per_s_end_to_end": sum(len(t) for t in res["tokens"]) / (st["end"] - st["start"]),
            "decode_s": decode_s, "prefill_s": st["decode_start"] - st["start"],
            "decode_tokens_per_s": len(depths) / decode_s, "token_loop_steps_per_s": st["row_steps"] / decode_s,
+           "device_ms": st.get("device_ms"), "wall_ms_per_recurrent_step": 1e3 * decode_s / max(st["recurrent_steps"], 1),
            "recurrent_steps": st["recurrent_steps"], "row_steps": st["row_steps"], "coda_calls": st["coda_calls"],
            "mean_depth": float(depths.mean()), "depth_histogram": np.bincount(depths, minlength=dims.R + 1)[1:].tolist(),
            "status": eng.cdb.poll_status()}
@@ -78,7 +79,8 @@ def main():
     ap.add_argument("--max-batch", type=int, default=0)
     ap.add_argument("--min-coda-batch", type=int, default=0)
     ap.add_argument("--max-live", type=int, default=0, help="sequences resident at once (0 = all); fewer than --seqs queues the rest")
-    ap.add_argument("--modes", default="cb,refill,no_refill", help="cb, refill, no_refill, refill_pipelined")
+    ap.add_argument("--modes", default="cb,refill,no_refill", help="cb, refill, no_refill, refill_pipelined, refill_nographs")
+    ap.add_argument("--time-device", action="store_true", help="bracket every GPU phase with CUDA events and report device_ms")
     args = ap.parse_args()
     torch.cuda.set_device(0)
     if args.model == "ouro":
@@ -103,8 +105,9 @@ def main():
         min_coda = args.min_coda_batch or 32
     for mode in args.modes.split(","):
         pipelined = mode.endswith("_pipelined")
-        mode = mode.replace("_pipelined", "")
-        out, _ = run(dims, w, prompts, args.tokens, mode=mode, pipelined=pipelined, gate_kind=gate_kind, forced_depths=None if mode == "cb" else forced,
+        nographs = mode.endswith("_nographs")
+        mode = mode.replace("_pipelined", "").replace("_nographs", "")
+        out, _ = run(dims, w, prompts, args.tokens, mode=mode, pipelined=pipelined, use_graphs=not nographs, time_device=args.time_device, gate_kind=gate_kind, forced_depths=None if mode == "cb" else forced,
                      max_batch=args.max_batch or None, max_live=args.max_live or None, min_coda_batch=min_coda)
         report["runs"].append(out)
         print(json.dumps(out), flush=True)

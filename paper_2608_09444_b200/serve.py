@@ -49,13 +49,15 @@ def summarize(arrivals, out_lens, stats):
 
 
 def run(dims, weights, arrivals, prompts, out_lens, *, mode, pipelined, gate_kind, q_or_eps=0.5, forced_depths=None,
-        max_batch=256, max_live=320, pool_tokens=400000, min_coda_batch=1, max_prefill_rows=4096):
+        max_batch=256, max_live=320, pool_tokens=400000, min_coda_batch=1, max_prefill_rows=4096,
+        admit_min=1, admit_wait_s=0.0):
     max_len = max(len(p) + t for p, t in zip(prompts, out_lens))
     pages = (pool_tokens + dims.page_size - 1) // dims.page_size
     eng = (PipelinedEngine if pipelined else Engine)(
         dims, weights, max_batch=max_batch, max_live=max_live, max_len=max_len, n_pages=pages, gate_kind=gate_kind,
         q_or_eps=q_or_eps, lookahead=True, mode=mode, min_coda_batch=min_coda_batch,
-        max_prefill_rows=max(max_prefill_rows, max(len(p) for p in prompts)), record_ticks=False)
+        max_prefill_rows=max(max_prefill_rows, max(len(p) for p in prompts)), record_ticks=False,
+        admit_min=admit_min, admit_wait_s=admit_wait_s)
     res = eng.generate(prompts, out_lens, forced_depths=forced_depths, arrivals=arrivals)
     out = summarize(arrivals, out_lens, eng.stats)
     out["mode"] = mode + ("_pipelined" if pipelined else "")
@@ -77,6 +79,8 @@ def main():
     ap.add_argument("--max-live", type=int, default=320)
     ap.add_argument("--pool-tokens", type=int, default=400000)
     ap.add_argument("--modes", default="cb,refill_pipelined")
+    ap.add_argument("--admit-min", type=int, default=1, help="hold arrived requests until this many wait ...")
+    ap.add_argument("--admit-wait-ms", type=float, default=0.0, help="... or the oldest has waited this long")
     args = ap.parse_args()
     torch.cuda.set_device(0)
     dims, seed = (synth.OURO_1P4B, 4) if args.model == "ouro" else (synth.HUGINN_3P5B, 5)
@@ -98,7 +102,8 @@ def main():
             m = mode.replace("_pipelined", "")
             out, _ = run(dims, w, arrivals, prompts, out_lens, mode=m, pipelined=pipelined, gate_kind=gate_kind,
                          forced_depths=None if m == "cb" else forced, max_batch=args.max_batch, max_live=args.max_live,
-                         pool_tokens=args.pool_tokens, min_coda_batch=1 if args.model == "ouro" else 32)
+                         pool_tokens=args.pool_tokens, min_coda_batch=1 if args.model == "ouro" else 32,
+                         admit_min=args.admit_min, admit_wait_s=args.admit_wait_ms * 1e-3)
             out["rate_req_per_s"] = rate
             report["runs"].append(out)
             print(json.dumps(out), flush=True)
