@@ -215,7 +215,9 @@ int cdb_paged_attention_static(const void* q, void* o, const void* pool, int32_t
                                int32_t H, int32_t Dh, int32_t dtype, void* stream);
 
 /* Synchronises the stream-less status word back to the host: 0 = clean, otherwise the first
- * out-of-range page id / position / sequence id a kernel met (the access was skipped). */
+ * out-of-range page id (1) / position (2) / sequence id (3) a kernel met since the last poll (the
+ * access was skipped), or 4 when a bounded wait inside a tensor-core kernel ran out.  A non-zero
+ * word is cleared by the call, so the next poll reports only what happened after this one. */
 int cdb_poll_status(cdb_t* h, int32_t* status_host);
 
 /* Instrumentation (not an operation of the paper): how many kernels the handle has launched, and

@@ -548,7 +548,8 @@ int cdb_linear(cdb_t* h, const void* x, const void* W, float* y, int32_t n, int3
 
 int cdb_poll_status(cdb_t* h, int32_t* status_host) {
     if (!h || !status_host) return CDB_ERR_ARG;
-    const cudaError_t e = cudaMemcpy(status_host, h->status, sizeof(int32_t), cudaMemcpyDeviceToHost);
+    cudaError_t e = cudaMemcpy(status_host, h->status, sizeof(int32_t), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && *status_host != 0) e = cudaMemset(h->status, 0, sizeof(int32_t));     // read and re-arm
     return e == cudaSuccess ? CDB_OK : fail_cuda(h, e, "cdb_poll_status");
 }
 

@@ -1,0 +1,151 @@
+"""Edge cases and invariants of the CUDA path through the C ABI: empty and all-pad batches, the largest
+position, reported (not faulting) range errors, capacity errors from the host checks, and batch
+invariance: a row's loop-step result is the same bit for bit alone or inside any batch, which is what
+lets continuous depth batching regroup rows freely without changing predictions (section 3)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import cdb_oracle as O
+from paper_2608_09444_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def dev(x, dtype=None):
+    t = torch.as_tensor(np.ascontiguousarray(x)).cuda()
+    return t if dtype is None else t.to(dtype)
+
+
+def i32(a):
+    return dev(np.asarray(a, dtype=np.int32))
+
+
+DIMS = synth.Dims(V=64, d=256, H=2, Dh=128, F=320, L_pre=0, L_core=2, L_coda=0, R=4, dtype="bf16")
+
+
+def setup(ctxs, max_rows, seed=3, dims=DIMS, extra_pages=1, **kw):
+    from paper_2608_09444_b200 import binding as B
+    w = synth.make_weights(dims, seed, std=0.05, gain_jitter=0.1, gate_std=0.1, b_gate=-0.2)
+    wd = {k: v.cuda() for k, v in w.items()}
+    table_np, n_pages = synth.make_page_table(np.asarray(ctxs), 16, seed=seed, permute=True, extra_pages=extra_pages)
+    cdb = B.Cdb(dims, wd, max_rows=max_rows, max_seqs=len(ctxs), max_position=table_np.shape[1] * 16,
+                gate_kind=B.GATE_SIGMOID_CDF, q_or_eps=0.4, **kw)
+    rng = np.random.default_rng(seed)
+    pool_np = synth.to_bf16_grid(rng.standard_normal(synth.kv_pool_shape(dims, n_pages)).astype(np.float32))
+    pool = dev(pool_np, torch.bfloat16)
+    cdb.kv_bind(pool)
+    return B, cdb, w, table_np, pool, pool_np
+
+
+def test_empty_and_all_pad_batches_change_nothing():
+    B, cdb, _, table_np, pool, pool_np = setup([40, 17], max_rows=4)
+    table = dev(table_np)
+    h = torch.randn((4, DIMS.d), device="cuda")
+    h0 = h.clone()
+    rows0 = B.Rows(i32([]), i32([]), table, loop_depth=i32([]), kv_slot=i32([]), n_rows=0)
+    cdb.loop_step(rows0, h[:0])
+    pads = B.Rows(i32([-1] * 4), i32([0] * 4), table, loop_depth=i32([1] * 4), kv_slot=i32([0] * 4))
+    gate, fire = torch.full((4,), 7.0, device="cuda"), torch.zeros(4, dtype=torch.uint8, device="cuda")
+    cdb.loop_step(pads, h, gate, fire)
+    surv, ex, counts = torch.zeros(4, dtype=torch.int32, device="cuda"), torch.zeros(4, dtype=torch.int32, device="cuda"), torch.full((2,), -1, dtype=torch.int32, device="cuda")
+    cdb.compact(pads, surv, ex, counts)
+    torch.cuda.synchronize()
+    assert cdb.poll_status() == 0
+    assert torch.equal(h, h0) and int(fire.sum()) == 0
+    assert counts.cpu().tolist() == [0, 0]
+    assert np.array_equal(pool.float().cpu().numpy(), pool_np)
+
+
+def test_last_position_of_the_configured_range():
+    """A row at position max_position - 1 (the last token of its last page) against the oracle."""
+    ctx = 64
+    B, cdb, w, table_np, pool, pool_np = setup([ctx], max_rows=1, extra_pages=0)
+    assert table_np.shape[1] * 16 == ctx
+    rows = B.Rows(i32([0]), i32([ctx - 1]), dev(table_np), loop_depth=i32([2]), kv_slot=i32([0]))
+    scratch = torch.zeros((1, DIMS.d), device="cuda")
+    cdb.boundary_embed(i32([0]), rows, scratch)
+    h_np = np.random.default_rng(5).standard_normal((1, DIMS.d)).astype(np.float32)
+    h = dev(h_np)
+    cdb.loop_step(rows, h)
+    torch.cuda.synchronize()
+    assert cdb.poll_status() == 0
+    orc = O.Oracle(DIMS, synth.weights_to_numpy(w), gate_kind=O.GATE_SIGMOID_CDF, q_or_eps=0.4)
+    Ks, Vs = zip(*[O.gather_pages(pool_np[l], table_np[0], ctx) for l in range(DIMS.L_core)])
+    h_ref = orc.loop_step_row(h_np[0], ctx - 1, 2, list(Ks), list(Vs))[0]
+    err = np.max(np.abs(h.cpu().numpy()[0] - h_ref)) / np.max(np.abs(h_ref))
+    assert err <= 2e-2, err
+
+
+def test_range_errors_are_reported_not_faulted():
+    """A page id outside the pool, a sequence id outside [0, max_seqs) and a position outside the range
+    make the kernels skip the access and latch a status word the host reads; capacity violations are
+    refused by the host checks before anything is launched."""
+    B, cdb, _, table_np, pool, pool_np = setup([40, 17], max_rows=2)
+    bad = table_np.copy()
+    bad[0, 1] = 10 ** 6                                    # logical page 1 of sequence 0
+    h = torch.randn((2, DIMS.d), device="cuda")
+    rows = B.Rows(i32([0, 1]), i32([39, 16]), dev(bad), loop_depth=i32([1, 1]), kv_slot=i32([0, 0]))
+    cdb.loop_step(rows, h)
+    torch.cuda.synchronize()
+    assert cdb.poll_status() == 1                          # page
+    assert cdb.poll_status() == 0                          # reading clears it
+    rows = B.Rows(i32([0, 5]), i32([39, 16]), dev(table_np), loop_depth=i32([1, 1]), kv_slot=i32([0, 0]))
+    cdb.loop_step(rows, h)
+    torch.cuda.synchronize()
+    assert cdb.poll_status() == 3                          # sequence
+    rows = B.Rows(i32([0, 1]), i32([39, 4096]), dev(table_np), loop_depth=i32([1, 1]), kv_slot=i32([0, 0]))
+    cdb.loop_step(rows, h)
+    torch.cuda.synchronize()
+    assert cdb.poll_status() == 2                          # position
+    assert bool(torch.isfinite(h[0]).all())                # the good row of the batch was still computed
+    big = B.Rows(i32([0, 1, -1]), i32([39, 16, 0]), dev(table_np), loop_depth=i32([1, 1, 1]), kv_slot=i32([0, 0, 0]))
+    with pytest.raises(B.CdbError) as e:
+        cdb.loop_step(big, torch.zeros((3, DIMS.d), device="cuda"))
+    assert e.value.code == -3                              # CDB_ERR_CAPACITY
+    assert "max_rows" in str(e.value) or "rows" in str(e.value)
+
+
+@pytest.mark.parametrize("flags,extra", [(0, 0), (4, 0), (0, 70), (0, 200)])
+def test_a_rows_result_does_not_depend_on_its_batch(flags, extra):
+    """Run nine rows together, then three of them alone, as a pair in another order and among pads: hidden
+    states, gate values, exit signals and the K/V written must be identical bit for bit (shape-only split-K
+    with fixed-order sums, attention splits that depend only on the row's own context).  flags=4 repeats the
+    check on the unfused layer flow; `extra` more rows make the full batch wide enough for the projection
+    kernel's 128- and 256-row tiles."""
+    ctxs = [1, 16, 17, 40, 255, 256, 257, 300, 33] + [int(c) for c in np.random.default_rng(2).integers(1, 90, extra)]
+    n = len(ctxs)
+    B, cdb, _, table_np, pool, pool_np = setup(ctxs, max_rows=n, flags=flags)
+    table = dev(table_np)
+    rng = np.random.default_rng(1)
+    h_np = rng.standard_normal((n, DIMS.d)).astype(np.float32)
+    depth = rng.integers(1, DIMS.R + 1, n)
+
+    def run(idx):
+        pool.copy_(dev(pool_np, torch.bfloat16))
+        seq = [int(i) if i >= 0 else -1 for i in idx]
+        pos = [ctxs[i] - 1 if i >= 0 else 0 for i in idx]
+        dep = [int(depth[i]) if i >= 0 else 1 for i in idx]
+        rows = B.Rows(i32(seq), i32(pos), table, loop_depth=i32(dep), kv_slot=i32([0] * len(idx)))
+        cdb.boundary_embed(i32([0] * len(idx)), rows, torch.zeros((len(idx), DIMS.d), device="cuda"))   # fresh gate state
+        h = dev(np.stack([h_np[i] if i >= 0 else np.zeros(DIMS.d, np.float32) for i in idx]))
+        gate, fire = torch.zeros(len(idx), device="cuda"), torch.zeros(len(idx), dtype=torch.uint8, device="cuda")
+        cdb.loop_step(rows, h, gate, fire)
+        torch.cuda.synchronize()
+        assert cdb.poll_status() == 0
+        out = {}
+        pl = pool.view(torch.int16).cpu().numpy()
+        for j, i in enumerate(idx):
+            if i >= 0:
+                page, off = table_np[i, (ctxs[i] - 1) // 16], (ctxs[i] - 1) % 16
+                out[i] = (h[j].cpu().numpy().view(np.int32), gate[j].cpu().numpy().view(np.int32), int(fire[j]),
+                          pl[:, page, :, :, off, :].copy())
+        return out
+
+    full = run(list(range(n)))
+    for subset in ([4], [7], [0], [7, 4], [-1, 5, -1, 2], [8, 6, 3, 1]):
+        part = run(subset)
+        for i, (hh, gg, ff, kv) in part.items():
+            assert np.array_equal(hh, full[i][0]), (subset, i)
+            assert np.array_equal(gg, full[i][1]) and ff == full[i][2], (subset, i)
+            assert np.array_equal(kv, full[i][3]), (subset, i)
