@@ -106,17 +106,22 @@ void layer_forward(cdb_t* h, int ln, int layer, const RowsDev& rows, float* x, c
 // with SwiGLU in its epilogue.  xn_ready: L.xn already holds RMSNorm(x; g_attn[layer]).  next_gain:
 // gain of the norm that follows this layer on the same rows (NULL: none).
 void layer_forward_tc(cdb_t* h, int ln, int layer, const RowsDev& rows, float* x, cudaStream_t st, bool xn_ready,
-                      const float* next_gain, cudaEvent_t attn_after = nullptr, cudaEvent_t attn_done = nullptr) {
+                      const float* next_gain, int next_layer, cudaEvent_t attn_after = nullptr, cudaEvent_t attn_done = nullptr) {
     const cdb_config_t& c = h->cfg;
     const Lane& L = h->lane[ln];
     const int n = rows.n_rows;
     const size_t d = c.d, F = c.F;
-    if (!xn_ready) launch_rmsnorm(h, x, h->g_attn + (size_t)layer * d, L.xn, rows, st);
+    int& qkv_parts = h->qkv_parts_ready[ln];                    // > 0: the previous layer's launch already left this layer's QKV parts in L.ws
+    if (!xn_ready) { launch_rmsnorm(h, x, h->g_attn + (size_t)layer * d, L.xn, rows, st); qkv_parts = 0; }
     {
         ProfScope ps(h, kProfLinear, st);
-        CDB_LAUNCH(h);
-        const int s = launch_linear_splitk_tc(h, L.xn, layer_ptr(h, h->w.W_qkv, layer, 3 * d * d), L.ws, kWsPerRow / 3, n, 3 * c.d, c.d, st);
-        if (!s) h->launch_error = 1;
+        int s = qkv_parts;
+        if (!s) {
+            CDB_LAUNCH(h);
+            s = launch_linear_splitk_tc(h, L.xn, layer_ptr(h, h->w.W_qkv, layer, 3 * d * d), L.ws, kWsPerRow / 3, n, 3 * c.d, c.d, st);
+            if (!s) h->launch_error = 1;
+        }
+        qkv_parts = 0;
         launch_rope_kv_write(h, ln, layer, L.ws, s, (size_t)n * 3 * d, rows, st);      // sums the parts
     }
     if (attn_after) cudaStreamWaitEvent(st, attn_after, 0);      // the other half-batch's attention goes first
@@ -124,6 +129,18 @@ void layer_forward_tc(cdb_t* h, int ln, int layer, const RowsDev& rows, float* x
     if (h->prefill_attention) launch_attention_prefill(h, ln, layer, rows, L.qrot, L.attn_o, st);
     else launch_attention(h, ln, layer, rows, L.qrot, L.attn_o, st);
     h->attn_split_done = nullptr;
+    if (c.flags & CDB_FLAG_FUSED_STAGES) {
+        // everything after the attention, and the next layer's QKV projection, in one cooperative launch
+        ProfScope ps(h, kProfLinear, st);
+        CDB_LAUNCH(h);
+        const int s = launch_layer_tail_tc(h, ln, rows, x, layer_ptr(h, h->w.W_o, layer, d * d), h->g_mlp + (size_t)layer * d,
+                                           layer_ptr(h, h->w.W_gate, layer, F * d), layer_ptr(h, h->w.W_up, layer, F * d),
+                                           layer_ptr(h, h->w.W_down, layer, d * F), next_gain,
+                                           next_layer >= 0 ? layer_ptr(h, h->w.W_qkv, next_layer, 3 * d * d) : nullptr, st);
+        if (s < 0) h->launch_error = 1;
+        qkv_parts = s > 0 ? s : 0;
+        return;
+    }
     {
         ProfScope ps(h, kProfLinear, st);
         CDB_LAUNCH(h);
@@ -160,7 +177,7 @@ void core_layers(cdb_t* h, int ln, const RowsDev& rows, float* x, cudaStream_t s
     cudaEvent_t after = layer == first ? attn_after_first : attn_after;
     if (use_tc_layers(h))
         layer_forward_tc(h, ln, layer, rows, x, st, layer > first, layer + 1 < last ? h->g_attn + (size_t)(layer + 1) * c.d : nullptr,
-                         after, attn_done);
+                         layer + 1 < last ? layer + 1 : -1, after, attn_done);
     else
         layer_forward(h, ln, layer, rows, x, st, after, attn_done);
 }
@@ -176,7 +193,7 @@ void lm_head(cdb_t* h, int ln, const RowsDev& rows, const float* x, int32_t* tok
 
 void free_all(cdb_t* h) {
     void* ptrs[] = {h->rope_cos, h->rope_sin, h->g_attn, h->g_mlp, h->g_final, h->gate_S, h->gate_fire,
-                    h->h_prev, h->h_work, h->logits, h->exit_flag, h->status, h->emit_tmp};
+                    h->h_prev, h->h_work, h->logits, h->exit_flag, h->status, h->emit_tmp, h->grid_sync};
     for (void* p : ptrs) if (p) cudaFree(p);
     for (Lane& L : h->lane) {
         void* lp[] = {L.xn, L.qrot, L.attn_o, L.act, L.qkv, L.gu, L.ws, L.attn_part, L.attn_item_start, L.attn_counters, L.pf_tile_rows, L.pf_n_tiles};
@@ -273,6 +290,7 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
     CDB_ALLOC(h->logits, float, R_ * (size_t)c.V);
     CDB_ALLOC(h->exit_flag, uint8_t, R_);
     CDB_ALLOC(h->status, int32_t, 1);
+    CDB_ALLOC(h->grid_sync, unsigned int, 2);
     CDB_ALLOC(h->emit_tmp, int32_t, R_);
 #undef CDB_ALLOC
     if (e != cudaSuccess) { free_all(h); delete h; cudaGetLastError(); return e == cudaErrorMemoryAllocation ? CDB_ERR_NOMEM : CDB_ERR_CUDA; }
@@ -311,6 +329,7 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
         gains_to_f32(h, w->g_final, h->g_final, d);
         init_gate_state_kernel<<<(c.max_seqs + 255) / 256, 256>>>(h->gate_S, h->gate_fire, c.max_seqs);
         cudaMemset(h->status, 0, sizeof(int32_t));
+        cudaMemset(h->grid_sync, 0, 2 * sizeof(unsigned int));
         for (int ln = 0; ln < 2; ++ln) cudaMemset(h->lane[ln].attn_counters, 0, sizeof(int32_t) * L);
         if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess) h->side = nullptr;
         cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
@@ -549,7 +568,10 @@ int cdb_linear(cdb_t* h, const void* x, const void* W, float* y, int32_t n, int3
 int cdb_poll_status(cdb_t* h, int32_t* status_host) {
     if (!h || !status_host) return CDB_ERR_ARG;
     cudaError_t e = cudaMemcpy(status_host, h->status, sizeof(int32_t), cudaMemcpyDeviceToHost);
-    if (e == cudaSuccess && *status_host != 0) e = cudaMemset(h->status, 0, sizeof(int32_t));     // read and re-arm
+    if (e == cudaSuccess && *status_host != 0) {                                                 // read and re-arm
+        e = cudaMemset(h->status, 0, sizeof(int32_t));
+        cudaMemset(h->grid_sync, 0, 2 * sizeof(unsigned int));        // a barrier a timed-out kernel left half way
+    }
     return e == cudaSuccess ? CDB_OK : fail_cuda(h, e, "cdb_poll_status");
 }
 

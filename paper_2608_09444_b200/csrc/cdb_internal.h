@@ -96,6 +96,7 @@ struct cdb {
     float* logits;                  // [max_rows][V]
     uint8_t* exit_flag;             // [max_rows]
     int32_t* status;                // [1] first out-of-range access seen (0 = clean)
+    unsigned int* grid_sync;        // [1] barrier word of the multi-stage layer kernel
     int32_t* emit_tmp;              // [max_rows]
     char err[256];
 
@@ -105,6 +106,7 @@ struct cdb {
     cudaEvent_t ev_fork, ev_join, ev_attn[2];
     mutable cudaEvent_t attn_split_done; // recorded right after the next attention split kernel when set
     mutable int attn_ctas_per_sm_cap;
+    mutable int qkv_parts_ready[2];     // per lane: split-K parts of the next layer's QKV projection already in the workspace
     mutable int prefill_attention;      // 1 while cdb_prefill runs: layers use the query-tiled causal attention
     mutable int gemm_smem_cap;          // > 0: projection kernels keep their shared-memory ring below this many bytes   // > 0: leave room on every SM for the other half-batch's kernels
 
@@ -187,6 +189,9 @@ void launch_repack_tiled(const void* W, void* Wt, int layers, int N, int K, cuda
 bool linear_tc_supported(const cdb* h, int n, int N, int K);
 bool launch_gate_up_swiglu_tc(const cdb* h, const void* x, const void* Wg, const void* Wu, void* act, int n, int F, int K, cudaStream_t st);
 int launch_linear_splitk_tc(const cdb* h, const void* x, const void* W, float* ws, int max_splits, int n, int N, int K, cudaStream_t st);
+int launch_layer_tail_tc(const cdb* h, int ln, const RowsDev& rows, float* x, const void* W_o, const float* g_mlp,
+                         const void* W_gate, const void* W_up, const void* W_down, const float* next_gain,
+                         const void* W_qkv_next, cudaStream_t st);
 
 // y[n,N] (fp32) = / += x[n,K] . W[N,K]^T ; x and W of the handle's dtype.
 void launch_linear(const cdb* h, const void* x, const void* W, float* y, int n, int N, int K, Epilogue ep, cudaStream_t st);

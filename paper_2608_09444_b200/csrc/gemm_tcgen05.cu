@@ -53,50 +53,31 @@ struct GemmParams {
 
 __device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t) :: "memory"); return t; }
 
-__global__ void __launch_bounds__(kThreads, 1)
-gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w2,
-                         const __grid_constant__ CUtensorMap map_x, GemmParams p) {
-    pdl_trigger();
-    if (p.dbg && threadIdx.x == 0) p.dbg[blockIdx.x * 8 + 0] = gtime();
-    extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bars[2 * 8 + 4];          // full[stages], empty[stages], acc_full[2], acc_empty[2]
-    __shared__ uint32_t tmem_base_slot;
-    __shared__ int abort_flag;
+// What one CTA needs to know about itself to run a projection: ring base, barrier block, TMEM base.
+struct CtaCtx {
+    uint32_t ring, bar0, tmem_base;
+    volatile int* abortp;
+};
 
+// The three roles of one projection over this CTA's share of the tiles (see the header of this file).  The
+// mbarriers at cx.bar0 must be freshly initialised (all phases 0) and the ring and TMEM idle.  wait_inputs()
+// is called by the producer warp after it has started the weight copies of its first ring fill and before
+// its first copy of an activation tile: it must return once the activations (and the output buffers) may
+// be touched.
+template <typename WaitInputs>
+__device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUtensorMap* map_w2, const CUtensorMap* map_x,
+                                           const GemmParams& p, const CtaCtx& cx, WaitInputs wait_inputs) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int S = p.stages, BN = p.BN;
     const bool dual = p.mode == kModeSwiGLU;                                 // two weight tiles, two accumulators
     const uint32_t w_bytes = BM * BK * 2, x_bytes = (uint32_t)BN * BK * 2;
     const uint32_t x_off = dual ? 2 * w_bytes : w_bytes, stage_bytes = x_off + x_bytes;
     const uint32_t acc_cols = dual ? 2u * BN : (uint32_t)BN;                 // TMEM columns of one accumulator set
-    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;            // swizzled tiles need 1024-byte alignment
-    const uint32_t bar0 = smem_u32(bars);
+    const uint32_t ring = cx.ring, bar0 = cx.bar0;
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (8 + s); };
     auto acc_full_bar = [&](int a) { return bar0 + 8u * (16 + a); };
     auto acc_empty_bar = [&](int a) { return bar0 + 8u * (18 + a); };
-    const uint32_t tmem_cols = 2u * acc_cols;                               // double-buffered; 128, 256 or 512
-
-    if (threadIdx.x == 0) {
-        abort_flag = 0;
-        for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 4); }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t tmem_base = tmem_base_slot;
-    volatile int* abortp = &abort_flag;
-    if (p.dbg && threadIdx.x == 0) p.dbg[blockIdx.x * 8 + 1] = gtime();
-    // Set-up above overlaps the previous kernel's tail.  The weights do not depend on that kernel, so the
-    // producer warp starts their copies before it waits (below); every other warp waits here.
-    if (warp != 0) pdl_wait();
-
     const int n_ftiles = (p.N + BM - 1) / BM, n_rtiles = (p.n + BN - 1) / BN;
     const int n_tiles = n_ftiles * n_rtiles * p.k_splits;                   // tile t = (split, row tile, feature tile)
     const int n_kb = (p.K + BK - 1) / BK;
@@ -112,8 +93,9 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
             // arms the stage barriers and starts the weight copies, then the warp waits for the previous
             // kernel, and pass 1 adds the activation copies.  Later stages take both copies at once.
             int n_pre = 0;                                   // stages filled by pass 0
+            int n_filled = 0;                                // stage fills of this CTA
             for (int pass = 0; pass < 2; ++pass) {
-                if (pass == 1) pdl_wait();
+                if (pass == 1) wait_inputs();
                 int g = 0;                                   // position in this CTA's (tile, k-block) sequence
                 for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
                     const int f0 = (t % n_ftiles) * BM, r0 = (t / n_ftiles % n_rtiles) * BN;
@@ -129,34 +111,43 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
                             const uint32_t dst = ring + (uint32_t)g * stage_bytes;
                             if (leader) {
                                 mbar_expect_tx(full_bar(g), stage_bytes);
-                                tma_load_2d(dst, &map_w, full_bar(g), wc, wr);
-                                if (dual) tma_load_2d(dst + w_bytes, &map_w2, full_bar(g), wc, wr);
+                                tma_load_2d(dst, map_w, full_bar(g), wc, wr);
+                                if (dual) tma_load_2d(dst + w_bytes, map_w2, full_bar(g), wc, wr);
                             }
                             __syncwarp();
                             n_pre = g + 1;
                             continue;
                         }
                         if (g < n_pre) {
-                            if (leader) tma_load_2d(ring + (uint32_t)g * stage_bytes + x_off, &map_x, full_bar(g), kb * BK, r0);
+                            if (leader) tma_load_2d(ring + (uint32_t)g * stage_bytes + x_off, map_x, full_bar(g), kb * BK, r0);
                             __syncwarp();
                             if (++s == S) { s = 0; ph ^= 1u; }
                             continue;
                         }
-                        if (!mbar_wait(empty_bar(s), ph ^ 1u, abortp)) { ok = false; break; }
+                        if (!mbar_wait(empty_bar(s), ph ^ 1u, cx.abortp)) { ok = false; break; }
                         const uint32_t dst = ring + (uint32_t)s * stage_bytes;
                         if (leader) {
                             mbar_expect_tx(full_bar(s), stage_bytes);
-                            tma_load_2d(dst, &map_w, full_bar(s), wc, wr);
-                            if (dual) tma_load_2d(dst + w_bytes, &map_w2, full_bar(s), wc, wr);
-                            tma_load_2d(dst + x_off, &map_x, full_bar(s), kb * BK, r0);
+                            tma_load_2d(dst, map_w, full_bar(s), wc, wr);
+                            if (dual) tma_load_2d(dst + w_bytes, map_w2, full_bar(s), wc, wr);
+                            tma_load_2d(dst + x_off, map_x, full_bar(s), kb * BK, r0);
                         }
                         __syncwarp();
                         if (++s == S) { s = 0; ph ^= 1u; }
                     }
                 }
+                if (pass == 1) n_filled = g;
             }
-            if (!ok || *abortp) {                        // give copies already in flight time to land
+            if (!ok || *cx.abortp) {                        // give copies already in flight time to land
                 for (int i = 0; i < 64; ++i) __nanosleep(1000);
+            } else {
+                // Drain: wait until every stage this CTA filled has been released, so that no tcgen05.commit
+                // arrival is still on its way when the caller re-arms the barriers for another projection.
+                const int n_fill = n_filled;
+                for (int j = 0; j < S && j < n_fill; ++j) {
+                    const int fills = n_fill / S + (j < n_fill % S ? 1 : 0);
+                    if (!mbar_wait(empty_bar(j), (uint32_t)(fills - 1) & 1u, cx.abortp)) break;
+                }
             }
         }
         __syncwarp();
@@ -172,12 +163,12 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
             for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
                 const int acc = it & 1;
                 const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
-                if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, abortp)) { ok = false; break; }
+                if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, cx.abortp)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t d_tmem = tmem_base + (uint32_t)acc * acc_cols;
+                const uint32_t d_tmem = cx.tmem_base + (uint32_t)acc * acc_cols;
                 const int kb0 = kb_begin(t), kb1 = kb_end(t);
                 for (int kb = kb0; kb < kb1; ++kb) {        // arrival order of the stages; which k-block is in one does not matter here
-                    if (!mbar_wait(full_bar(s), ph, abortp)) { ok = false; break; }
+                    if (!mbar_wait(full_bar(s), ph, cx.abortp)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a_addr = ring + (uint32_t)s * stage_bytes;
                     const uint64_t a_desc = smem_desc_sw128(a_addr), a2_desc = smem_desc_sw128(a_addr + w_bytes);
@@ -207,10 +198,10 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
             const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
             const int f = (t % n_ftiles) * BM + q * 32 + lane, r0 = (t / n_ftiles % n_rtiles) * BN;
             const int split = t / (n_ftiles * n_rtiles);
-            if (!mbar_wait(acc_full_bar(acc), acc_ph, abortp)) { ok = false; break; }
+            if (!mbar_wait(acc_full_bar(acc), acc_ph, cx.abortp)) { ok = false; break; }
             if (p.dbg && it == 0 && warp == 2 && lane == 0) p.dbg[blockIdx.x * 8 + 4] = gtime();
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * acc_cols;
+            const uint32_t t_addr = cx.tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * acc_cols;
             // 16 columns (= 16 batch rows) of this thread's feature per pass: a small register footprint
             const int n_cols = min(BN, p.n - r0);               // columns holding real rows (warp-uniform)
             if (dual) {
@@ -301,12 +292,250 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
         }
     }
 
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w2,
+                         const __grid_constant__ CUtensorMap map_x, GemmParams p) {
+    pdl_trigger();
+    if (p.dbg && threadIdx.x == 0) p.dbg[blockIdx.x * 8 + 0] = gtime();
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bars[2 * 8 + 4];          // full[stages], empty[stages], acc_full[2], acc_empty[2]
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int S = p.stages, BN = p.BN;
+    const bool dual = p.mode == kModeSwiGLU;                                 // two weight tiles, two accumulators
+    const uint32_t w_bytes = BM * BK * 2, x_bytes = (uint32_t)BN * BK * 2;
+    const uint32_t x_off = dual ? 2 * w_bytes : w_bytes, stage_bytes = x_off + x_bytes;
+    const uint32_t acc_cols = dual ? 2u * BN : (uint32_t)BN;                 // TMEM columns of one accumulator set
+    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;            // swizzled tiles need 1024-byte alignment
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (8 + s); };
+    auto acc_full_bar = [&](int a) { return bar0 + 8u * (16 + a); };
+    auto acc_empty_bar = [&](int a) { return bar0 + 8u * (18 + a); };
+    const uint32_t tmem_cols = 2u * acc_cols;                               // double-buffered; 128, 256 or 512
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+    if (p.dbg && threadIdx.x == 0) p.dbg[blockIdx.x * 8 + 1] = gtime();
+    // Set-up above overlaps the previous kernel's tail.  The weights do not depend on that kernel, so the
+    // producer warp starts their copies before it waits (below); every other warp waits here.
+    if (warp != 0) pdl_wait();
+
+    CtaCtx cx;
+    cx.ring = ring; cx.bar0 = bar0; cx.tmem_base = tmem_base; cx.abortp = abortp;
+    gemm_roles(&map_w, &map_w2, &map_x, p, cx, [] { pdl_wait(); });
+
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (threadIdx.x == 0 && abort_flag) atomicCAS(p.status, 0, kStatusTimeout);
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------
+// Several dependent stages of a layer in ONE launch (opt-in, CDB_FLAG_FUSED_STAGES): projections (as above)
+// and the row-wise "sum the split-K parts + residual + RMSNorm" step, separated by grid-wide barriers instead
+// of kernel boundaries; the producer warp starts the NEXT projection's weight copies before it waits at the
+// barrier.  The launch is cooperative (every CTA resident), all waits are bounded.  Measured: a barrier
+// among 148 CTAs plus re-arming the pipeline costs MORE (~11.7 us per stage) than a kernel boundary chained
+// with programmatic dependent launch (~8 us per stage, set-up already overlapped, weights already
+// prefetched), so the separate launches stay the default.
+constexpr int kTailMaxPhases = 6;
+enum { kPhaseProjection = 0, kPhaseReduceNorm = 1 };
+
+struct TailPhase {
+    int kind;
+    int map_w, map_w2, map_x;          // projection: indices into TailMaps
+    GemmParams g;
+    const float* ws;                   // reduce: parts [splits][n_rows][d]
+    int splits;
+    size_t split_stride;
+    float* x;                          // reduce: residual stream, updated in place
+    const float* gain;                 // reduce: NULL = no normed output
+    __nv_bfloat16* out;
+};
+
+struct TailParams {
+    int n_phases;
+    TailPhase ph[kTailMaxPhases];
+    const int32_t* seq_id;             // pads (< 0) are skipped by the row-wise stage
+    int n_rows, d;
+    float eps;
+    unsigned int* sync;                // grid barrier word (top bit flips once per barrier)
+    int32_t* status;
+};
+
+struct TailMaps { CUtensorMap m[3 * kTailMaxPhases]; };
+
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Arrive at the grid barrier (one thread per CTA); returns the ticket to wait on.  CTA 0 adds what is
+// missing to carry into the top bit once all gridDim.x CTAs have arrived, so the word needs no reset.
+__device__ __forceinline__ unsigned int grid_arrive(unsigned int* word) {
+    const unsigned int inc = blockIdx.x == 0 ? 0x80000000u - (gridDim.x - 1) : 1u;
+    __threadfence();
+    return atomicAdd(word, inc);
+}
+__device__ __forceinline__ bool grid_wait(const unsigned int* word, unsigned int ticket, volatile int* abort_flag) {
+    const long long t0 = clock64();
+    for (uint32_t it = 0;; ++it) {
+        if (((ticket ^ ld_acquire_u32(word)) & 0x80000000u) != 0) return true;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitCycles) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+layer_tail_tcgen05_kernel(const __grid_constant__ TailMaps maps, const __grid_constant__ TailParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bars[2 * 8 + 4];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+    __shared__ unsigned int ticket;               // of the grid barrier in flight
+    __shared__ float red[4];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bar0 = smem_u32(bars);
+    constexpr uint32_t tmem_cols = 512;
+    auto init_barriers = [&]() {
+        for (int s = 0; s < 8; ++s) { mbar_init(bar0 + 8u * s, 1); mbar_init(bar0 + 8u * (8 + s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(bar0 + 8u * (16 + a), 1); mbar_init(bar0 + 8u * (18 + a), 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    };
+    if (threadIdx.x == 0) { abort_flag = 0; init_barriers(); }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    CtaCtx cx;
+    cx.ring = ring; cx.bar0 = bar0; cx.tmem_base = tmem_base_slot; cx.abortp = &abort_flag;
+    volatile int* abortp = &abort_flag;
+    if (warp != 0) pdl_wait();
+
+    for (int pi = 0; pi < P.n_phases; ++pi) {
+        const TailPhase& ph = P.ph[pi];
+        const bool last_wait = pi + 1 == P.n_phases;        // whoever passes the last barrier lets the next kernel launch
+        if (ph.kind == kPhaseProjection) {
+            gemm_roles(&maps.m[ph.map_w], &maps.m[ph.map_w2], &maps.m[ph.map_x], ph.g, cx, [&] {
+                if (pi == 0) {
+                    pdl_wait();
+                } else {
+                    if (lane == 0) grid_wait(P.sync, ticket, abortp);
+                    __syncwarp();
+                    asm volatile("fence.proxy.async;" ::: "memory");     // other CTAs' stores, then this warp's TMA reads
+                }
+                if (last_wait && lane == 0) pdl_trigger();
+            });
+        } else if (warp >= 2) {
+            const int et = threadIdx.x - 64, q = warp - 2;                // 128 threads share a row
+            if (pi > 0) {
+                if (et == 0) grid_wait(P.sync, ticket, abortp);
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+            }
+            if (last_wait && et == 0) pdl_trigger();
+            constexpr int MAXV = 12;                                      // float4 chunks per thread: d <= 12 * 4 * 128
+            const int d4 = P.d / 4;
+            for (int row = blockIdx.x; row < P.n_rows; row += gridDim.x) {
+                if (P.seq_id != nullptr && P.seq_id[row] < 0) {
+                    if (ph.gain)
+                        for (int i = et; i < d4; i += 128) *reinterpret_cast<uint2*>(ph.out + (size_t)row * P.d + 4 * i) = make_uint2(0u, 0u);
+                    continue;
+                }
+                float4 v[MAXV];
+                float ss = 0.f;
+#pragma unroll
+                for (int k = 0; k < MAXV; ++k) {
+                    const int i = et + 128 * k;
+                    if (i < d4) {
+                        const size_t at = (size_t)row * d4 + i;
+                        float4 a = __ldcg(reinterpret_cast<const float4*>(ph.x) + at);
+                        for (int s = 0; s < ph.splits; ++s) {             // fixed order: part 0, 1, ...
+                            const float4 b = __ldcg(reinterpret_cast<const float4*>(ph.ws + (size_t)s * ph.split_stride) + at);
+                            a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+                        }
+                        reinterpret_cast<float4*>(ph.x)[at] = a;
+                        v[k] = a;
+                        ss = fmaf(a.x, a.x, fmaf(a.y, a.y, fmaf(a.z, a.z, fmaf(a.w, a.w, ss))));
+                    }
+                }
+                if (!ph.gain) continue;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+                asm volatile("bar.sync 1, 128;" ::: "memory");            // previous row's sums consumed
+                if (lane == 0) red[q] = ss;
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                const float inv = rsqrtf((red[0] + red[1] + red[2] + red[3]) / (float)P.d + P.eps);
+#pragma unroll
+                for (int k = 0; k < MAXV; ++k) {
+                    const int i = et + 128 * k;
+                    if (i < d4) {
+                        const float4 g = reinterpret_cast<const float4*>(ph.gain)[i];
+                        const __nv_bfloat162 lo = __floats2bfloat162_rn(v[k].x * inv * g.x, v[k].y * inv * g.y);
+                        const __nv_bfloat162 hi = __floats2bfloat162_rn(v[k].z * inv * g.z, v[k].w * inv * g.w);
+                        uint2 w;
+                        w.x = *reinterpret_cast<const uint32_t*>(&lo);
+                        w.y = *reinterpret_cast<const uint32_t*>(&hi);
+                        *reinterpret_cast<uint2*>(ph.out + (size_t)row * P.d + 4 * i) = w;
+                    }
+                }
+            }
+        }
+        if (pi + 1 < P.n_phases) {
+            // Stage boundary: everything this CTA wrote is made visible (to plain loads and to TMA reads of
+            // other CTAs), the pipeline barriers are re-armed, and the CTA arrives at the grid barrier.  The
+            // wait happens where the next stage first needs another CTA's data.
+            __threadfence();
+            asm volatile("fence.proxy.async;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                for (int b = 0; b < 20; ++b) asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(bar0 + 8u * b) : "memory");
+                init_barriers();
+                ticket = grid_arrive(P.sync);
+            }
+            __syncthreads();
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (abort_flag) break;
+        }
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag) atomicCAS(P.status, 0, kStatusTimeout);
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(cx.tmem_base), "r"(tmem_cols) : "memory");
     }
 }
 
@@ -352,21 +581,12 @@ void launch_repack_tiled(const void* W, void* Wt, int layers, int N, int K, cuda
     repack_tiled_kernel<<<148 * 8, 256, 0, st>>>((const __nv_bfloat16*)W, (__nv_bfloat16*)Wt, layers, N, K);
 }
 
-// Common launcher.  W2 / act only in SwiGLU mode.  k_splits > 1 only with kModeStore (y = workspace).
-static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* W2, float* y, __nv_bfloat16* act, int n,
-                        int N, int K, int mode, int k_splits, size_t split_stride, cudaStream_t st) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-        if (getenv("CDB_GEMM_CARVEOUT"))
-            cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, atoi(getenv("CDB_GEMM_CARVEOUT")));
-        attr_set = true;
-    }
-    GemmParams p;
+// Parameters and tensor maps of one projection.  W2 / act only in SwiGLU mode.  k_splits > 1 only with
+// kModeStore (y = workspace).  Returns the number of tiles, 0 on failure.
+static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2, float* y, __nv_bfloat16* act, int n,
+                      int N, int K, int mode, int k_splits, size_t split_stride, GemmParams& p, CUtensorMap* map_w,
+                      CUtensorMap* map_w2, CUtensorMap* map_x, size_t* smem) {
     p.y = y; p.act = act; p.n = n; p.N = N; p.K = K; p.mode = mode; p.k_splits = k_splits; p.split_stride = split_stride;
-    int sms = 148, dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int n_ft = (N + BM - 1) / BM;
     static const int forced_bn = getenv("CDB_GEMM_BN") ? atoi(getenv("CDB_GEMM_BN")) : 0;     // tuning aid
     const int bn_max = mode == kModeSwiGLU ? 128 : 256;
@@ -384,24 +604,61 @@ static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* 
     if (p.stages > 8) p.stages = 8;
     p.stage_out_off = (uint32_t)(p.stages * stage_bytes);
     p.status = h->status;
-    p.dbg = getenv("CDB_GEMM_DBG") ? (unsigned long long*)strtoull(getenv("CDB_GEMM_DBG"), nullptr, 0) : nullptr;
-    if (getenv("CDB_GEMM_DBG_ONLY") && atoi(getenv("CDB_GEMM_DBG_ONLY")) != mode * 100000 + N) p.dbg = nullptr;   // tuning aid: one launch kind
-    CUtensorMap map_w, map_w2, map_x;
+    p.dbg = nullptr;
     const int n_kb = (K + BK - 1) / BK;
     const void* Wt = find_tiled(h, W, N, K);
     const void* Wt2 = W2 ? find_tiled(h, W2, N, K) : Wt;
     p.w_tiled = (Wt && Wt2) ? 1 : 0;
     if (p.w_tiled) {
-        if (!make_map(&map_w, Wt, n_ft * n_kb * BM, BK, BM) || !make_map(&map_w2, Wt2, n_ft * n_kb * BM, BK, BM)) return false;
+        if (!make_map(map_w, Wt, n_ft * n_kb * BM, BK, BM) || !make_map(map_w2, Wt2, n_ft * n_kb * BM, BK, BM)) return 0;
     } else {
-        if (!make_map(&map_w, W, N, K, BM) || !make_map(&map_w2, W2 ? W2 : W, N, K, BM)) return false;
+        if (!make_map(map_w, W, N, K, BM) || !make_map(map_w2, W2 ? W2 : W, N, K, BM)) return 0;
     }
-    if (!make_map(&map_x, x, n, K, p.BN)) return false;
-    const int n_tiles = n_ft * ((n + p.BN - 1) / p.BN) * k_splits;
+    if (!make_map(map_x, x, n, K, p.BN)) return 0;
+    *smem = (size_t)p.stages * stage_bytes + stage_out + 1024;
+    return n_ft * ((n + p.BN - 1) / p.BN) * k_splits;
+}
+
+static int device_sms() {
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    return sms;
+}
+
+static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* W2, float* y, __nv_bfloat16* act, int n,
+                        int N, int K, int mode, int k_splits, size_t split_stride, cudaStream_t st) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (getenv("CDB_GEMM_CARVEOUT"))
+            cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, atoi(getenv("CDB_GEMM_CARVEOUT")));
+        attr_set = true;
+    }
+    GemmParams p;
+    CUtensorMap map_w, map_w2, map_x;
+    size_t smem = 0;
+    const int n_tiles = setup_gemm(h, x, W, W2, y, act, n, N, K, mode, k_splits, split_stride, p, &map_w, &map_w2, &map_x, &smem);
+    if (!n_tiles) return false;
+    p.dbg = getenv("CDB_GEMM_DBG") ? (unsigned long long*)strtoull(getenv("CDB_GEMM_DBG"), nullptr, 0) : nullptr;
+    if (getenv("CDB_GEMM_DBG_ONLY") && atoi(getenv("CDB_GEMM_DBG_ONLY")) != mode * 100000 + N) p.dbg = nullptr;   // tuning aid: one launch kind
+    const int sms = device_sms();
     const int grid = n_tiles < sms ? n_tiles : sms;
-    const size_t smem = (size_t)p.stages * stage_bytes + stage_out + 1024;
     launch_pdl(gemm_bf16_tcgen05_kernel, dim3(grid), dim3(kThreads), smem, st, map_w, map_w2, map_x, p);
     return true;
+}
+
+// Part count of a split-K projection.  It depends on the weight's shape alone, never on the number of rows,
+// so that a row's result does not depend on the batch it is computed in: about one tile per SM for a batch
+// that fills one row tile, and at least four k-blocks per part.
+static int splitk_parts(int N, int K, int max_splits) {
+    const int sms = device_sms();
+    const int n_ft = (N + BM - 1) / BM, n_kb = (K + BK - 1) / BK;
+    int splits = (sms + n_ft / 2) / n_ft;
+    if (splits > n_kb / 4) splits = n_kb / 4;
+    if (splits > max_splits) splits = max_splits;
+    if (splits < 1) splits = 1;
+    return splits;
 }
 
 bool launch_linear_tc(const cdb* h, const void* x, const void* W, float* y, int n, int N, int K, Epilogue ep, cudaStream_t st) {
@@ -416,19 +673,82 @@ bool launch_gate_up_swiglu_tc(const cdb* h, const void* x, const void* Wg, const
 // Split-K: partial products ws[s][n][N] (fp32), s < returned split count; the caller reduces them in
 // split order (deterministic).
 int launch_linear_splitk_tc(const cdb* h, const void* x, const void* W, float* ws, int max_splits, int n, int N, int K, cudaStream_t st) {
-    // The part count depends on the weight's shape alone, never on the number of rows, so that a row's
-    // result does not depend on the batch it is computed in: about one tile per SM for a batch that
-    // fills one row tile, and at least four k-blocks per part.
-    (void)n;
-    int sms = 148, dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int n_ft = (N + BM - 1) / BM, n_kb = (K + BK - 1) / BK;
-    int splits = (sms + n_ft / 2) / n_ft;
-    if (splits > n_kb / 4) splits = n_kb / 4;
-    if (splits > max_splits) splits = max_splits;
-    if (splits < 1) splits = 1;
+    const int splits = splitk_parts(N, K, max_splits);
     return launch_gemm(h, x, W, nullptr, ws, nullptr, n, N, K, kModeStore, splits, (size_t)n * N, st) ? splits : 0;
+}
+
+// Everything of a layer after its attention in one cooperative launch: output projection (split-K) ->
+// parts + residual + RMSNorm(g_mlp) -> gate/up projections with SwiGLU -> down projection (split-K) ->
+// parts + residual + RMSNorm(next_gain) [-> the next layer's QKV projection (split-K) into qkv_ws].  Same
+// arithmetic as the separate launches; returns the part count of the QKV stage (0 when it was not asked
+// for), -1 on failure.
+int launch_layer_tail_tc(const cdb* h, int ln, const RowsDev& rows, float* x, const void* W_o, const float* g_mlp,
+                         const void* W_gate, const void* W_up, const void* W_down, const float* next_gain,
+                         const void* W_qkv_next, cudaStream_t st) {
+    const Lane& L = h->lane[ln];
+    const cdb_config_t& c = h->cfg;
+    const int n = rows.n_rows, d = c.d, F = c.F;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(layer_tail_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess) return -1;
+        attr_set = true;
+    }
+    TailMaps maps;
+    TailParams P;
+    size_t smem = 0, smem_max = 0;
+    int np = 0;
+    auto projection = [&](const void* xin, const void* W, const void* W2, float* y, __nv_bfloat16* act, int N, int K, int mode, int splits) {
+        TailPhase& ph = P.ph[np];
+        ph.kind = kPhaseProjection;
+        ph.map_w = 3 * np; ph.map_w2 = 3 * np + 1; ph.map_x = 3 * np + 2;
+        ph.ws = nullptr; ph.splits = 0; ph.split_stride = 0; ph.x = nullptr; ph.gain = nullptr; ph.out = nullptr;
+        const int tiles = setup_gemm(h, xin, W, W2, y, act, n, N, K, mode, splits, (size_t)n * N, ph.g, &maps.m[ph.map_w],
+                                     &maps.m[ph.map_w2], &maps.m[ph.map_x], &smem);
+        if (smem > smem_max) smem_max = smem;
+        ++np;
+        return tiles > 0;
+    };
+    auto reduce = [&](int splits, const float* gain) {
+        TailPhase& ph = P.ph[np];
+        ph.kind = kPhaseReduceNorm;
+        ph.map_w = ph.map_w2 = ph.map_x = 0;
+        ph.g = GemmParams();
+        ph.ws = L.ws; ph.splits = splits; ph.split_stride = (size_t)n * d; ph.x = x; ph.gain = gain; ph.out = (__nv_bfloat16*)L.xn;
+        ++np;
+    };
+    const int s_o = splitk_parts(d, d, kMaxKSplits), s_d = splitk_parts(d, F, kMaxKSplits);
+    int s_q = 0;
+    if (!projection(L.attn_o, W_o, nullptr, L.ws, nullptr, d, d, kModeStore, s_o)) return -1;
+    reduce(s_o, g_mlp);
+    if (!projection(L.xn, W_gate, W_up, nullptr, (__nv_bfloat16*)L.act, F, d, kModeSwiGLU, 1)) return -1;
+    if (!projection(L.act, W_down, nullptr, L.ws, nullptr, d, F, kModeStore, s_d)) return -1;
+    reduce(s_d, next_gain);
+    if (W_qkv_next) {
+        s_q = splitk_parts(3 * d, d, kWsPerRow / 3);
+        if (!projection(L.xn, W_qkv_next, nullptr, L.ws, nullptr, 3 * d, d, kModeStore, s_q)) return -1;
+    }
+    P.n_phases = np;
+    P.seq_id = rows.seq_id; P.n_rows = n; P.d = d; P.eps = c.eps; P.sync = h->grid_sync; P.status = h->status;
+    for (int i = 3 * np; i < 3 * kTailMaxPhases; ++i) maps.m[i] = maps.m[0];
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(device_sms()); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem_max; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    static int with_pdl = getenv("CDB_NO_PDL") ? 0 : 1;
+    cfg.numAttrs = 1 + with_pdl;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, layer_tail_tcgen05_kernel, maps, P);
+    if (e != cudaSuccess && with_pdl) {            // this driver does not combine the two attributes: plain cooperative launch
+        cudaGetLastError();
+        with_pdl = 0;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, layer_tail_tcgen05_kernel, maps, P);
+    }
+    return e == cudaSuccess ? s_q : -1;
 }
 
 }  // namespace cdbk

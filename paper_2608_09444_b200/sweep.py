@@ -50,7 +50,7 @@ def fit(points):
             "max_rel_residual": float(np.max(np.abs(pred - y) / y))}
 
 
-def sweep(dims, batches, lengths, *, pool_tokens, warmup=3, steps=10, seed=7, device="cuda:0"):
+def sweep(dims, batches, lengths, *, pool_tokens, warmup=3, steps=10, seed=7, device="cuda:0", flags=0, graph=False):
     dev = torch.device(device)
     torch.cuda.set_device(dev)
     max_rows, max_len = max(batches), max(lengths)
@@ -58,7 +58,7 @@ def sweep(dims, batches, lengths, *, pool_tokens, warmup=3, steps=10, seed=7, de
     n_pages = (pool_tokens + dims.page_size - 1) // dims.page_size
     weights = synth.make_weights(dims, seed, device=str(dev), std=0.02, gate_std=2.0 / np.sqrt(dims.d))
     cdb = B.Cdb(dims, weights, max_rows=max_rows, max_seqs=max_rows, max_position=width * dims.page_size,
-                gate_kind=B.GATE_SIGMOID_CDF, q_or_eps=0.5)
+                gate_kind=B.GATE_SIGMOID_CDF, q_or_eps=0.5, flags=flags)
     dt = torch.float32 if dims.dtype == "fp32" else torch.bfloat16
     pool = torch.empty(synth.kv_pool_shape(dims, n_pages), dtype=dt, device=dev)
     synth.fill_kv_pool(pool, seed + 1000)
@@ -95,7 +95,15 @@ def sweep(dims, batches, lengths, *, pool_tokens, warmup=3, steps=10, seed=7, de
                 else:
                     cdb.boundary_embed(tokens[:nb], rows, h_new[:nb])
 
-            t = _median_ms(step, warmup, steps, dev)
+            if graph:                     # replay the step as one CUDA graph (what the engines do)
+                step()
+                torch.cuda.synchronize(dev)
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    step()
+                t = _median_ms(g.replay, warmup, steps, dev)
+            else:
+                t = _median_ms(step, warmup, steps, dev)
             points.append([nb, L, t])
             boundary.append([nb, L, _median_ms(bound, warmup, steps, dev)])
             st = cdb.poll_status()
@@ -127,10 +135,12 @@ def main(argv=None):
     ap.add_argument("--pool-tokens", type=int, default=524288, help="KV pool size in tokens (Ouro: 192 KiB each)")
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--flags", type=int, default=0, help="library flags (binding.FLAG_*), e.g. 2 = two-stream half-batches")
+    ap.add_argument("--graph", action="store_true", help="time CUDA-graph replays of the step instead of direct launches")
     args = ap.parse_args(argv)
     dims = {"ouro": synth.OURO_1P4B, "huginn": synth.HUGINN_3P5B, "tiny": synth.TINY}[args.model]
     out = sweep(dims, [int(x) for x in args.batches.split(",")], [int(x) for x in args.lengths.split(",")],
-                pool_tokens=args.pool_tokens, warmup=args.warmup, steps=args.steps)
+                pool_tokens=args.pool_tokens, warmup=args.warmup, steps=args.steps, flags=args.flags, graph=args.graph)
     print(json.dumps(out))
 
 

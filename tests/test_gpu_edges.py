@@ -106,12 +106,12 @@ def test_range_errors_are_reported_not_faulted():
     assert "max_rows" in str(e.value) or "rows" in str(e.value)
 
 
-@pytest.mark.parametrize("flags,extra", [(0, 0), (4, 0), (0, 70), (0, 200)])
+@pytest.mark.parametrize("flags,extra", [(0, 0), (4, 0), (0, 70), (0, 200), (16, 0), (16, 200)])
 def test_a_rows_result_does_not_depend_on_its_batch(flags, extra):
     """Run nine rows together, then three of them alone, as a pair in another order and among pads: hidden
     states, gate values, exit signals and the K/V written must be identical bit for bit (shape-only split-K
     with fixed-order sums, attention splits that depend only on the row's own context).  flags=4 repeats the
-    check on the unfused layer flow; `extra` more rows make the full batch wide enough for the projection
+    check on the unfused layer flow, flags=16 on the multi-stage cooperative layer kernel; `extra` more rows make the full batch wide enough for the projection
     kernel's 128- and 256-row tiles."""
     ctxs = [1, 16, 17, 40, 255, 256, 257, 300, 33] + [int(c) for c in np.random.default_rng(2).integers(1, 90, extra)]
     n = len(ctxs)

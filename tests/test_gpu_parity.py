@@ -203,8 +203,9 @@ STEP_CASES = [
 ]
 
 
-@pytest.mark.parametrize("dims,gate_kind", STEP_CASES)
-def test_loop_step_rows_match_oracle(dims, gate_kind):
+@pytest.mark.parametrize("dims,gate_kind,flags", [c + (0,) for c in STEP_CASES] + [STEP_CASES[1] + (16,), STEP_CASES[2] + (16,)])
+def test_loop_step_rows_match_oracle(dims, gate_kind, flags):
+    """flags=16: the same step with everything after the attention in one cooperative multi-stage launch."""
     binding = B()
     wd, wn = make_model(dims, 21, gate_std=0.1, b_gate=-0.2)
     ctxs = np.array([1, 16, 17, 40, 255, 256, 257, 300, 33])
@@ -212,7 +213,7 @@ def test_loop_step_rows_match_oracle(dims, gate_kind):
     table_np, n_pages = synth.make_page_table(ctxs, 16, seed=9, permute=True, extra_pages=2)
     eps_l2 = 1e30 if gate_kind == 2 else 0.5
     cdb = binding.Cdb(dims, wd, max_rows=n + 1, max_seqs=n, max_position=table_np.shape[1] * 16,
-                      gate_kind=gate_kind, q_or_eps=0.4 if gate_kind == 1 else eps_l2)
+                      gate_kind=gate_kind, q_or_eps=0.4 if gate_kind == 1 else eps_l2, flags=flags)
     rng = np.random.default_rng(8)
     pool_np = rng.standard_normal(synth.kv_pool_shape(dims, n_pages)).astype(np.float32)
     h_np = rng.standard_normal((n + 1, dims.d)).astype(np.float32)
