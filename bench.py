@@ -121,6 +121,7 @@ def main():
     ap.add_argument("--ctx-lo", type=int, default=128)
     ap.add_argument("--ctx-hi", type=int, default=2048)
     ap.add_argument("--layers", type=int, default=0, help="override the core layer count (small ncu captures only)")
+    ap.add_argument("--contiguous-pages", action="store_true", help="ascending physical pages instead of a random permutation")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--simt-gemm", action="store_true", help="run projections on the plain-FMA cross-check kernel")
     ap.add_argument("--two-stream", action="store_true", help="split the step into two half-batches on two streams (experimental)")
@@ -141,7 +142,7 @@ def main():
 
     dims = synth.OURO_1P4B if args.layers <= 0 else synth.OURO_1P4B.replace(L_core=args.layers)
     workload = f"ouro-1.4b-shaped loop step, {args.rows} rows, depth U{{1..{dims.R}}}, context U{{{args.ctx_lo}..{args.ctx_hi}}}, 16-token pages"
-    config = {"workload": workload, "rows": args.rows, "core_layers": dims.L_core, "page_table": "random permutation",
+    config = {"workload": workload, "rows": args.rows, "core_layers": dims.L_core, "page_table": "contiguous" if args.contiguous_pages else "random permutation",
               "l2": "inputs larger than L2 (each step streams the whole KV pool and all core weights)"}
 
     if world > 1:
@@ -151,7 +152,7 @@ def main():
     from paper_2608_09444_b200 import binding as B
     from paper_2608_09444_b200.workloads import LoopStepWorkload
     wl = LoopStepWorkload(dims, n_rows=args.rows, seed=D.rank_seed(1, rank), ctx_lo=args.ctx_lo, ctx_hi=args.ctx_hi,
-                          device=f"cuda:{local_rank}", flags=(B.FLAG_SIMT_GEMM if args.simt_gemm else 0) | (B.FLAG_TWO_STREAM if args.two_stream else 0))
+                          permute=not args.contiguous_pages, device=f"cuda:{local_rank}", flags=(B.FLAG_SIMT_GEMM if args.simt_gemm else 0) | (B.FLAG_TWO_STREAM if args.two_stream else 0))
     alg = wl.algorithmic()
     cores = len(os.sched_getaffinity(0))
 
@@ -217,7 +218,7 @@ def main():
     # half-batch launches): bytes per launch = bytes of all launches / number of launches
     att_bytes_per_launch = alg["attention_per_launch"] * dims.L_core * args.steps / max(att["count"], 1)
     achieved = att_bytes_per_launch / (att_ms * 1e-3) / 1e9 if att_ms > 0 else 0.0
-    default_workload = args.rows == 256 and args.ctx_lo == 128 and args.ctx_hi == 2048
+    default_workload = args.rows == 256 and args.ctx_lo == 128 and args.ctx_hi == 2048 and not args.contiguous_pages
     out = {"metric": METRIC, "value": world * args.rows / (ms_step * 1e-3), "unit": "token-loop-steps/s",
            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
