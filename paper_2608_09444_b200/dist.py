@@ -31,3 +31,35 @@ def max_over_ranks(value: float, device="cpu") -> float:
     t = torch.tensor([float(value)], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def route_least_loaded(arrivals, kv_tokens, out_lens, world: int, est_s_per_token: float = 0.01):
+    """Front-end assignment of requests to replicas: each request, in arrival order, goes to the replica
+    that holds the fewest reserved KV tokens at its arrival time (ties: lowest rank).  A request reserves
+    kv_tokens[i] (prompt + output) from its arrival until its estimated finish, arrival + out_lens[i] *
+    est_s_per_token.  A pure function of the trace, so every rank computes the same assignment without
+    talking to the others.  Returns the replica index of every request."""
+    import heapq
+    load = [0] * world
+    releases = []                                   # (time, rank, tokens)
+    out = []
+    for i in range(len(arrivals)):
+        t = float(arrivals[i])
+        while releases and releases[0][0] <= t:
+            _, r, k = heapq.heappop(releases)
+            load[r] -= k
+        r = min(range(world), key=lambda j: (load[j], j))
+        load[r] += int(kv_tokens[i])
+        heapq.heappush(releases, (t + int(out_lens[i]) * est_s_per_token, r, int(kv_tokens[i])))
+        out.append(r)
+    return out
+
+
+def gather_objects(obj):
+    """[obj of rank 0, obj of rank 1, ...] on every rank; [obj] when there is one rank."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [obj]
+    out = [None] * dist.get_world_size()
+    dist.all_gather_object(out, obj)
+    return out

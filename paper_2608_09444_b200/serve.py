@@ -9,6 +9,10 @@ continuous batching (every token loops r_max times) and continuous depth batchin
     python -m paper_2608_09444_b200.serve --model ouro --rates 4,8,16 --requests 300
 
 The engines run against the wall clock, so a run lasts requests / rate seconds plus the drain.
+
+Under torchrun (one rank per GPU) every rank is a full replica with its own page pool and scheduler; a
+front-end rule (least reserved KV tokens at arrival, `dist.route_least_loaded`) assigns each request to a
+replica, the ranks serve their shares against the same clock, and rank 0 merges the per-request times.
 """
 from __future__ import annotations
 
@@ -19,6 +23,7 @@ import numpy as np
 import torch
 
 from . import binding as B
+from . import dist as D
 from . import synth
 from .engine import Engine
 from .engine_async import PipelinedEngine
@@ -48,18 +53,31 @@ def summarize(arrivals, out_lens, stats):
             "prefill_calls": stats["prefill_calls"], "coda_calls": stats["coda_calls"]}
 
 
+def merge_replicas(parts, n_requests):
+    """Per-request time stamps and summed counters of all replicas, in request order."""
+    merged = {"finish_s": [None] * n_requests, "first_token_s": [None] * n_requests,
+              "recurrent_steps": 0, "row_steps": 0, "prefill_calls": 0, "coda_calls": 0}
+    for p in parts:
+        for j, i in enumerate(p["ids"]):
+            merged["finish_s"][i], merged["first_token_s"][i] = p["finish_s"][j], p["first_token_s"][j]
+        for k, v in p["counters"].items():
+            merged[k] += v
+    return merged
+
+
 def run(dims, weights, arrivals, prompts, out_lens, *, mode, pipelined, gate_kind, q_or_eps=0.5, forced_depths=None,
         max_batch=256, max_live=320, pool_tokens=400000, min_coda_batch=1, max_prefill_rows=4096,
-        admit_min=1, admit_wait_s=0.0):
+        admit_min=1, admit_wait_s=0.0, device="cuda:0"):
     max_len = max(len(p) + t for p, t in zip(prompts, out_lens))
     pages = (pool_tokens + dims.page_size - 1) // dims.page_size
     eng = (PipelinedEngine if pipelined else Engine)(
         dims, weights, max_batch=max_batch, max_live=max_live, max_len=max_len, n_pages=pages, gate_kind=gate_kind,
         q_or_eps=q_or_eps, lookahead=True, mode=mode, min_coda_batch=min_coda_batch,
         max_prefill_rows=max(max_prefill_rows, max(len(p) for p in prompts)), record_ticks=False,
-        admit_min=admit_min, admit_wait_s=admit_wait_s)
+        admit_min=admit_min, admit_wait_s=admit_wait_s, device=device)
     res = eng.generate(prompts, out_lens, forced_depths=forced_depths, arrivals=arrivals)
     out = summarize(arrivals, out_lens, eng.stats)
+    out["finish_s"], out["first_token_s"] = list(eng.stats["finish_s"]), list(eng.stats["first_token_s"])
     out["mode"] = mode + ("_pipelined" if pipelined else "")
     out["status"] = eng.cdb.poll_status()
     d = np.concatenate([x for x in res["depths"] if len(x)]) if any(len(x) for x in res["depths"]) else np.zeros(0)
@@ -82,9 +100,13 @@ def main():
     ap.add_argument("--admit-min", type=int, default=1, help="hold arrived requests until this many wait ...")
     ap.add_argument("--admit-wait-ms", type=float, default=0.0, help="... or the oldest has waited this long")
     args = ap.parse_args()
-    torch.cuda.set_device(0)
+    rank, local_rank, world = D.env_rank()
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl")
+    torch.cuda.set_device(local_rank)
     dims, seed = (synth.OURO_1P4B, 4) if args.model == "ouro" else (synth.HUGINN_3P5B, 5)
-    w = synth.make_weights(dims, seed, device="cuda:0", gate_std=2.0 / np.sqrt(dims.d))
+    w = synth.make_weights(dims, seed, device=f"cuda:{local_rank}", gate_std=2.0 / np.sqrt(dims.d))
     report = {"model": args.model, "requests": args.requests, "runs": []}
     if args.model == "ouro":
         gate_kind = B.GATE_SIGMOID_CDF
@@ -97,17 +119,30 @@ def main():
         forced = None
         if args.model == "huginn":       # replayed exit depths: truncated geometric, mean 12
             forced = [list(synth.forced_exit_depths((1, max(t - 1, 1)), seed + 100 + i, 12.0, dims.R)[0]) for i, t in enumerate(out_lens)]
+        # this replica's share of the trace (all of it on one GPU)
+        owner = D.route_least_loaded(arrivals, [len(p) + t for p, t in zip(prompts, out_lens)], out_lens, world)
+        mine = [i for i in range(args.requests) if owner[i] == rank]
         for mode in args.modes.split(","):
             pipelined = mode.endswith("_pipelined")
             m = mode.replace("_pipelined", "")
-            out, _ = run(dims, w, arrivals, prompts, out_lens, mode=m, pipelined=pipelined, gate_kind=gate_kind,
-                         forced_depths=None if m == "cb" else forced, max_batch=args.max_batch, max_live=args.max_live,
+            if world > 1:
+                torch.distributed.barrier()           # the replicas start their clocks together
+            out, _ = run(dims, w, arrivals[mine], [prompts[i] for i in mine], [out_lens[i] for i in mine], mode=m,
+                         pipelined=pipelined, gate_kind=gate_kind,
+                         forced_depths=None if (m == "cb" or forced is None) else [forced[i] for i in mine],
+                         max_batch=args.max_batch, max_live=args.max_live,
                          pool_tokens=args.pool_tokens, min_coda_batch=1 if args.model == "ouro" else 32,
-                         admit_min=args.admit_min, admit_wait_s=args.admit_wait_ms * 1e-3)
-            out["rate_req_per_s"] = rate
-            report["runs"].append(out)
-            print(json.dumps(out), flush=True)
-    print(json.dumps(report))
+                         admit_min=args.admit_min, admit_wait_s=args.admit_wait_ms * 1e-3, device=f"cuda:{local_rank}")
+            parts = D.gather_objects({"ids": mine, "finish_s": out.pop("finish_s"), "first_token_s": out.pop("first_token_s"),
+                                      "counters": {k: out[k] for k in ("recurrent_steps", "row_steps", "prefill_calls", "coda_calls")}})
+            if rank == 0:
+                merged = merge_replicas(parts, args.requests)
+                out.update(summarize(arrivals, out_lens, merged))
+                out["rate_req_per_s"], out["replicas"] = rate, world
+                report["runs"].append(out)
+                print(json.dumps(out), flush=True)
+    if rank == 0:
+        print(json.dumps(report))
 
 
 if __name__ == "__main__":

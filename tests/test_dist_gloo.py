@@ -79,3 +79,50 @@ def test_serving_trace_and_latency_summary():
     assert abs(s["normalized_latency_s_per_token"]["mean"] - lat.mean()) < 1e-12
     assert abs(s["normalized_latency_s_per_token"]["p99"] - 0.5) < 1e-12
     assert abs(s["generated_tokens_per_s"] - 13 / 5.0) < 1e-12 and abs(s["time_to_first_token_s"]["mean"] - (0.5 + 0.5 + 0.25) / 3) < 1e-12
+
+
+def _serve_worker(rank, world, port, out):
+    """Two replicas of the serving front end on CPU: same routing on both ranks, each fakes its own requests'
+    time stamps, rank 0 merges them."""
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank))
+    from paper_2608_09444_b200 import dist as D
+    from paper_2608_09444_b200.serve import make_requests, merge_replicas, summarize
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    arrivals, prompts, out_lens = make_requests(40, 16.0, 9, 1000)
+    owner = D.route_least_loaded(arrivals, [len(p) + t for p, t in zip(prompts, out_lens)], out_lens, world)
+    mine = [i for i in range(40) if owner[i] == rank]
+    part = {"ids": mine, "finish_s": [float(arrivals[i]) + 0.01 * out_lens[i] for i in mine],
+            "first_token_s": [float(arrivals[i]) + 0.005 for i in mine],
+            "counters": {"recurrent_steps": 10 + rank, "row_steps": 100, "prefill_calls": len(mine), "coda_calls": 7}}
+    parts = D.gather_objects(part)
+    merged = merge_replicas(parts, 40)
+    summary = summarize(arrivals, out_lens, merged)
+    out.put((rank, owner, mine, summary["normalized_latency_s_per_token"]["mean"], merged["recurrent_steps"], merged["prefill_calls"]))
+    dist.destroy_process_group()
+
+
+def test_two_replicas_route_gather_and_merge():
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_serve_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert res[0][1] == res[1][1]                                           # the same assignment on every rank
+    assert sorted(res[0][2] + res[1][2]) == list(range(40))                 # a partition of the requests
+    assert min(len(res[0][2]), len(res[1][2])) >= 10                        # both replicas get work
+    assert abs(res[0][3] - 0.01) < 1e-9 and abs(res[1][3] - 0.01) < 1e-9    # merged latency = the faked 10 ms/token
+    assert res[0][4] == 21 and res[0][5] == 40
+
+
+def test_router_prefers_the_replica_with_fewer_reserved_tokens():
+    from paper_2608_09444_b200.dist import route_least_loaded
+    # three requests at the same time: sizes 100, 10, 10 -> ranks 0, 1, 1; after the big one finishes the next goes to 0
+    owner = route_least_loaded([0.0, 0.0, 0.0, 5.0], [100, 10, 10, 50], [10, 1000, 1000, 10], 2, est_s_per_token=0.01)
+    assert owner == [0, 1, 1, 0]
+    assert route_least_loaded([0.0, 1.0], [5, 5], [1, 1], 1) == [0, 0]
