@@ -89,27 +89,28 @@ struct cdb {
     TiledWeight tiled[6];           // W_qkv, W_o, W_gate, W_up, W_down, W_lm (bf16 configs)
     int n_tiled;
 
-    // per-lane scratch: lane 0 holds max_rows rows, lane 1 half of that (second half-batch of a split step)
+    // per-lane scratch, max_rows rows each: lane 0 serves the loop step and prefill, lane 1 the boundary calls (so
+    // that they may overlap a loop step on another stream) and the second half-batch of a two-stream step
     cdbk::Lane lane[2];
     float* h_prev;                  // [max_rows][d] state at step entry (convergence gate)
     float* h_work;                  // [max_rows][d] prefill working state
     float* logits;                  // [max_rows][V]
     uint8_t* exit_flag;             // [max_rows]
     int32_t* status;                // [1] first out-of-range access seen (0 = clean)
-    unsigned int* grid_sync;        // [1] barrier word of the multi-stage layer kernel
+    unsigned int* grid_sync;        // [2] per lane: barrier word of the multi-stage layer kernel
     int32_t* emit_tmp;              // [max_rows]
     char err[256];
 
-    // instrumentation: kernel launch count, and CUDA-event pairs around the two heavy kernel classes
     // two-stream execution of a loop step: second half-batch on `side`, joined by events
     cudaStream_t side;
     cudaEvent_t ev_fork, ev_join, ev_attn[2];
     mutable cudaEvent_t attn_split_done; // recorded right after the next attention split kernel when set
-    mutable int attn_ctas_per_sm_cap;
+    mutable int attn_ctas_per_sm_cap;   // > 0 (two-stream step): attention runs one CTA of this many x 4 warps per SM
     mutable int qkv_parts_ready[2];     // per lane: split-K parts of the next layer's QKV projection already in the workspace
     mutable int prefill_attention;      // 1 while cdb_prefill runs: layers use the query-tiled causal attention
-    mutable int gemm_smem_cap;          // > 0: projection kernels keep their shared-memory ring below this many bytes   // > 0: leave room on every SM for the other half-batch's kernels
+    mutable int gemm_smem_cap;          // > 0 (two-stream step): projection kernels keep their shared-memory ring below this many bytes
 
+    // instrumentation: kernel launch count, and CUDA-event pairs around the two heavy kernel classes
     mutable uint64_t launches;
     mutable int launch_error;       // a launcher could not set up its kernel (tensor-map encode failed)
     mutable int prof_on, prof_used;

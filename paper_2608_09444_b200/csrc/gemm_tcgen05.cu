@@ -728,7 +728,7 @@ int launch_layer_tail_tc(const cdb* h, int ln, const RowsDev& rows, float* x, co
         if (!projection(L.xn, W_qkv_next, nullptr, L.ws, nullptr, 3 * d, d, kModeStore, s_q)) return -1;
     }
     P.n_phases = np;
-    P.seq_id = rows.seq_id; P.n_rows = n; P.d = d; P.eps = c.eps; P.sync = h->grid_sync; P.status = h->status;
+    P.seq_id = rows.seq_id; P.n_rows = n; P.d = d; P.eps = c.eps; P.sync = h->grid_sync + ln; P.status = h->status;
     for (int i = 3 * np; i < 3 * kTailMaxPhases; ++i) maps.m[i] = maps.m[0];
 
     cudaLaunchConfig_t cfg = {};
