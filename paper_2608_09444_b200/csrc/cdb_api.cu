@@ -75,6 +75,8 @@ const void* layer_ptr(const cdb_t* h, const void* base, int layer, size_t elems_
     return (const char*)base + (size_t)layer * wstride(h, elems_per_layer);
 }
 
+bool use_tc_layers(const cdb_t* h);
+
 // One transformer layer on `x` (fp32 [n_rows, d], updated in place).  Steps A1-A6 of the loop step:
 // RMSNorm + QKV projection, RoPE + KV page write, paged attention, output projection + residual,
 // RMSNorm + gate/up projections + SwiGLU, down projection + residual.
@@ -94,9 +96,18 @@ void layer_forward(cdb_t* h, int ln, int layer, const RowsDev& rows, float* x, c
     h->attn_split_done = nullptr;
     launch_linear(h, L.attn_o, layer_ptr(h, h->w.W_o, layer, d * d), x, n, c.d, c.d, Epilogue::ResidualAdd, st);
     launch_rmsnorm(h, x, h->g_mlp + (size_t)layer * d, L.xn, rows, st);
-    launch_linear(h, L.xn, layer_ptr(h, h->w.W_gate, layer, F * d), L.gu, n, c.F, c.d, Epilogue::Store, st);
-    launch_linear(h, L.xn, layer_ptr(h, h->w.W_up, layer, F * d), L.gu + (size_t)L.rows_cap * F, n, c.F, c.d, Epilogue::Store, st);
-    launch_swiglu(h, ln, n, st);
+    bool fused_mlp = false;
+    if (use_tc_layers(h)) {                  // bf16 tensor-core path: gate and up in one launch, SwiGLU in its epilogue
+        ProfScope ps(h, kProfLinear, st);
+        CDB_LAUNCH(h);
+        fused_mlp = launch_gate_up_swiglu_tc(h, L.xn, layer_ptr(h, h->w.W_gate, layer, F * d), layer_ptr(h, h->w.W_up, layer, F * d),
+                                             L.act, n, c.F, c.d, st);
+    }
+    if (!fused_mlp) {
+        launch_linear(h, L.xn, layer_ptr(h, h->w.W_gate, layer, F * d), L.gu, n, c.F, c.d, Epilogue::Store, st);
+        launch_linear(h, L.xn, layer_ptr(h, h->w.W_up, layer, F * d), L.gu + (size_t)L.rows_cap * F, n, c.F, c.d, Epilogue::Store, st);
+        launch_swiglu(h, ln, n, st);
+    }
     launch_linear(h, L.act, layer_ptr(h, h->w.W_down, layer, d * F), x, n, c.d, c.F, Epilogue::ResidualAdd, st);
 }
 
