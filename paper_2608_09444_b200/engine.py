@@ -439,7 +439,10 @@ def _run_step(eng: "Engine", k: int, seq, depth, pos, slot, forced):
         _step_body(eng, _static_rows(eng, nb), nb)
         return
     if nb not in eng.graphs:
-        # warm-up on an all-pad descriptor (touches no state), then capture
+        # Warm-up on an all-pad descriptor, then capture.  Pads touch neither the KV pool nor the gate state, but
+        # the body ends by moving the (empty) survivor list to the front of h_rec, which would overwrite the
+        # rows waiting there for this very step: keep them aside.
+        saved = eng.h_rec[:nb].clone()
         eng.desc_dev[0, :nb].fill_(-1)
         rows = _static_rows(eng, nb)
         _step_body(eng, rows, nb)
@@ -447,6 +450,7 @@ def _run_step(eng: "Engine", k: int, seq, depth, pos, slot, forced):
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
             _step_body(eng, rows, nb)
+        eng.h_rec[:nb].copy_(saved)
         eng.graphs[nb] = (g, rows)
     eng.desc_dev.copy_(dh, non_blocking=True)
     eng.graphs[nb][0].replay()

@@ -69,6 +69,25 @@ def calibrate_gate_bias(dims, weights, prompts, T, target, q=0.5, iters=10):
     return b
 
 
+def calibrate_convergence_eps(dims, weights, prompts, T, target, iters=14):
+    """Threshold of the convergence criterion (appendix C.2: exit once the L2 distance between consecutive
+    recurrent states is below eps) for which the mean exit depth of a short adaptive run is closest to
+    `target`: bisection on log(eps) on the product path (a larger eps exits earlier).  Returns (eps, mean depth)."""
+    lo, hi = np.log(1e-4), np.log(1e6)
+    best = None
+    for _ in range(iters):
+        mid = 0.5 * (lo + hi)
+        out, _ = run(dims, weights, prompts, T, mode="refill", gate_kind=B.GATE_L2_CONVERGENCE, q_or_eps=float(np.exp(mid)),
+                     max_prefill_rows=2048)
+        if best is None or abs(out["mean_depth"] - target) < abs(best[1] - target):
+            best = (float(np.exp(mid)), out["mean_depth"])
+        if out["mean_depth"] > target:
+            lo = mid
+        else:
+            hi = mid
+    return best
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--model", default="ouro", choices=["ouro", "huginn"])
@@ -80,6 +99,8 @@ def main():
     ap.add_argument("--min-coda-batch", type=int, default=0)
     ap.add_argument("--max-live", type=int, default=0, help="sequences resident at once (0 = all); fewer than --seqs queues the rest")
     ap.add_argument("--modes", default="cb,refill,no_refill", help="cb, refill, no_refill, refill_pipelined, refill_nographs")
+    ap.add_argument("--exits", default="forced", choices=["forced", "criterion"],
+                    help="huginn: replayed geometric exit depths, or the convergence criterion with a calibrated threshold")
     ap.add_argument("--time-device", action="store_true", help="bracket every GPU phase with CUDA events and report device_ms")
     args = ap.parse_args()
     torch.cuda.set_device(0)
@@ -95,19 +116,25 @@ def main():
                                             "layers": [dims.L_pre, dims.L_core, dims.L_coda], "R": dims.R},
               "seqs": args.seqs, "prompt": args.prompt, "tokens": args.tokens, "runs": []}
     forced = None
+    q_or_eps = 0.5
     if args.model == "ouro":
         gate_kind = B.GATE_SIGMOID_CDF
         report["b_gate"] = calibrate_gate_bias(dims, w, prompts[:16], min(args.tokens, 24), 2.5)
         min_coda = args.min_coda_batch or 1
-    else:                                   # forced exit depths from a truncated geometric distribution (mean 12, cap 32)
+    elif args.exits == "forced":            # forced exit depths from a truncated geometric distribution (mean 12, cap 32)
         gate_kind = B.GATE_NONE
         forced = [list(r) for r in synth.forced_exit_depths((args.seqs, args.tokens - 1), seed, 12.0, dims.R)]
+        min_coda = args.min_coda_batch or 32
+    else:                                   # training-free convergence criterion, threshold calibrated to mean depth ~12
+        gate_kind = B.GATE_L2_CONVERGENCE
+        q_or_eps, cal_depth = calibrate_convergence_eps(dims, w, prompts[:8], min(args.tokens, 12), 12.0)
+        report["eps"], report["calibration_mean_depth"] = q_or_eps, cal_depth
         min_coda = args.min_coda_batch or 32
     for mode in args.modes.split(","):
         pipelined = mode.endswith("_pipelined")
         nographs = mode.endswith("_nographs")
         mode = mode.replace("_pipelined", "").replace("_nographs", "")
-        out, _ = run(dims, w, prompts, args.tokens, mode=mode, pipelined=pipelined, use_graphs=not nographs, time_device=args.time_device, gate_kind=gate_kind, forced_depths=None if mode == "cb" else forced,
+        out, _ = run(dims, w, prompts, args.tokens, mode=mode, pipelined=pipelined, use_graphs=not nographs, time_device=args.time_device, gate_kind=gate_kind, q_or_eps=q_or_eps, forced_depths=None if mode == "cb" else forced,
                      max_batch=args.max_batch or None, max_live=args.max_live or None, min_coda_batch=min_coda)
         report["runs"].append(out)
         print(json.dumps(out), flush=True)

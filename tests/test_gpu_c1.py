@@ -191,3 +191,28 @@ def test_c1_requests_arriving_over_time_give_the_same_tokens(oracle_runs, pipeli
         assert np.array_equal(res["depths"][s], ref[s]["depths"][:lens[s] - 1]), s
         assert arrivals[s] <= eng.stats["first_token_s"][s] <= eng.stats["finish_s"][s]
     assert not [p for row in eng.page_table_host for p in row if p >= 0]
+
+
+def test_graph_buckets_first_used_mid_run_leave_waiting_rows_alone():
+    """40 sequences of different output lengths: the batch starts in the 64-row bucket and falls into the
+    32-row bucket while refilled rows are waiting at the front of the step's input; capturing that bucket's
+    graph then (its warm-up runs the step body once on pads) must not disturb them.  Graph replay, direct
+    launches and the pipelined engine must agree token for token and depth for depth."""
+    from paper_2608_09444_b200 import binding as B
+    from paper_2608_09444_b200.engine import Engine
+    from paper_2608_09444_b200.engine_async import PipelinedEngine
+    dims, w, _ = c1_inputs()
+    wd = {k: v.cuda() for k, v in w.items()}
+    n = 40
+    prompts = list(synth.make_prompts(n, 12, dims.V, 77))
+    lens = [int(t) for t in np.random.default_rng(5).integers(2, 14, n)]
+    runs = []
+    for cls, kw in ((Engine, {"use_graphs": True}), (Engine, {"use_graphs": False}), (PipelinedEngine, {})):
+        eng = cls(dims, wd, max_batch=n, max_live=n, max_len=32, n_pages=2 * n, gate_kind=B.GATE_SIGMOID_CDF, q_or_eps=0.5,
+                  max_prefill_rows=512, **kw)
+        runs.append(eng.generate(prompts, lens))
+        assert eng.cdb.poll_status() == 0
+    for other in runs[1:]:
+        for s in range(n):
+            assert np.array_equal(runs[0]["tokens"][s], other["tokens"][s]), s
+            assert np.array_equal(runs[0]["depths"][s], other["depths"][s]), s
