@@ -132,6 +132,16 @@ def test_c1_depth_aware_kv_layouts(layout):
     ref = [orc.generate(p, 16, keep_states=True) for p in prompts]
     eng, res = run_engine("refill", n_slots=O.n_slots(o_layout, dims.R), kv_layout=b_layout)
     compare(eng, res, ref)
+    # the asynchronous pipeline runs copy-on-exit and the boundary stages on its side stream: same tokens and depths
+    from paper_2608_09444_b200.engine_async import PipelinedEngine
+    n_slots = O.n_slots(o_layout, dims.R)
+    peng = PipelinedEngine(dims, {k: v.cuda() for k, v in w.items()}, max_batch=5, max_live=6, max_len=48, n_pages=3 * 6 * n_slots,
+                           gate_kind=B.GATE_SIGMOID_CDF, q_or_eps=0.5, max_prefill_rows=256, kv_layout=b_layout)
+    pres = peng.generate(list(prompts), 16)
+    assert peng.cdb.poll_status() == 0
+    for s in range(8):
+        assert np.array_equal(pres["tokens"][s], ref[s]["tokens"]), s
+        assert np.array_equal(pres["depths"][s], ref[s]["depths"]), s
 
 
 def test_c1_graph_replay_equals_direct_launches(oracle_runs):
