@@ -400,6 +400,19 @@ class Engine:
                 "gates": [s.gates for s in seqs]}
 
 
+def kv_footprint(dims, n_slots: int) -> tuple[int, int]:
+    """KV bytes per cached token: (in use, reserved by this library's pool).  In use is what the paper's
+    Table 1 counts: one K and one V vector per layer, the core layers once per depth slot.  The pool gives
+    every (sequence, slot) pair its own pages in ALL layers (page ids are shared by the layers), so the
+    prelude and coda layers' share of the pages of slots > 0 stays empty: reserved >= in use, equal for
+    fully looped models and for the shared layout."""
+    eb = 4 if dims.dtype == "fp32" else 2
+    per_layer = 2 * dims.H * dims.Dh * eb
+    used = (dims.L_pre + dims.L_coda + dims.L_core * n_slots) * per_layer
+    reserved = (dims.L_pre + dims.L_coda + dims.L_core) * n_slots * per_layer
+    return used, reserved
+
+
 def _bucket(k: int, cap: int) -> int:
     return min(cap, (k + 31) // 32 * 32)
 

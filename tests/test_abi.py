@@ -37,3 +37,20 @@ def test_null_handle_is_an_error_not_a_crash():
     assert binding.lib.cdb_set_gate(None, 0.0, 0.0) == binding.ERR_ARG
     assert binding.lib.cdb_poll_status(None, None) == binding.ERR_ARG
     assert binding.lib.cdb_last_error(None) == b"invalid handle"
+
+
+def test_kv_footprint_accounting_matches_table1():
+    """The driver's KV accounting against the sizes printed in the paper's Table 1 (appendix C.1), and the
+    pool's own reservation, which exceeds them only for models with boundary layers and more than one slot."""
+    import os
+    from paper_2608_09444_b200 import synth
+    from paper_2608_09444_b200.engine import kv_footprint
+    dims = {"ouro": synth.OURO_1P4B, "huginn": synth.HUGINN_3P5B}
+    golden = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "table1_kv_footprint.txt")
+    for line in open(golden):
+        if line.startswith("#") or not line.strip():
+            continue
+        model, slots, kib, gib = line.split()
+        used, reserved = kv_footprint(dims[model], int(slots))
+        assert abs(used / 1024 - float(kib)) <= 0.5 and abs(used * 4096 / 2**30 - float(gib)) <= 0.006
+        assert reserved >= used and (reserved == used) == (model == "ouro" or int(slots) == 1)
