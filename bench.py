@@ -145,9 +145,9 @@ def main():
     config = {"workload": workload, "rows": args.rows, "core_layers": dims.L_core, "page_table": "contiguous" if args.contiguous_pages else "random permutation",
               "l2": "inputs larger than L2 (each step streams the whole KV pool and all core weights)"}
 
-    if world > 1:
+    if world > 1 and args.impl == "cdb":     # the reference arm runs on rank 0 alone: no process group
         import torch.distributed as dist
-        dist.init_process_group("nccl" if args.impl == "cdb" else "gloo")
+        dist.init_process_group("nccl")
     torch.cuda.set_device(local_rank)
     from paper_2608_09444_b200 import binding as B
     from paper_2608_09444_b200.workloads import LoopStepWorkload
