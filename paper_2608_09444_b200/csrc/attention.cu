@@ -621,6 +621,10 @@ __global__ void __launch_bounds__(128) attn_prefill_kernel(AttnParams p, const i
 // Tile list of a prompt batch into the lane's split-scan buffer (first rows), pf_tile_rows and pf_n_tiles.
 void launch_prefill_plan(const cdb* h, int ln, const RowsDev& rows, int tile, cudaStream_t st) {
     const Lane& L = h->lane[ln];
+    // one plan per prompt call: every layer of the call sees the same rows (prefill_attention: 1 = no plan yet,
+    // otherwise 2 + the tile size of the plan in the lane's buffers)
+    if (h->prefill_attention == 2 + tile) return;
+    if (h->prefill_attention >= 1) h->prefill_attention = 2 + tile;
     CDB_LAUNCH(h);
     launch_pdl(prefill_plan_kernel, dim3(1), dim3(1024), 0, st, rows, tile, L.attn_item_start, L.pf_tile_rows, L.pf_n_tiles);
 }

@@ -107,7 +107,7 @@ struct cdb {
     mutable cudaEvent_t attn_split_done; // recorded right after the next attention split kernel when set
     mutable int attn_ctas_per_sm_cap;   // > 0 (two-stream step): attention runs one CTA of this many x 4 warps per SM
     mutable int qkv_parts_ready[2];     // per lane: split-K parts of the next layer's QKV projection already in the workspace
-    mutable int prefill_attention;      // 1 while cdb_prefill runs: layers use the query-tiled causal attention
+    mutable int prefill_attention;      // != 0 while cdb_prefill runs: layers use the query-tiled causal attention (1: tile list not planned yet)
     mutable int gemm_smem_cap;          // > 0 (two-stream step): projection kernels keep their shared-memory ring below this many bytes
 
     // instrumentation: kernel launch count, and CUDA-event pairs around the two heavy kernel classes
