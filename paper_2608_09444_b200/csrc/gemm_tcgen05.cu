@@ -581,6 +581,13 @@ void launch_repack_tiled(const void* W, void* Wt, int layers, int N, int K, cuda
     repack_tiled_kernel<<<148 * 8, 256, 0, st>>>((const __nv_bfloat16*)W, (__nv_bfloat16*)Wt, layers, N, K);
 }
 
+static int device_sms() {
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    return sms;
+}
+
 // Parameters and tensor maps of one projection.  W2 / act only in SwiGLU mode.  k_splits > 1 only with
 // kModeStore (y = workspace).  Returns the number of tiles, 0 on failure.
 static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2, float* y, __nv_bfloat16* act, int n,
@@ -593,6 +600,14 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
     // Rows per tile (MMA N): the widest of 64 / 128 / 256 the batch can fill: one tcgen05.mma then does the
     // most work per issue and each weight tile is pulled through L2 the fewest times.
     p.BN = n <= 64 ? 64 : (n <= 128 || bn_max == 128) ? 128 : 256;
+    // ... unless that leaves most SMs without a tile (projections without split-K on a few hundred rows, as in
+    // prompt processing): narrower row tiles then give more CTAs a share of the weight stream.  The tile
+    // width changes which CTA computes an output element, never how it is summed.
+    {
+        const int sms = device_sms();
+        auto tiles = [&](int bn) { return n_ft * ((n + bn - 1) / bn) * k_splits; };
+        while (p.BN > 64 && tiles(p.BN) * 2 < sms && n > p.BN / 2) p.BN /= 2;
+    }
     if ((forced_bn == 64 || forced_bn == 128 || forced_bn == 256) && forced_bn <= bn_max) p.BN = forced_bn;
     const int stage_bytes = (mode == kModeSwiGLU ? 2 : 1) * BM * BK * 2 + p.BN * BK * 2;
     static const int smem_cap = getenv("CDB_GEMM_SMEM_KB") ? atoi(getenv("CDB_GEMM_SMEM_KB")) * 1024 : kMaxSmem;   // tuning aid
@@ -617,13 +632,6 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
     if (!make_map(map_x, x, n, K, p.BN)) return 0;
     *smem = (size_t)p.stages * stage_bytes + stage_out + 1024;
     return n_ft * ((n + p.BN - 1) / p.BN) * k_splits;
-}
-
-static int device_sms() {
-    int sms = 148, dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    return sms;
 }
 
 static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* W2, float* y, __nv_bfloat16* act, int n,
