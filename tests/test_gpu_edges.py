@@ -149,3 +149,37 @@ def test_a_rows_result_does_not_depend_on_its_batch(flags, extra):
             assert np.array_equal(hh, full[i][0]), (subset, i)
             assert np.array_equal(gg, full[i][1]) and ff == full[i][2], (subset, i)
             assert np.array_equal(kv, full[i][3]), (subset, i)
+
+
+def test_host_checks_refuse_bad_calls_with_an_error_code():
+    """The error behaviour the header promises: inconsistent dims, a missing or undersized KV pool, the wrong
+    layout for copy-on-exit and an out-of-range layer come back as negative codes with a message; nothing is
+    launched and the handle stays usable."""
+    from paper_2608_09444_b200 import binding as B
+    w = synth.make_weights(DIMS, 3, std=0.05)
+    wd = {k: v.cuda() for k, v in w.items()}
+    with pytest.raises(B.CdbError) as e:
+        B.Cdb(DIMS.replace(d=DIMS.d + 8), wd, max_rows=4, max_seqs=4, max_position=64)       # d != H * Dh
+    assert e.value.code == -1
+    cdb = B.Cdb(DIMS, wd, max_rows=4, max_seqs=4, max_position=64)
+    table = i32(np.arange(16).reshape(4, 4))
+    rows = B.Rows(i32([0, 1]), i32([3, 5]), table, loop_depth=i32([1, 1]), kv_slot=i32([0, 0]))
+    h = torch.zeros((2, DIMS.d), device="cuda")
+    with pytest.raises(B.CdbError) as e:
+        cdb.loop_step(rows, h)                                                                   # no pool bound yet
+    assert e.value.code == -5 and "pool" in str(e.value)
+    with pytest.raises(B.CdbError) as e:
+        cdb.kv_bind(torch.zeros((1, 1000), dtype=torch.bfloat16, device="cuda"))                 # 1000 pages claimed, 2000 bytes given
+    assert e.value.code == -1 and "smaller" in str(e.value)
+    pool = torch.zeros(synth.kv_pool_shape(DIMS, 16), dtype=torch.bfloat16, device="cuda")
+    cdb.kv_bind(pool)
+    with pytest.raises(B.CdbError) as e:
+        cdb.kv_copy_on_exit(rows, i32([2, 2]))                                                   # shared layout
+    assert e.value.code == -5
+    with pytest.raises(B.CdbError) as e:
+        cdb.paged_attention(rows, 99, torch.zeros((2, DIMS.d), dtype=torch.bfloat16, device="cuda"),
+                            torch.zeros((2, DIMS.d), dtype=torch.bfloat16, device="cuda"))
+    assert e.value.code == -4
+    cdb.loop_step(rows, h)                                                                       # still usable
+    torch.cuda.synchronize()
+    assert cdb.poll_status() == 0
