@@ -193,6 +193,18 @@ void core_layers(cdb_t* h, int ln, const RowsDev& rows, float* x, cudaStream_t s
         layer_forward(h, ln, layer, rows, x, st, after, attn_done);
 }
 
+// layers [first, last) of the prelude or coda on a decode batch (one row per sequence): the split-K flow when
+// the tensor-core path is available, else the plain sequence
+void boundary_layers(cdb_t* h, int ln, int first, int last, const RowsDev& rows, float* x, cudaStream_t st) {
+    for (int l = first; l < last; ++l) {
+        if (use_tc_layers(h))
+            layer_forward_tc(h, ln, l, rows, x, st, l > first, l + 1 < last ? h->g_attn + (size_t)(l + 1) * h->cfg.d : nullptr,
+                             l + 1 < last ? l + 1 : -1);
+        else
+            layer_forward(h, ln, l, rows, x, st);
+    }
+}
+
 // final RMSNorm + LM head + greedy argmax on n rows of x
 void lm_head(cdb_t* h, int ln, const RowsDev& rows, const float* x, int32_t* token_out, float* logits_out, cudaStream_t st) {
     const cdb_config_t& c = h->cfg;
@@ -396,7 +408,7 @@ static int boundary_in(cdb_t* h, const int32_t* token_ids, const cdb_rows_t* row
         if (!h->pool.base) return fail(h, CDB_ERR_STATE, "no KV pool bound");
         rd.slot_override = 0;
         launch_attention_plan(h, kBoundaryLane, rd, st);
-        for (int l = 0; l < h->cfg.L_pre; ++l) layer_forward(h, kBoundaryLane, l, rd, h_out, st);
+        boundary_layers(h, kBoundaryLane, 0, h->cfg.L_pre, rd, h_out, st);
     }
     return check_launch(h, "cdb_boundary_embed/prelude");
 }
@@ -499,7 +511,7 @@ int cdb_boundary_coda_lmhead(cdb_t* h, const cdb_rows_t* rows, float* h_exit, in
         if (!h->pool.base) return fail(h, CDB_ERR_STATE, "no KV pool bound");
         rd.slot_override = 0;
         launch_attention_plan(h, kBoundaryLane, rd, st);
-        for (int l = c.L_pre + c.L_core; l < c.L_pre + c.L_core + c.L_coda; ++l) layer_forward(h, kBoundaryLane, l, rd, h_exit, st);
+        boundary_layers(h, kBoundaryLane, c.L_pre + c.L_core, c.L_pre + c.L_core + c.L_coda, rd, h_exit, st);
     }
     lm_head(h, kBoundaryLane, rd, h_exit, token_out, logits_out, st);
     return check_launch(h, "cdb_boundary_coda_lmhead");
