@@ -246,17 +246,39 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(AttnParams p, T* __rest
         return;
     }
     const float* part = p.part + (size_t)(row * H + head) * p.max_splits * (DH + 2);
+    // Splits are taken four at a time with all their loads issued before the first use (a loop that waits for
+    // each split's loads in turn costs one memory latency per split); the sums keep their split order.
+    constexpr int U = 4;
     float M = -INFINITY;
-    for (int s = 0; s < ns; ++s) M = fmaxf(M, part[(size_t)s * (DH + 2) + DH]);
+    for (int s0 = 0; s0 < ns; s0 += U) {
+        float mv[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) mv[u] = s0 + u < ns ? part[(size_t)(s0 + u) * (DH + 2) + DH] : -INFINITY;
+#pragma unroll
+        for (int u = 0; u < U; ++u) M = fmaxf(M, mv[u]);
+    }
     float L = 0.f, acc[PER];
 #pragma unroll
     for (int k = 0; k < PER; ++k) acc[k] = 0.f;
-    for (int s = 0; s < ns; ++s) {
-        const float* ps = part + (size_t)s * (DH + 2);
-        const float w = exp2f(ps[DH] - M);
-        L = fmaf(ps[DH + 1], w, L);
+    for (int s0 = 0; s0 < ns; s0 += U) {
+        float mv[U], lv[U], ov[U][PER];
 #pragma unroll
-        for (int k = 0; k < PER; ++k) if (lane + 32 * k < DH) acc[k] = fmaf(ps[lane + 32 * k], w, acc[k]);
+        for (int u = 0; u < U; ++u) {
+            const bool on = s0 + u < ns;
+            const float* ps = part + (size_t)(on ? s0 + u : s0) * (DH + 2);
+            mv[u] = ps[DH]; lv[u] = ps[DH + 1];
+#pragma unroll
+            for (int k = 0; k < PER; ++k) ov[u][k] = lane + 32 * k < DH ? ps[lane + 32 * k] : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (s0 + u < ns) {
+                const float w = exp2f(mv[u] - M);
+                L = fmaf(lv[u], w, L);
+#pragma unroll
+                for (int k = 0; k < PER; ++k) if (lane + 32 * k < DH) acc[k] = fmaf(ov[u][k], w, acc[k]);
+            }
+        }
     }
     const float inv = 1.f / L;
 #pragma unroll

@@ -146,10 +146,11 @@ __global__ void __launch_bounds__(256) rope_kv_write_kernel(const float* __restr
     pdl_trigger();
     pdl_wait();
     const int row = blockIdx.x;
+    // the three descriptor loads go out together, then the page-table load: two memory latencies instead of four
     const int seq = rows.seq_id[row];
-    if (seq < 0) return;
     const int pos = rows.position[row];
     const int slot = rows.slot_of(row);
+    if (seq < 0) return;
     if (seq >= max_seqs || slot < 0 || slot >= rows.n_slots) { if (threadIdx.x == 0) atomicCAS(status, 0, kStatusSeq); return; }
     if (pos < 0 || pos >= max_position) { if (threadIdx.x == 0) atomicCAS(status, 0, kStatusPosition); return; }
     const int page = rows.page_table[((size_t)seq * rows.n_slots + slot) * rows.page_table_stride + pos / kPageSize];
