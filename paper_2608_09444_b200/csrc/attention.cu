@@ -95,8 +95,12 @@ __global__ void __launch_bounds__(1024) attn_plan_kernel(RowsDev rows, int32_t* 
     if (threadIdx.x == 0) item_start[rows.n_rows] = base;
 }
 
-template <typename T, int DH, int LPT, int CPL>
-__global__ void __maxnreg__(96) attn_split_kernel(AttnParams p) {
+// LAT: the variant for batches too small to fill the GPU, where a warp's own chain of memory latencies sets the
+// pace: the split's page ids come from one coalesced load, and the K/V tiles of the next page are in flight
+// while the current page is computed (twice the registers, which an almost empty GPU has to spare).  Same
+// arithmetic in the same order as the throughput variant.
+template <typename T, int DH, int LPT, int CPL, bool LAT>
+__global__ void __maxnreg__(LAT ? 208 : 96) attn_split_kernel(AttnParams p) {
     pdl_trigger();
     pdl_wait();
     constexpr int EPC = Chunk<T>::EPC;
@@ -149,20 +153,42 @@ __global__ void __maxnreg__(96) attn_split_kernel(AttnParams p) {
             for (int e = 0; e < EPC; ++e) o[j][e] = 0.f;
 
         const int page_lo = tok0 / kPageSize, page_hi = (tok1 - 1) / kPageSize;
-        for (int pi = page_lo; pi <= page_hi; ++pi) {
-            const int page = table[pi];
-            if (page < 0 || page >= p.pool.n_phys_pages) { if (lane == 0) atomicCAS(p.status, 0, kStatusPage); continue; }
+        static_assert(kSplitTokens / kPageSize <= 32, "a split's page ids must fit one warp");
+        int my_page = 0;
+        if constexpr (LAT) my_page = page_lo + lane <= page_hi ? table[page_lo + lane] : -1;
+        // starts the loads of one page's K and V tile; false (and a status word) when the page id is out of range
+        auto issue = [&](int pi, uint4 (&kd)[IPP][CPL], uint4 (&vd)[IPP][CPL]) -> bool {
+            const int page = LAT ? __shfl_sync(0xffffffffu, my_page, pi - page_lo) : table[pi];
+            if (page < 0 || page >= p.pool.n_phys_pages) { if (lane == 0) atomicCAS(p.status, 0, kStatusPage); return false; }
             const uint4* kt = (const uint4*)(pool_base + p.pool.tile_offset(p.layer, page, 0, head));
             const uint4* vt = (const uint4*)(pool_base + p.pool.tile_offset(p.layer, page, 1, head));
+#pragma unroll
+            for (int it = 0; it < IPP; ++it)
+#pragma unroll
+                for (int j = 0; j < CPL; ++j) kd[it][j] = ld_stream(kt + (it * TPI + g) * CPT + c + LPT * j);
+#pragma unroll
+            for (int it = 0; it < IPP; ++it)
+#pragma unroll
+                for (int j = 0; j < CPL; ++j) vd[it][j] = ld_stream(vt + (it * TPI + g) * CPT + c + LPT * j);
+            return true;
+        };
+        uint4 kn[LAT ? IPP : 1][LAT ? CPL : 1], vn[LAT ? IPP : 1][LAT ? CPL : 1];
+        bool next_ok = false;
+        if constexpr (LAT) next_ok = issue(page_lo, kn, vn);
+        for (int pi = page_lo; pi <= page_hi; ++pi) {
             uint4 kr[IPP][CPL], vr[IPP][CPL];
+            bool page_ok;
+            if constexpr (LAT) {
 #pragma unroll
-            for (int it = 0; it < IPP; ++it)
+                for (int it = 0; it < IPP; ++it)
 #pragma unroll
-                for (int j = 0; j < CPL; ++j) kr[it][j] = ld_stream(kt + (it * TPI + g) * CPT + c + LPT * j);
-#pragma unroll
-            for (int it = 0; it < IPP; ++it)
-#pragma unroll
-                for (int j = 0; j < CPL; ++j) vr[it][j] = ld_stream(vt + (it * TPI + g) * CPT + c + LPT * j);
+                    for (int j = 0; j < CPL; ++j) { kr[it][j] = kn[it][j]; vr[it][j] = vn[it][j]; }
+                page_ok = next_ok;
+                if (pi < page_hi) next_ok = issue(pi + 1, kn, vn);
+            } else {
+                page_ok = issue(pi, kr, vr);
+            }
+            if (!page_ok) continue;
 
             float s[IPP];
             const int tbase = pi * kPageSize + g;
@@ -290,15 +316,15 @@ void launch_attention_plan(const cdb* h, int ln, const RowsDev& rows, cudaStream
     launch_pdl(attn_plan_kernel, dim3(1), dim3(1024), 0, st, rows, h->lane[ln].attn_item_start, h->lane[ln].attn_counters, h->cfg.L_pre + h->cfg.L_core + h->cfg.L_coda);
 }
 
-template <typename T, int DH, int LPT, int CPL>
+template <typename T, int DH, int LPT, int CPL, bool LAT>
 static void launch_attention_t(const cdb* h, const AttnParams& p, void* o, cudaStream_t st) {
     static int blocks_per_sm = 0;
     if (blocks_per_sm == 0) {
         // The kernel uses no shared memory; asking for the largest shared-memory carve-out keeps the SM in the
         // configuration the projection kernel needs, so that its CTAs can become resident beside this one.
-        cudaFuncSetAttribute(attn_split_kernel<T, DH, LPT, CPL>, cudaFuncAttributePreferredSharedMemoryCarveout,
+        cudaFuncSetAttribute(attn_split_kernel<T, DH, LPT, CPL, LAT>, cudaFuncAttributePreferredSharedMemoryCarveout,
                              getenv("CDB_ATTN_CARVEOUT") ? atoi(getenv("CDB_ATTN_CARVEOUT")) : kAttnSharedCarveoutPct);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, attn_split_kernel<T, DH, LPT, CPL>, 128, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, attn_split_kernel<T, DH, LPT, CPL, LAT>, 128, 0);
         if (blocks_per_sm < 1) blocks_per_sm = 1;
     }
     int sms = 148;
@@ -319,7 +345,7 @@ static void launch_attention_t(const cdb* h, const AttnParams& p, void* o, cudaS
     {
         ProfScope ps(h, kProfAttention, st);
         CDB_LAUNCH(h);
-        launch_pdl(attn_split_kernel<T, DH, LPT, CPL>, dim3(grid), dim3(threads), 0, st, p);
+        launch_pdl(attn_split_kernel<T, DH, LPT, CPL, LAT>, dim3(grid), dim3(threads), 0, st, p);
     }
     if (h->attn_split_done) cudaEventRecord(h->attn_split_done, st);     // the KV stream is over: the merge is tiny
     CDB_LAUNCH(h);
@@ -335,15 +361,19 @@ void launch_attention(const cdb* h, int ln, int layer, const RowsDev& rows, cons
     p.max_seqs = h->cfg.max_seqs;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)h->cfg.Dh);
     p.part = h->lane[ln].attn_part; p.item_start = h->lane[ln].attn_item_start; p.counter = h->lane[ln].attn_counters + layer; p.status = h->status;
+    static const int force_lat = getenv("CDB_ATTN_LAT") ? atoi(getenv("CDB_ATTN_LAT")) : -1;      // tuning aid
+    // Few (row, head) pairs: the GPU is far from full whatever the contexts are, and a warp's own latency chain
+    // sets the pace (measured cross-over: ~64 rows of 16 heads; above it the throughput variant wins by 0-5 %).
+    const bool lat = force_lat >= 0 ? force_lat != 0 : p.rows.n_rows * p.pool.H <= 1024;
     const int Dh = h->cfg.Dh;
     if (h->cfg.dtype == CDB_BF16) {
-        if (Dh == 128) launch_attention_t<__nv_bfloat16, 128, 8, 2>(h, p, o, st);
-        else if (Dh == 96) launch_attention_t<__nv_bfloat16, 96, 4, 3>(h, p, o, st);
-        else launch_attention_t<__nv_bfloat16, 64, 8, 1>(h, p, o, st);
+        if (Dh == 128) { if (lat) launch_attention_t<__nv_bfloat16, 128, 8, 2, true>(h, p, o, st); else launch_attention_t<__nv_bfloat16, 128, 8, 2, false>(h, p, o, st); }
+        else if (Dh == 96) { if (lat) launch_attention_t<__nv_bfloat16, 96, 4, 3, true>(h, p, o, st); else launch_attention_t<__nv_bfloat16, 96, 4, 3, false>(h, p, o, st); }
+        else { if (lat) launch_attention_t<__nv_bfloat16, 64, 8, 1, true>(h, p, o, st); else launch_attention_t<__nv_bfloat16, 64, 8, 1, false>(h, p, o, st); }
     } else {
-        if (Dh == 128) launch_attention_t<float, 128, 8, 4>(h, p, o, st);
-        else if (Dh == 96) launch_attention_t<float, 96, 8, 3>(h, p, o, st);
-        else launch_attention_t<float, 64, 8, 2>(h, p, o, st);
+        if (Dh == 128) launch_attention_t<float, 128, 8, 4, false>(h, p, o, st);
+        else if (Dh == 96) launch_attention_t<float, 96, 8, 3, false>(h, p, o, st);
+        else launch_attention_t<float, 64, 8, 2, false>(h, p, o, st);
     }
 }
 
@@ -401,7 +431,7 @@ void launch_attention_static_t(const AttnParams& p, void* o, int max_context, cu
     const int max_items = p.rows.n_rows * p.pool.H * p.max_splits;
     int grid = 148 * 4;
     if ((max_items + 3) / 4 < grid) grid = (max_items + 3) / 4;
-    launch_pdl(attn_split_kernel<T, DH, LPT, CPL>, dim3(grid), dim3(128), 0, st, p);
+    launch_pdl(attn_split_kernel<T, DH, LPT, CPL, false>, dim3(grid), dim3(128), 0, st, p);
     const int warps = p.rows.n_rows * p.pool.H;
     launch_pdl(attn_merge_kernel<T, DH>, dim3((warps + 3) / 4), dim3(128), 0, st, p, (T*)o);
 }
