@@ -117,6 +117,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cdb", choices=["cdb", "reference"])
+    ap.add_argument("--model", default="ouro", choices=["ouro", "huginn"], help="layer shapes of the step (the headline metric is quoted on ouro)")
     ap.add_argument("--rows", type=int, default=256)
     ap.add_argument("--ctx-lo", type=int, default=128)
     ap.add_argument("--ctx-hi", type=int, default=2048)
@@ -140,8 +141,9 @@ def main():
         __graft_entry__.build()
     from paper_2608_09444_b200 import synth
 
-    dims = synth.OURO_1P4B if args.layers <= 0 else synth.OURO_1P4B.replace(L_core=args.layers)
-    workload = f"ouro-1.4b-shaped loop step, {args.rows} rows, depth U{{1..{dims.R}}}, context U{{{args.ctx_lo}..{args.ctx_hi}}}, 16-token pages"
+    base = synth.OURO_1P4B if args.model == "ouro" else synth.HUGINN_3P5B
+    dims = base if args.layers <= 0 else base.replace(L_core=args.layers)
+    workload = f"{'ouro-1.4b' if args.model == 'ouro' else 'huginn-3.5b'}-shaped loop step, {args.rows} rows, depth U{{1..{dims.R}}}, context U{{{args.ctx_lo}..{args.ctx_hi}}}, 16-token pages"
     config = {"workload": workload, "rows": args.rows, "core_layers": dims.L_core, "page_table": "contiguous" if args.contiguous_pages else "random permutation",
               "l2": "inputs larger than L2 (each step streams the whole KV pool and all core weights)"}
 
@@ -218,7 +220,7 @@ def main():
     # half-batch launches): bytes per launch = bytes of all launches / number of launches
     att_bytes_per_launch = alg["attention_per_launch"] * dims.L_core * args.steps / max(att["count"], 1)
     achieved = att_bytes_per_launch / (att_ms * 1e-3) / 1e9 if att_ms > 0 else 0.0
-    default_workload = args.rows == 256 and args.ctx_lo == 128 and args.ctx_hi == 2048 and not args.contiguous_pages
+    default_workload = args.model == "ouro" and args.rows == 256 and args.ctx_lo == 128 and args.ctx_hi == 2048 and not args.contiguous_pages
     out = {"metric": METRIC, "value": world * args.rows / (ms_step * 1e-3), "unit": "token-loop-steps/s",
            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",

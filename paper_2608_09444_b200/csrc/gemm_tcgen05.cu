@@ -657,12 +657,12 @@ static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* 
 }
 
 // Part count of a split-K projection.  It depends on the weight's shape alone, never on the number of rows,
-// so that a row's result does not depend on the batch it is computed in: about one tile per SM for a batch
+// so that a row's result does not depend on the batch it is computed in: at most one tile per SM for a batch
 // that fills one row tile, and at least four k-blocks per part.
 static int splitk_parts(int N, int K, int max_splits) {
     const int sms = device_sms();
     const int n_ft = (N + BM - 1) / BM, n_kb = (K + BK - 1) / BK;
-    int splits = (sms + n_ft / 2) / n_ft;
+    int splits = sms / n_ft;                      // rounded down: one tile too many per wave would cost a second wave
     if (splits > n_kb / 4) splits = n_kb / 4;
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
