@@ -24,6 +24,8 @@
  *    GEMM A-operands are of the configured dtype (fp32 or bf16); accumulation is fp32.
  *  - A row with seq_id < 0 is a pad: it computes nothing that is visible, writes no KV and
  *    appears in neither compaction list.
+ *  - Except in cdb_prefill, a call holds at most one row per sequence (the exit-gate state is kept per
+ *    sequence, and a row reads KV that only earlier calls wrote).
  *  - Scratch is per handle: two calls on the same handle must not overlap on the GPU, with one
  *    exception: a boundary call (cdb_boundary_embed / _prelude / _coda_lmhead) may run on another
  *    stream while cdb_loop_step / cdb_compact / cdb_gather_rows run, for rows of other sequences
