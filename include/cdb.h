@@ -74,7 +74,8 @@ typedef struct {
 } cdb_config_t;
 
 enum { CDB_FLAG_SIMT_GEMM = 1,         /* run bf16 projections on the plain-FMA kernel (cross-check) */
-       CDB_FLAG_TWO_STREAM = 2,        /* run a loop step of >= 64 rows as two half-batches on two streams (experimental) */
+       CDB_FLAG_TWO_STREAM = 2,        /* run a loop step of >= 64 rows as two half-batches on two streams (experimental; the second
+                                         * half uses the boundary calls' scratch, so no boundary call may overlap such a step) */
        CDB_FLAG_UNFUSED_LAYER = 4,     /* one launch per projection, separate norm and SwiGLU kernels (cross-check) */
        CDB_FLAG_SIMT_PREFILL = 8,      /* prompt attention of bf16 pools on the plain-FMA kernel instead of the tensor cores (cross-check) */
        CDB_FLAG_FUSED_STAGES = 16 };   /* everything of a layer after its attention as ONE cooperative launch with grid barriers between
