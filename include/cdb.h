@@ -26,10 +26,12 @@
  *    appears in neither compaction list.
  *  - Except in cdb_prefill, a call holds at most one row per sequence (the exit-gate state is kept per
  *    sequence, and a row reads KV that only earlier calls wrote).
- *  - Scratch is per handle: two calls on the same handle must not overlap on the GPU, with one
- *    exception: a boundary call (cdb_boundary_embed / _prelude / _coda_lmhead) may run on another
- *    stream while cdb_loop_step / cdb_compact / cdb_gather_rows run, for rows of other sequences
- *    (the coda and prelude of exited tokens overlap the next loop step, Fig. 3 of the paper).
+ *  - Scratch is per handle: two calls on the same handle must not overlap on the GPU, with two
+ *    exceptions, each for rows of sequences the other calls do not touch: a boundary call
+ *    (cdb_boundary_embed / _prelude / _coda_lmhead) may run on another stream while cdb_loop_step /
+ *    cdb_compact / cdb_gather_rows run (the coda and prelude of exited tokens overlap the next loop
+ *    step, Fig. 3 of the paper), and so may one cdb_prefill call on a third stream (prompts are
+ *    processed beside the running decode batch).  The three groups have scratch of their own.
  */
 #ifndef CDB_H
 #define CDB_H

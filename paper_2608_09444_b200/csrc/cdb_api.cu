@@ -15,6 +15,7 @@ using namespace cdbk;
 // boundary call on one stream may overlap a loop step on another (the two-stream half-batch mode also uses
 // lane 1 and must not be combined with that).
 constexpr int kBoundaryLane = 1;
+constexpr int kPrefillLane = 2;
 constexpr int kMinSplitRows = 64;          // below this a loop step runs as one batch on one stream
 constexpr int kSplitGemmSmemBytes = 0;            // no cap: a projection CTA co-resides with attention only when its ring is large
 constexpr int kSplitAttnCtasPerSm = 3;     // attention CTAs per SM when two half-batches share the GPU
@@ -208,7 +209,7 @@ void boundary_layers(cdb_t* h, int ln, int first, int last, const RowsDev& rows,
 // final RMSNorm + LM head + greedy argmax on n rows of x
 void lm_head(cdb_t* h, int ln, const RowsDev& rows, const float* x, int32_t* token_out, float* logits_out, cudaStream_t st) {
     const cdb_config_t& c = h->cfg;
-    float* logits = logits_out ? logits_out : h->logits;
+    float* logits = logits_out ? logits_out : h->logits + (size_t)ln * h->cfg.max_rows * h->cfg.V;
     launch_rmsnorm(h, x, h->g_final, h->lane[ln].xn, rows, st);
     launch_linear(h, h->lane[ln].xn, h->w.W_lm, logits, rows.n_rows, c.V, c.d, Epilogue::Store, st);
     launch_argmax(h, logits, rows.n_rows, token_out, st);
@@ -216,7 +217,7 @@ void lm_head(cdb_t* h, int ln, const RowsDev& rows, const float* x, int32_t* tok
 
 void free_all(cdb_t* h) {
     void* ptrs[] = {h->rope_cos, h->rope_sin, h->g_attn, h->g_mlp, h->g_final, h->gate_S, h->gate_fire,
-                    h->h_prev, h->h_work, h->logits, h->exit_flag, h->status, h->emit_tmp, h->grid_sync};
+                    h->h_prev, h->h_work, h->h_emit, h->logits, h->exit_flag, h->status, h->emit_tmp, h->grid_sync};
     for (void* p : ptrs) if (p) cudaFree(p);
     for (Lane& L : h->lane) {
         void* lp[] = {L.xn, L.qrot, L.attn_o, L.act, L.qkv, L.gu, L.ws, L.attn_part, L.attn_item_start, L.attn_counters, L.pf_tile_rows, L.pf_n_tiles};
@@ -291,7 +292,7 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
     CDB_ALLOC(h->g_final, float, d);
     CDB_ALLOC(h->gate_S, float, c.max_seqs);
     CDB_ALLOC(h->gate_fire, uint8_t, c.max_seqs);
-    for (int ln = 0; ln < 2; ++ln) {
+    for (int ln = 0; ln < 3; ++ln) {
         Lane& L = h->lane[ln];
         L.rows_cap = c.max_rows;
         const size_t r = L.rows_cap;
@@ -310,10 +311,11 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
     }
     CDB_ALLOC(h->h_prev, float, R_ * d);
     CDB_ALLOC(h->h_work, float, R_ * d);
-    CDB_ALLOC(h->logits, float, R_ * (size_t)c.V);
+    CDB_ALLOC(h->logits, float, 3 * R_ * (size_t)c.V);
+    CDB_ALLOC(h->h_emit, float, R_ * d);
     CDB_ALLOC(h->exit_flag, uint8_t, R_);
     CDB_ALLOC(h->status, int32_t, 1);
-    CDB_ALLOC(h->grid_sync, unsigned int, 2);
+    CDB_ALLOC(h->grid_sync, unsigned int, 3);
     CDB_ALLOC(h->emit_tmp, int32_t, R_);
 #undef CDB_ALLOC
     if (e != cudaSuccess) { free_all(h); delete h; cudaGetLastError(); return e == cudaErrorMemoryAllocation ? CDB_ERR_NOMEM : CDB_ERR_CUDA; }
@@ -352,8 +354,8 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
         gains_to_f32(h, w->g_final, h->g_final, d);
         init_gate_state_kernel<<<(c.max_seqs + 255) / 256, 256>>>(h->gate_S, h->gate_fire, c.max_seqs);
         cudaMemset(h->status, 0, sizeof(int32_t));
-        cudaMemset(h->grid_sync, 0, 2 * sizeof(unsigned int));
-        for (int ln = 0; ln < 2; ++ln) cudaMemset(h->lane[ln].attn_counters, 0, sizeof(int32_t) * L);
+        cudaMemset(h->grid_sync, 0, 3 * sizeof(unsigned int));
+        for (int ln = 0; ln < 3; ++ln) cudaMemset(h->lane[ln].attn_counters, 0, sizeof(int32_t) * L);
         if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess) h->side = nullptr;
         cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
         cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
@@ -532,23 +534,23 @@ int cdb_prefill(cdb_t* h, const int32_t* token_ids, const cdb_rows_t* rows, cons
     float* x = h->h_work;
     h->prefill_attention = 1;
     launch_embed(h, token_ids, rd, x, true, st);
-    launch_attention_plan(h, 0, rd, st);
+    launch_attention_plan(h, kPrefillLane, rd, st);
     rd.slot_override = 0;
-    for (int l = 0; l < c.L_pre; ++l) layer_forward(h, 0, l, rd, x, st);
+    for (int l = 0; l < c.L_pre; ++l) layer_forward(h, kPrefillLane, l, rd, x, st);
     for (int r = 1; r <= c.R; ++r) {
         rd.slot_override = slot_of_loop(c.kv_layout, r);
-        for (int l = c.L_pre; l < c.L_pre + c.L_core; ++l) layer_forward(h, 0, l, rd, x, st);
+        for (int l = c.L_pre; l < c.L_pre + c.L_core; ++l) layer_forward(h, kPrefillLane, l, rd, x, st);
     }
     rd.slot_override = 0;
-    for (int l = c.L_pre + c.L_core; l < c.L_pre + c.L_core + c.L_coda; ++l) layer_forward(h, 0, l, rd, x, st);
+    for (int l = c.L_pre + c.L_core; l < c.L_pre + c.L_core + c.L_coda; ++l) layer_forward(h, kPrefillLane, l, rd, x, st);
     h->prefill_attention = 0;
     if (n_emit > 0) {
-        // gather the emitting rows to the front of h_prev (free during prefill), then LM head on them
-        launch_gather(h, x, emit_idx, nullptr, n_emit, h->h_prev, st);
+        // gather the emitting rows, then LM head on them
+        launch_gather(h, x, emit_idx, nullptr, n_emit, h->h_emit, st);
         RowsDev re = rd;
         re.n_rows = n_emit;
         re.seq_id = nullptr;
-        lm_head(h, 0, re, h->h_prev, token_out, logits_out, st);
+        lm_head(h, kPrefillLane, re, h->h_emit, token_out, logits_out, st);
     }
     return check_launch(h, "cdb_prefill");
 }
@@ -593,7 +595,7 @@ int cdb_poll_status(cdb_t* h, int32_t* status_host) {
     cudaError_t e = cudaMemcpy(status_host, h->status, sizeof(int32_t), cudaMemcpyDeviceToHost);
     if (e == cudaSuccess && *status_host != 0) {                                                 // read and re-arm
         e = cudaMemset(h->status, 0, sizeof(int32_t));
-        cudaMemset(h->grid_sync, 0, 2 * sizeof(unsigned int));        // a barrier a timed-out kernel left half way
+        cudaMemset(h->grid_sync, 0, 3 * sizeof(unsigned int));        // a barrier a timed-out kernel left half way
     }
     return e == cudaSuccess ? CDB_OK : fail_cuda(h, e, "cdb_poll_status");
 }

@@ -89,15 +89,17 @@ struct cdb {
     TiledWeight tiled[6];           // W_qkv, W_o, W_gate, W_up, W_down, W_lm (bf16 configs)
     int n_tiled;
 
-    // per-lane scratch, max_rows rows each: lane 0 serves the loop step and prefill, lane 1 the boundary calls (so
-    // that they may overlap a loop step on another stream) and the second half-batch of a two-stream step
-    cdbk::Lane lane[2];
+    // per-lane scratch, max_rows rows each: lane 0 serves the loop step, lane 1 the boundary calls and the second
+    // half-batch of a two-stream step, lane 2 prompt processing - so that a boundary call and a prompt call may
+    // each overlap a loop step on streams of their own
+    cdbk::Lane lane[3];
     float* h_prev;                  // [max_rows][d] state at step entry (convergence gate)
     float* h_work;                  // [max_rows][d] prefill working state
-    float* logits;                  // [max_rows][V]
+    float* h_emit;                  // [max_rows][d] prefill: rows whose token is emitted
+    float* logits;                  // [3][max_rows][V], one per lane
     uint8_t* exit_flag;             // [max_rows]
     int32_t* status;                // [1] first out-of-range access seen (0 = clean)
-    unsigned int* grid_sync;        // [2] per lane: barrier word of the multi-stage layer kernel
+    unsigned int* grid_sync;        // [3] per lane: barrier word of the multi-stage layer kernel
     int32_t* emit_tmp;              // [max_rows]
     char err[256];
 
@@ -106,7 +108,7 @@ struct cdb {
     cudaEvent_t ev_fork, ev_join, ev_attn[2];
     mutable cudaEvent_t attn_split_done; // recorded right after the next attention split kernel when set
     mutable int attn_ctas_per_sm_cap;   // > 0 (two-stream step): attention runs one CTA of this many x 4 warps per SM
-    mutable int qkv_parts_ready[2];     // per lane: split-K parts of the next layer's QKV projection already in the workspace
+    mutable int qkv_parts_ready[3];     // per lane: split-K parts of the next layer's QKV projection already in the workspace
     mutable int prefill_attention;      // != 0 while cdb_prefill runs: layers use the query-tiled causal attention (1: tile list not planned yet)
     mutable int gemm_smem_cap;          // > 0 (two-stream step): projection kernels keep their shared-memory ring below this many bytes
 

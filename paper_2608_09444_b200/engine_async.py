@@ -27,13 +27,19 @@ from .engine import Engine, _bucket, _static_rows
 
 
 class PipelinedEngine(Engine):
-    def __init__(self, *a, **kw):
+    def __init__(self, *a, background_prefill=True, **kw):
         kw.setdefault("mode", "refill")
         kw.setdefault("lookahead", True)
         super().__init__(*a, **kw)
         if self.mode != "refill" or not self.lookahead:
             raise ValueError("the pipelined engine implements refill mode with the lookahead gate")
-        self.side = torch.cuda.Stream(device=self.dev)
+        # decode work (main and side stream) outranks prompt processing when both have kernels waiting for SMs
+        self.main = torch.cuda.Stream(device=self.dev, priority=-1)
+        self.side = torch.cuda.Stream(device=self.dev, priority=-1)
+        # prompts of newly admitted requests are processed on a stream of their own beside the running decode
+        # batch (the library gives prompt calls their own scratch); False = drain the pipeline and process them alone
+        self.background_prefill = background_prefill
+        self.pstream = torch.cuda.Stream(device=self.dev, priority=0)
         d = self.dims.d
         self.h_exit2 = [torch.zeros((self.max_rows, d), dtype=torch.float32, device=self.dev) for _ in range(2)]
         self.h_coda_in = torch.zeros((self.cap, d), dtype=torch.float32, device=self.dev)
@@ -77,6 +83,14 @@ class PipelinedEngine(Engine):
     def generate(self, prompts, T, forced_depths=None, teacher_tokens=None, arrivals=None):
         """Same contract as Engine.generate (teacher tokens are not supported: sampled tokens stay on the
         device and feed the prelude directly).  Gate values are not read back."""
+        caller = torch.cuda.current_stream(self.dev)
+        self.main.wait_stream(caller)
+        with torch.cuda.stream(self.main):
+            out = self._generate(prompts, T, forced_depths, teacher_tokens, arrivals)
+        caller.wait_stream(self.main)
+        return out
+
+    def _generate(self, prompts, T, forced_depths, teacher_tokens, arrivals):
         if teacher_tokens is not None:
             raise ValueError("lock-step replay needs the synchronous engine")
         dims, cdb, dev = self.dims, self.cdb, self.dev
@@ -96,6 +110,8 @@ class PipelinedEngine(Engine):
         ring = [torch.zeros((5, self.max_rows), dtype=torch.int32).pin_memory() for _ in range(4)]
         tok_ring = [torch.zeros(self.cap, dtype=torch.int32).pin_memory() for _ in range(16)]
         tok_dev = torch.zeros(self.cap, dtype=torch.int32, device=dev)
+        tokp_dev = torch.zeros(self.cap, dtype=torch.int32, device=dev)      # first tokens of a prompt call
+        tokp_host = torch.zeros(self.cap, dtype=torch.int32).pin_memory()
         counts_h = torch.zeros(2, dtype=torch.int32).pin_memory()
         surv_h = torch.zeros(self.max_rows, dtype=torch.int32).pin_memory()
         exit_h = torch.zeros(self.max_rows, dtype=torch.int32).pin_memory()
@@ -143,6 +159,61 @@ class PipelinedEngine(Engine):
             ev = torch.cuda.Event()
             ev.record(stream)
             ready.extend((s, slot, ev, it) for s, slot in zip(sids, slots))
+
+        prefill_inflight = []                           # at most one: (event, batch, pinned token buffer)
+
+        def admit_background():
+            """prompt processing of waiting requests on the prompt stream, beside the running decode batch"""
+            if prefill_inflight:
+                return
+            batch, rows_total = [], 0
+            while waiting and free_slots and rows_total + P[waiting[0]] <= self.max_rows:
+                s = waiting[0]
+                if not self._reserve_pages(free_slots[-1], P[s] + Ts[s]):
+                    break
+                live_slot[s] = free_slots.pop()
+                waiting.pop(0)
+                batch.append(s)
+                rows_total += P[s]
+            if not batch:
+                return
+            table_ready = torch.cuda.Event()
+            table_ready.record(main)                    # the page-table rows were updated on the main stream
+            toks = np.concatenate([np.asarray(prompts[s], dtype=np.int32) for s in batch])
+            sl = np.concatenate([np.full(P[s], live_slot[s]) for s in batch])
+            pos = np.concatenate([np.arange(P[s]) for s in batch])
+            ends = np.cumsum([P[s] for s in batch]) - 1
+            m = len(batch)
+            with torch.cuda.stream(self.pstream):
+                self.pstream.wait_event(table_ready)
+                cdb.prefill(i32(toks), B.Rows(i32(sl), i32(pos), self.page_table), i32(ends), tokp_dev[:m], stream=self.pstream)
+                tokp_host[:m].copy_(tokp_dev[:m], non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(self.pstream)
+            prefill_inflight.append((ev, batch))
+            self.stats["prefill_calls"] += 1
+
+        def poll_prefill(block):
+            """first tokens of a finished prompt call: record them, start the prelude of the sequences that go on"""
+            if not prefill_inflight or not (block or prefill_inflight[0][0].query()):
+                return
+            ev, batch = prefill_inflight.pop(0)
+            ev.synchronize()
+            vals = tokp_host[:len(batch)].numpy().copy()
+            cont = []
+            for j, s in enumerate(batch):
+                tokens[s][0] = int(vals[j])
+                gen[s] = 1
+                self.stats["first_token_s"][s] = now()
+                if gen[s] >= Ts[s]:
+                    self.stats["finish_s"][s] = now()
+                    self._release_pages(live_slot[s])
+                    free_slots.append(live_slot.pop(s))
+                else:
+                    cont.append(j)
+            if cont:                                     # boundary calls share one scratch lane: all of them on the side stream
+                with torch.cuda.stream(side):
+                    enqueue_prelude([batch[j] for j in cont], i32(vals[cont]), side, it)
 
         def admit():
             """prompt processing of waiting requests while live slots and pages are free (drains the pipeline)"""
@@ -234,10 +305,14 @@ class PipelinedEngine(Engine):
                 t_now = now()
                 while future and arrivals[future[0]] <= t_now:
                     waiting.append(future.pop(0))
+            poll_prefill(False)
             if waiting and free_slots and (arrivals is None or len(waiting) >= self.admit_min or not live_slot
                                            or now() - arrivals[waiting[0]] >= self.admit_wait_s):
-                admit()
-            if "decode_start" not in self.stats and not waiting and not future:
+                if self.background_prefill:
+                    admit_background()
+                else:
+                    admit()
+            if "decode_start" not in self.stats and not waiting and not future and not prefill_inflight:
                 torch.cuda.synchronize(dev)
                 self.stats["decode_start"] = time.perf_counter()
             # ---- refills whose prelude was enqueued in an earlier iteration join this step
@@ -304,6 +379,9 @@ class PipelinedEngine(Engine):
                 prev = {"parity": parity, "ne": ne, "exits": exits, "G": G}
                 rec = [[rec[int(i)][0], rec[int(i)][1] + 1] for i in surv]
             it += 1
+            if not rec and prev is None and not ready and not coda_q and prefill_inflight:
+                poll_prefill(True)                      # nothing else to run: wait for the prompt call
+                continue
             if not rec and prev is None and not ready and not coda_q and not waiting:
                 if future and not pending_tokens and not pending_release:
                     time.sleep(min(1e-3, max(0.0, arrivals[future[0]] - now())))

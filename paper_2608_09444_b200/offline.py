@@ -31,9 +31,10 @@ def run(dims, weights, prompts, T, *, mode, gate_kind, q_or_eps=0.5, forced_dept
     n, P = len(prompts), max(len(p) for p in prompts)
     live = min(n, max_live or n)
     pages = live * ((P + T + dims.page_size - 1) // dims.page_size)
+    kw = {"background_prefill": False} if pipelined else {}     # offline: prompts first, then the timed decode phase
     eng = (PipelinedEngine if pipelined else Engine)(dims, weights, max_batch=min(max_batch or n, live), max_live=live, max_len=P + T, n_pages=pages, gate_kind=gate_kind,
                  q_or_eps=q_or_eps, lookahead=True, mode=mode, min_coda_batch=min_coda_batch,
-                 max_prefill_rows=max_prefill_rows, record_ticks=False, use_graphs=use_graphs, time_device=time_device)
+                 max_prefill_rows=max_prefill_rows, record_ticks=False, use_graphs=use_graphs, time_device=time_device, **kw)
     res = eng.generate(prompts, T, forced_depths=forced_depths)
     st = eng.stats
     depths = np.concatenate(res["depths"])

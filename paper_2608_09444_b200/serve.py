@@ -125,14 +125,19 @@ def main():
         for mode in args.modes.split(","):
             pipelined = mode.endswith("_pipelined")
             m = mode.replace("_pipelined", "")
+            fixed = m == "cb" and pipelined                  # continuous batching on the pipelined engine: every token replays depth R
+            if fixed:
+                m = "refill"
             if world > 1:
                 torch.distributed.barrier()           # the replicas start their clocks together
             out, _ = run(dims, w, arrivals[mine], [prompts[i] for i in mine], [out_lens[i] for i in mine], mode=m,
-                         pipelined=pipelined, gate_kind=gate_kind,
-                         forced_depths=None if (m == "cb" or forced is None) else [forced[i] for i in mine],
+                         pipelined=pipelined, gate_kind=B.GATE_NONE if fixed else gate_kind,
+                         forced_depths=[[dims.R] * max(out_lens[i] - 1, 1) for i in mine] if fixed else
+                         None if (m == "cb" or forced is None) else [forced[i] for i in mine],
                          max_batch=args.max_batch, max_live=args.max_live,
                          pool_tokens=args.pool_tokens, min_coda_batch=1 if args.model == "ouro" else 32,
                          admit_min=args.admit_min, admit_wait_s=args.admit_wait_ms * 1e-3, device=f"cuda:{local_rank}")
+            out["mode"] = mode
             parts = D.gather_objects({"ids": mine, "finish_s": out.pop("finish_s"), "first_token_s": out.pop("first_token_s"),
                                       "counters": {k: out[k] for k in ("recurrent_steps", "row_steps", "prefill_calls", "coda_calls")}})
             if rank == 0:
