@@ -96,7 +96,7 @@ def main():
     ap.add_argument("--max-batch", type=int, default=256)
     ap.add_argument("--max-live", type=int, default=320)
     ap.add_argument("--pool-tokens", type=int, default=400000)
-    ap.add_argument("--modes", default="cb,refill_pipelined")
+    ap.add_argument("--modes", default="cb_pipelined,refill_pipelined", help="cb, refill, no_refill (synchronous engine); cb_pipelined, refill_pipelined")
     ap.add_argument("--admit-min", type=int, default=1, help="hold arrived requests until this many wait ...")
     ap.add_argument("--admit-wait-ms", type=float, default=0.0, help="... or the oldest has waited this long")
     args = ap.parse_args()
