@@ -97,6 +97,7 @@ def main():
     ap.add_argument("--max-live", type=int, default=320)
     ap.add_argument("--pool-tokens", type=int, default=400000)
     ap.add_argument("--modes", default="cb_pipelined,refill_pipelined", help="cb, refill, no_refill (synchronous engine); cb_pipelined, refill_pipelined")
+    ap.add_argument("--min-coda-batch", type=int, default=0, help="exits gathered before a coda call (0: 1 for ouro, 8 for huginn; the offline runs use 32 for huginn)")
     ap.add_argument("--admit-min", type=int, default=1, help="hold arrived requests until this many wait ...")
     ap.add_argument("--admit-wait-ms", type=float, default=0.0, help="... or the oldest has waited this long")
     args = ap.parse_args()
@@ -135,7 +136,7 @@ def main():
                          forced_depths=[[dims.R] * max(out_lens[i] - 1, 1) for i in mine] if fixed else
                          None if (m == "cb" or forced is None) else [forced[i] for i in mine],
                          max_batch=args.max_batch, max_live=args.max_live,
-                         pool_tokens=args.pool_tokens, min_coda_batch=1 if args.model == "ouro" else 32,
+                         pool_tokens=args.pool_tokens, min_coda_batch=args.min_coda_batch or (1 if args.model == "ouro" else 8),
                          admit_min=args.admit_min, admit_wait_s=args.admit_wait_ms * 1e-3, device=f"cuda:{local_rank}")
             out["mode"] = mode
             parts = D.gather_objects({"ids": mine, "finish_s": out.pop("finish_s"), "first_token_s": out.pop("first_token_s"),
