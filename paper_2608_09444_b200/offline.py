@@ -31,7 +31,8 @@ def run(dims, weights, prompts, T, *, mode, gate_kind, q_or_eps=0.5, forced_dept
     n, P = len(prompts), max(len(p) for p in prompts)
     live = min(n, max_live or n)
     pages = live * ((P + T + dims.page_size - 1) // dims.page_size)
-    kw = {"background_prefill": False} if pipelined else {}     # offline: prompts first, then the timed decode phase
+    # all sequences live: prompts first, then the timed decode phase; a queue of waiting sequences: prompts overlap decode
+    kw = {"background_prefill": live < n} if pipelined else {}
     eng = (PipelinedEngine if pipelined else Engine)(dims, weights, max_batch=min(max_batch or n, live), max_live=live, max_len=P + T, n_pages=pages, gate_kind=gate_kind,
                  q_or_eps=q_or_eps, lookahead=True, mode=mode, min_coda_batch=min_coda_batch,
                  max_prefill_rows=max_prefill_rows, record_ticks=False, use_graphs=use_graphs, time_device=time_device, **kw)
@@ -99,7 +100,7 @@ def main():
     ap.add_argument("--max-batch", type=int, default=0)
     ap.add_argument("--min-coda-batch", type=int, default=0)
     ap.add_argument("--max-live", type=int, default=0, help="sequences resident at once (0 = all); fewer than --seqs queues the rest")
-    ap.add_argument("--modes", default="cb,refill,no_refill", help="cb, refill, no_refill, refill_pipelined, refill_nographs")
+    ap.add_argument("--modes", default="cb,refill,no_refill", help="cb, refill, no_refill, refill_nographs (synchronous engine); cb_pipelined, refill_pipelined")
     ap.add_argument("--exits", default="forced", choices=["forced", "criterion"],
                     help="huginn: replayed geometric exit depths, or the convergence criterion with a calibrated threshold")
     ap.add_argument("--time-device", action="store_true", help="bracket every GPU phase with CUDA events and report device_ms")
@@ -134,12 +135,19 @@ def main():
     for mode in args.modes.split(","):
         pipelined = mode.endswith("_pipelined")
         nographs = mode.endswith("_nographs")
+        name = mode
         mode = mode.replace("_pipelined", "").replace("_nographs", "")
-        out, _ = run(dims, w, prompts, args.tokens, mode=mode, pipelined=pipelined, use_graphs=not nographs, time_device=args.time_device, gate_kind=gate_kind, q_or_eps=q_or_eps, forced_depths=None if mode == "cb" else forced,
+        fixed = mode == "cb" and pipelined              # continuous batching on the pipelined engine: every token replays depth R
+        out, _ = run(dims, w, prompts, args.tokens, mode="refill" if fixed else mode, pipelined=pipelined, use_graphs=not nographs,
+                     time_device=args.time_device, gate_kind=B.GATE_NONE if fixed else gate_kind, q_or_eps=q_or_eps,
+                     forced_depths=[[dims.R] * (args.tokens - 1)] * args.seqs if fixed else None if mode == "cb" else forced,
                      max_batch=args.max_batch or None, max_live=args.max_live or None, min_coda_batch=min_coda)
+        out["mode"] = name
         report["runs"].append(out)
         print(json.dumps(out), flush=True)
     by = {r["mode"]: r for r in report["runs"]}
+    if "cb" not in by and "cb_pipelined" in by:
+        by["cb"] = by["cb_pipelined"]
     if "cb" in by:
         for m in ("refill", "no_refill", "refill_pipelined"):
             if m in by:
