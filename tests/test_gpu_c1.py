@@ -226,3 +226,20 @@ def test_graph_buckets_first_used_mid_run_leave_waiting_rows_alone():
         for s in range(n):
             assert np.array_equal(runs[0]["tokens"][s], other["tokens"][s]), s
             assert np.array_equal(runs[0]["depths"][s], other["depths"][s]), s
+
+
+def test_c1_fixed_depth_on_the_pipelined_engine_equals_continuous_batching(oracle_runs):
+    """Standard continuous batching (every token loops R times) expressed on the pipelined engine as replayed
+    exit depths of R, the like-for-like baseline of the serving and batch-64 runs: the oracle's fixed-depth tokens."""
+    from paper_2608_09444_b200 import binding as B
+    from paper_2608_09444_b200.engine_async import PipelinedEngine
+    dims, w, prompts = c1_inputs()
+    wd = {k: v.cuda() for k, v in w.items()}
+    eng = PipelinedEngine(dims, wd, max_batch=4, max_live=6, max_len=48, n_pages=18, gate_kind=B.GATE_NONE, q_or_eps=0.5,
+                          max_prefill_rows=256)
+    res = eng.generate(list(prompts), 16, forced_depths=[[dims.R] * 15] * 8)
+    assert eng.cdb.poll_status() == 0
+    ref = oracle_runs["fixed"]
+    for s in range(8):
+        assert np.array_equal(res["tokens"][s], ref[s]["tokens"]), s
+        assert np.all(res["depths"][s] == dims.R)
