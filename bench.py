@@ -231,7 +231,7 @@ def main():
            "roofline": {"kernel": "attn_split_kernel (paged decode attention)", "bound": "hbm", "achieved": achieved,
                         "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                         "traffic": NCU_TRAFFIC_PER_ALGORITHMIC_BYTE * att_bytes_per_launch if default_workload else None,
-                        "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of this kernel on the same rows with one core layer (profiles/attn_split_kernel_ouro_1layer_256rows.md): 2.3371 GB per launch for 2.3133 GB algorithmic",
+                        "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of this kernel on the same rows with one core layer (summary kept under profiles/): 2.3371 GB per launch for 2.3133 GB algorithmic",
                         "launches": att["count"], "avg_launch_ms": att_ms,
                         "algorithmic_bytes_per_launch": att_bytes_per_launch},
            "kernel_time_ms_per_step": {"attention": att["ms"] / args.steps, "projections": prof["linear"]["ms"] / args.steps},
