@@ -27,20 +27,23 @@ def flop_bound(dims, mean_depth):
 
 
 def run(dims, weights, prompts, T, *, mode, gate_kind, q_or_eps=0.5, forced_depths=None, max_batch=None, max_live=None,
-        min_coda_batch=1, max_prefill_rows=4096, pipelined=False, use_graphs=True, time_device=False):
+        min_coda_batch=1, max_prefill_rows=4096, pipelined=False, use_graphs=True, time_device=False, kv_layout=B.KV_SHARED):
     n, P = len(prompts), max(len(p) for p in prompts)
     live = min(n, max_live or n)
-    pages = live * ((P + T + dims.page_size - 1) // dims.page_size)
+    n_slots = {B.KV_SHARED: 1, B.KV_DEPTH_INDEXED: dims.R, B.KV_FIRST_THEN_SHARED: 2}[kv_layout]
+    pages = live * n_slots * ((P + T + dims.page_size - 1) // dims.page_size)
     # all sequences live: prompts first, then the timed decode phase; a queue of waiting sequences: prompts overlap decode
     kw = {"background_prefill": live < n} if pipelined else {}
-    eng = (PipelinedEngine if pipelined else Engine)(dims, weights, max_batch=min(max_batch or n, live), max_live=live, max_len=P + T, n_pages=pages, gate_kind=gate_kind,
+    eng = (PipelinedEngine if pipelined else Engine)(dims, weights, max_batch=min(max_batch or n, live), max_live=live, max_len=P + T, n_pages=pages, gate_kind=gate_kind, kv_layout=kv_layout,
                  q_or_eps=q_or_eps, lookahead=True, mode=mode, min_coda_batch=min_coda_batch,
                  max_prefill_rows=max_prefill_rows, record_ticks=False, use_graphs=use_graphs, time_device=time_device, **kw)
     res = eng.generate(prompts, T, forced_depths=forced_depths)
     st = eng.stats
     depths = np.concatenate(res["depths"])
     decode_s = st["end"] - st["decode_start"]
-    out = {"mode": mode + ("_pipelined" if pipelined else "") + ("" if use_graphs else "_nographs"), "max_batch": eng.max_batch, "max_live": live, "total_s": st["end"] - st["start"],
+    from .engine import kv_footprint
+    out = {"kv_layout": kv_layout, "kv_kib_per_token_in_use": kv_footprint(dims, n_slots)[0] / 1024,
+           "mode": mode + ("_pipelined" if pipelined else "") + ("" if use_graphs else "_nographs"), "max_batch": eng.max_batch, "max_live": live, "total_s": st["end"] - st["start"],
            "generated_tokens_per_s_end_to_end": sum(len(t) for t in res["tokens"]) / (st["end"] - st["start"]),
            "decode_s": decode_s, "prefill_s": st["decode_start"] - st["start"],
            "decode_tokens_per_s": len(depths) / decode_s, "token_loop_steps_per_s": st["row_steps"] / decode_s,
@@ -101,6 +104,8 @@ def main():
     ap.add_argument("--min-coda-batch", type=int, default=0)
     ap.add_argument("--max-live", type=int, default=0, help="sequences resident at once (0 = all); fewer than --seqs queues the rest")
     ap.add_argument("--modes", default="cb,refill,no_refill", help="cb, refill, no_refill, refill_nographs (synchronous engine); cb_pipelined, refill_pipelined")
+    ap.add_argument("--kv-layout", default="shared", choices=["shared", "depth_indexed", "first_then_shared"],
+                    help="depth_indexed = last-exited cache (copy-on-exit), section 4.2")
     ap.add_argument("--exits", default="forced", choices=["forced", "criterion"],
                     help="huginn: replayed geometric exit depths, or the convergence criterion with a calibrated threshold")
     ap.add_argument("--time-device", action="store_true", help="bracket every GPU phase with CUDA events and report device_ms")
@@ -141,7 +146,8 @@ def main():
         out, _ = run(dims, w, prompts, args.tokens, mode="refill" if fixed else mode, pipelined=pipelined, use_graphs=not nographs,
                      time_device=args.time_device, gate_kind=B.GATE_NONE if fixed else gate_kind, q_or_eps=q_or_eps,
                      forced_depths=[[dims.R] * (args.tokens - 1)] * args.seqs if fixed else None if mode == "cb" else forced,
-                     max_batch=args.max_batch or None, max_live=args.max_live or None, min_coda_batch=min_coda)
+                     max_batch=args.max_batch or None, max_live=args.max_live or None, min_coda_batch=min_coda,
+                     kv_layout={"shared": B.KV_SHARED, "depth_indexed": B.KV_DEPTH_INDEXED, "first_then_shared": B.KV_FIRST_THEN_SHARED}[args.kv_layout])
         out["mode"] = name
         report["runs"].append(out)
         print(json.dumps(out), flush=True)
