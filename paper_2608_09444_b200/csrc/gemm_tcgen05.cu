@@ -44,7 +44,6 @@ struct GemmParams {
     int stages;
     int mode;
     int k_splits;               // the K range is cut into this many parts, each a tile of its own
-    int wide;                   // store / accumulate: a tile is 256 features (two weight tiles and accumulators share the x tile)
     int w_tiled;                // weights come from the tile-major copy: tile (ft, kb) starts at row (ft * n_kb + kb) * 128
     size_t split_stride;
     uint32_t stage_out_off;     // SwiGLU mode: byte offset (from the ring base) of a [BN][128] bf16 output staging tile
@@ -70,19 +69,16 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
                                            const GemmParams& p, const CtaCtx& cx, WaitInputs wait_inputs) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int S = p.stages, BN = p.BN;
-    const bool swiglu = p.mode == kModeSwiGLU;
-    const bool dual = swiglu || p.wide;                                      // two weight tiles, two accumulators
+    const bool dual = p.mode == kModeSwiGLU;                                 // two weight tiles, two accumulators
     const uint32_t w_bytes = BM * BK * 2, x_bytes = (uint32_t)BN * BK * 2;
     const uint32_t x_off = dual ? 2 * w_bytes : w_bytes, stage_bytes = x_off + x_bytes;
     const uint32_t acc_cols = dual ? 2u * BN : (uint32_t)BN;                 // TMEM columns of one accumulator set
-    const int n_acc = 2u * acc_cols <= 512u ? 2 : 1;                         // accumulator sets that fit TMEM
-    const int FT = p.wide ? 2 * BM : BM;                                     // features per tile
     const uint32_t ring = cx.ring, bar0 = cx.bar0;
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (8 + s); };
     auto acc_full_bar = [&](int a) { return bar0 + 8u * (16 + a); };
     auto acc_empty_bar = [&](int a) { return bar0 + 8u * (18 + a); };
-    const int n_ftiles = (p.N + FT - 1) / FT, n_rtiles = (p.n + BN - 1) / BN;
+    const int n_ftiles = (p.N + BM - 1) / BM, n_rtiles = (p.n + BN - 1) / BN;
     const int n_tiles = n_ftiles * n_rtiles * p.k_splits;                   // tile t = (split, row tile, feature tile)
     const int n_kb = (p.K + BK - 1) / BK;
     auto kb_begin = [&](int t) { return (int)((long long)(t / (n_ftiles * n_rtiles)) * n_kb / p.k_splits); };
@@ -102,12 +98,10 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
                 if (pass == 1) wait_inputs();
                 int g = 0;                                   // position in this CTA's (tile, k-block) sequence
                 for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-                    const int f0 = (t % n_ftiles) * FT, r0 = (t / n_ftiles % n_rtiles) * BN;
+                    const int f0 = (t % n_ftiles) * BM, r0 = (t / n_ftiles % n_rtiles) * BN;
                     // Every CTA walks its k-blocks from a different starting point (a function of its feature
                     // tile only), so that the CTAs do not all pull the same activation lines from L2 at once.
-                    // (the starting point is shared by a pair of neighbouring 128-feature tiles, so that a
-                    // 256-feature tile sums every feature's k-blocks in the same order as two narrow tiles do)
-                    const int kb0 = kb_begin(t), nk = kb_end(t) - kb0, rot = (((f0 / BM) >> 1) * 7) % nk;
+                    const int kb0 = kb_begin(t), nk = kb_end(t) - kb0, rot = ((t % n_ftiles) * 7) % nk;
                     if (pass == 0 && g >= S) break;
                     for (int j = 0; j < nk; ++j, ++g) {
                         if (pass == 0 && g >= S) break;
@@ -167,8 +161,8 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
             bool ok = true;
             const long long mma_t0 = clock64();
             for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
-                const int acc = it % n_acc;
-                const uint32_t acc_ph = (uint32_t)(it / n_acc) & 1u;
+                const int acc = it & 1;
+                const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
                 if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, cx.abortp)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = cx.tmem_base + (uint32_t)acc * acc_cols;
@@ -200,9 +194,9 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
         int it = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
-            const int acc = it % n_acc;
-            const uint32_t acc_ph = (uint32_t)(it / n_acc) & 1u;
-            const int r0 = (t / n_ftiles % n_rtiles) * BN;
+            const int acc = it & 1;
+            const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
+            const int f = (t % n_ftiles) * BM + q * 32 + lane, r0 = (t / n_ftiles % n_rtiles) * BN;
             const int split = t / (n_ftiles * n_rtiles);
             if (!mbar_wait(acc_full_bar(acc), acc_ph, cx.abortp)) { ok = false; break; }
             if (p.dbg && it == 0 && warp == 2 && lane == 0) p.dbg[blockIdx.x * 8 + 4] = gtime();
@@ -210,7 +204,7 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
             const uint32_t t_addr = cx.tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * acc_cols;
             // 16 columns (= 16 batch rows) of this thread's feature per pass: a small register footprint
             const int n_cols = min(BN, p.n - r0);               // columns holding real rows (warp-uniform)
-            if (swiglu) {
+            if (dual) {
                 // gate and up accumulators side by side; loads of the next 16 columns fly while these are finished
                 uint32_t v[2][16], u[2][16];
                 tmem_ld16(t_addr, v[0]);
@@ -261,12 +255,9 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");              // staging tile free for the next tile
             } else {
-              for (int half = 0; half < (p.wide ? 2 : 1); ++half) {       // a 256-feature tile: one accumulator after the other
-                const int f = (t % n_ftiles) * FT + half * BM + q * 32 + lane;
-                const uint32_t h_addr = t_addr + (uint32_t)(half * BN);
                 // software pipeline: the TMEM load of the next 16 columns is in flight while these are stored
                 uint32_t v[2][16];
-                tmem_ld16(h_addr, v[0]);
+                tmem_ld16(t_addr, v[0]);
 #pragma unroll 1
                 for (int c0 = 0; c0 < n_cols; c0 += 32) {
 #pragma unroll
@@ -274,7 +265,7 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
                         const int c = c0 + 16 * hh;
                         if (c >= n_cols) break;
                         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                        if (c + 16 < n_cols) tmem_ld16(h_addr + (uint32_t)(c + 16), v[hh ^ 1]);
+                        if (c + 16 < n_cols) tmem_ld16(t_addr + (uint32_t)(c + 16), v[hh ^ 1]);
                         if (f < p.N) {
                             float* dst = p.y + (size_t)split * p.split_stride + (size_t)(r0 + c) * p.N + f;
                             if (p.mode == kModeAccumulate) {
@@ -293,7 +284,6 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
                     }
                 }
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-              }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
@@ -314,9 +304,11 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
-    const int warp = threadIdx.x >> 5;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int S = p.stages, BN = p.BN;
-    const bool dual = p.mode == kModeSwiGLU || p.wide;                       // two weight tiles, two accumulators
+    const bool dual = p.mode == kModeSwiGLU;                                 // two weight tiles, two accumulators
+    const uint32_t w_bytes = BM * BK * 2, x_bytes = (uint32_t)BN * BK * 2;
+    const uint32_t x_off = dual ? 2 * w_bytes : w_bytes, stage_bytes = x_off + x_bytes;
     const uint32_t acc_cols = dual ? 2u * BN : (uint32_t)BN;                 // TMEM columns of one accumulator set
     const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;            // swizzled tiles need 1024-byte alignment
     const uint32_t bar0 = smem_u32(bars);
@@ -324,7 +316,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
     auto empty_bar = [&](int s) { return bar0 + 8u * (8 + s); };
     auto acc_full_bar = [&](int a) { return bar0 + 8u * (16 + a); };
     auto acc_empty_bar = [&](int a) { return bar0 + 8u * (18 + a); };
-    const uint32_t tmem_cols = 2u * acc_cols <= 512u ? 2u * acc_cols : 512u;   // double-buffered when two sets fit; 128, 256 or 512
+    const uint32_t tmem_cols = 2u * acc_cols;                               // double-buffered; 128, 256 or 512
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -617,15 +609,7 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
         while (p.BN > 64 && tiles(p.BN) * 2 < sms && n > p.BN / 2) p.BN /= 2;
     }
     if ((forced_bn == 64 || forced_bn == 128 || forced_bn == 256) && forced_bn <= bn_max) p.BN = forced_bn;
-    // Long reductions on many rows (prompt processing): 256 features per tile, i.e. two weight tiles and two
-    // accumulators per x tile - a third less traffic through the SM's L2 port per flop; the accumulators then
-    // fill TMEM, so the epilogue no longer overlaps the next tile, which only pays when the main loop is long.
-    const int n_kb_ = (K + BK - 1) / BK;
-    p.wide = (mode != kModeSwiGLU && k_splits == 1 && n >= 512 && n_kb_ >= 64 && find_tiled(h, W, N, K) &&
-              ((n_ft + 1) / 2) * ((n + 255) / 256) >= 2 * device_sms() &&          // still at least two waves of tiles
-              !getenv("CDB_GEMM_NARROW")) ? 1 : 0;
-    if (p.wide) p.BN = 256;
-    const int stage_bytes = (mode == kModeSwiGLU || p.wide ? 2 : 1) * BM * BK * 2 + p.BN * BK * 2;
+    const int stage_bytes = (mode == kModeSwiGLU ? 2 : 1) * BM * BK * 2 + p.BN * BK * 2;
     static const int smem_cap = getenv("CDB_GEMM_SMEM_KB") ? atoi(getenv("CDB_GEMM_SMEM_KB")) * 1024 : kMaxSmem;   // tuning aid
     int budget = smem_cap < kMaxSmem ? smem_cap : kMaxSmem;
     if (h->gemm_smem_cap > 0 && h->gemm_smem_cap < budget) budget = h->gemm_smem_cap;
@@ -640,18 +624,14 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
     const void* Wt = find_tiled(h, W, N, K);
     const void* Wt2 = W2 ? find_tiled(h, W2, N, K) : Wt;
     p.w_tiled = (Wt && Wt2) ? 1 : 0;
-    if (p.wide) {
-        // second weight tile of a pair = the next feature tile: the same coordinates in a map that starts one tile later
-        const char* Wt_next = (const char*)Wt + (size_t)n_kb * BM * BK * 2;
-        if (!make_map(map_w, Wt, n_ft * n_kb * BM, BK, BM) || !make_map(map_w2, Wt_next, (n_ft - 1) * n_kb * BM, BK, BM)) return 0;
-    } else if (p.w_tiled) {
+    if (p.w_tiled) {
         if (!make_map(map_w, Wt, n_ft * n_kb * BM, BK, BM) || !make_map(map_w2, Wt2, n_ft * n_kb * BM, BK, BM)) return 0;
     } else {
         if (!make_map(map_w, W, N, K, BM) || !make_map(map_w2, W2 ? W2 : W, N, K, BM)) return 0;
     }
     if (!make_map(map_x, x, n, K, p.BN)) return 0;
     *smem = (size_t)p.stages * stage_bytes + stage_out + 1024;
-    return (p.wide ? (n_ft + 1) / 2 : n_ft) * ((n + p.BN - 1) / p.BN) * k_splits;
+    return n_ft * ((n + p.BN - 1) / p.BN) * k_splits;
 }
 
 static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* W2, float* y, __nv_bfloat16* act, int n,
