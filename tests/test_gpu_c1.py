@@ -243,3 +243,24 @@ def test_c1_fixed_depth_on_the_pipelined_engine_equals_continuous_batching(oracl
     for s in range(8):
         assert np.array_equal(res["tokens"][s], ref[s]["tokens"]), s
         assert np.all(res["depths"][s] == dims.R)
+
+
+@pytest.mark.parametrize("pipelined", [False, True])
+def test_c1_kv_pool_smaller_than_the_live_set(oracle_runs, pipelined):
+    """Eight live slots but pages for only four sequences: admission has to wait for finished sequences to hand
+    their pages back ("prefill up to a KV-cache limit", section 4.1); everything still completes with the oracle's
+    tokens and every page returns to the free list."""
+    from paper_2608_09444_b200 import binding as B
+    from paper_2608_09444_b200.engine import Engine
+    from paper_2608_09444_b200.engine_async import PipelinedEngine
+    dims, w, prompts = c1_inputs()
+    wd = {k: v.cuda() for k, v in w.items()}
+    eng = (PipelinedEngine if pipelined else Engine)(dims, wd, max_batch=8, max_live=8, max_len=48, n_pages=12,
+                                                      gate_kind=B.GATE_SIGMOID_CDF, q_or_eps=0.5, max_prefill_rows=256)
+    res = eng.generate(list(prompts), 16)
+    assert eng.cdb.poll_status() == 0
+    ref = oracle_runs["adaptive"]
+    for s in range(8):
+        assert np.array_equal(res["tokens"][s], ref[s]["tokens"]), s
+        assert np.array_equal(res["depths"][s], ref[s]["depths"]), s
+    assert len(eng.free_pages) == 12 and not [p for row in eng.page_table_host for p in row if p >= 0]
