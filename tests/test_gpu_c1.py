@@ -264,3 +264,41 @@ def test_c1_kv_pool_smaller_than_the_live_set(oracle_runs, pipelined):
         assert np.array_equal(res["tokens"][s], ref[s]["tokens"]), s
         assert np.array_equal(res["depths"][s], ref[s]["depths"]), s
     assert len(eng.free_pages) == 12 and not [p for row in eng.page_table_host for p in row if p >= 0]
+
+
+def test_c1_convergence_criterion_end_to_end():
+    """The training-free exit rule of appendix C.2 (L2 distance between consecutive recurrent states below a
+    threshold, first comparison at loop 2, applied one step ahead: no exit below depth 3) through both engines
+    against the oracle.  The threshold is picked by the oracle in a gap of its own distances, so that no decision
+    sits within 1e-4 (relative) of it."""
+    from paper_2608_09444_b200 import binding as B
+    from paper_2608_09444_b200.engine import Engine
+    from paper_2608_09444_b200.engine_async import PipelinedEngine
+    dims, w, prompts = c1_inputs()
+    wn = synth.weights_to_numpy(w)
+    prompts = list(prompts)[:4]
+    T = 10
+    probe = O.Oracle(dims, wn, gate_kind=O.GATE_L2_CONVERGENCE, q_or_eps=0.0, lookahead=True)
+    dist = np.sort(np.concatenate([np.asarray(p["gate"][1:]) for pr in prompts[:2] for p in probe.generate(pr, T)["passes"]]))
+    ref = eps = None
+    for q in (0.5, 0.35, 0.65, 0.2, 0.8):
+        i = int(q * (len(dist) - 1))
+        cand = 0.5 * (dist[i] + dist[i + 1])
+        orc = O.Oracle(dims, wn, gate_kind=O.GATE_L2_CONVERGENCE, q_or_eps=float(cand), lookahead=True)
+        runs = [orc.generate(pr, T) for pr in prompts]
+        gates = np.concatenate([np.asarray(p["gate"][1:]) for r in runs for p in r["passes"]])
+        depths = np.concatenate([r["depths"] for r in runs])
+        if np.min(np.abs(gates - cand)) > 1e-4 * cand and len(set(depths.tolist())) >= 2:
+            ref, eps = runs, float(cand)
+            break
+    assert ref is not None, "no threshold with a clear margin found"
+    assert min(int(r["depths"].min()) for r in ref) >= 3
+    wd = {k: v.cuda() for k, v in w.items()}
+    for cls in (Engine, PipelinedEngine):
+        eng = cls(dims, wd, max_batch=3, max_live=4, max_len=48, n_pages=12, gate_kind=B.GATE_L2_CONVERGENCE, q_or_eps=eps,
+                  max_prefill_rows=256)
+        res = eng.generate(prompts, T)
+        assert eng.cdb.poll_status() == 0
+        for s in range(len(prompts)):
+            assert np.array_equal(res["tokens"][s], ref[s]["tokens"]), (cls.__name__, s)
+            assert np.array_equal(res["depths"][s], ref[s]["depths"]), (cls.__name__, s)
