@@ -302,3 +302,27 @@ def test_c1_convergence_criterion_end_to_end():
         for s in range(len(prompts)):
             assert np.array_equal(res["tokens"][s], ref[s]["tokens"]), (cls.__name__, s)
             assert np.array_equal(res["depths"][s], ref[s]["depths"]), (cls.__name__, s)
+
+
+@pytest.mark.parametrize("pipelined", [False, True])
+def test_c1_minimum_coda_batch_changes_timing_not_tokens(oracle_runs, pipelined):
+    """Exited tokens wait until three of them can share a coda call (section 4.1: a heavier coda is worth
+    batching); when nothing else can run the queue is flushed.  Same tokens and depths as the oracle, fewer calls."""
+    from paper_2608_09444_b200 import binding as B
+    from paper_2608_09444_b200.engine import Engine
+    from paper_2608_09444_b200.engine_async import PipelinedEngine
+    dims, w, prompts = c1_inputs()
+    wd = {k: v.cuda() for k, v in w.items()}
+    calls = {}
+    for mcb in (1, 3):
+        eng = (PipelinedEngine if pipelined else Engine)(dims, wd, max_batch=6, max_live=8, max_len=48, n_pages=24,
+                                                          gate_kind=B.GATE_SIGMOID_CDF, q_or_eps=0.5, max_prefill_rows=256,
+                                                          min_coda_batch=mcb)
+        res = eng.generate(list(prompts), 16)
+        assert eng.cdb.poll_status() == 0
+        ref = oracle_runs["adaptive"]
+        for s in range(8):
+            assert np.array_equal(res["tokens"][s], ref[s]["tokens"]), (mcb, s)
+            assert np.array_equal(res["depths"][s], ref[s]["depths"]), (mcb, s)
+        calls[mcb] = eng.stats["coda_calls"]
+    assert calls[3] < calls[1]
