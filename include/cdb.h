@@ -221,6 +221,11 @@ int cdb_paged_attention_static(const void* q, void* o, const void* pool, int32_t
                                int32_t page_table_stride, int32_t n_rows, int32_t max_seqs, int32_t max_context,
                                int32_t H, int32_t Dh, int32_t dtype, void* stream);
 
+/* Debug aid: every scratch buffer of the handle lies between two 256-byte guard words that no kernel of the
+ * library may touch.  Synchronises the device's default stream order (plain cudaMemcpy) and counts the buffers
+ * whose guards were overwritten (0 = clean). */
+int cdb_debug_check_guards(cdb_t* h, int32_t* n_clobbered);
+
 /* Synchronises the stream-less status word back to the host: 0 = clean, otherwise the first
  * out-of-range page id (1) / position (2) / sequence id (3) a kernel met since the last poll (the
  * access was skipped), or 4 when a bounded wait inside a tensor-core kernel ran out.  A non-zero

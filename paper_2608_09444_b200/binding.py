@@ -30,7 +30,7 @@ FLAG_FUSED_STAGES = 16
 EXPORTS = ["cdb_create", "cdb_destroy", "cdb_last_error", "cdb_kv_bind", "cdb_set_gate", "cdb_boundary_embed",
            "cdb_boundary_prelude", "cdb_loop_step", "cdb_compact", "cdb_gather_rows", "cdb_boundary_coda_lmhead",
            "cdb_prefill", "cdb_kv_copy_on_exit", "cdb_paged_attention", "cdb_linear", "cdb_poll_status",
-           "cdb_profile_begin", "cdb_profile_read", "cdb_paged_attention_static"]
+           "cdb_profile_begin", "cdb_profile_read", "cdb_paged_attention_static", "cdb_debug_check_guards"]
 
 
 class Config(C.Structure):
@@ -226,6 +226,12 @@ class Cdb:
     def poll_status(self) -> int:
         v = C.c_int32(0)
         self._check(lib.cdb_poll_status(self.h, C.byref(v)))
+        return v.value
+
+    def check_guards(self) -> int:
+        """Number of library scratch buffers whose guard words were overwritten (0 = clean)."""
+        v = C.c_int32(0)
+        self._check(lib.cdb_debug_check_guards(self.h, C.byref(v)))
         return v.value
 
     def profile_begin(self, record_events: bool = True):

@@ -38,9 +38,22 @@ int check_launch(cdb_t* h, const char* where) {
     return e == cudaSuccess ? CDB_OK : fail_cuda(h, e, where);
 }
 
-template <typename T> cudaError_t dev_alloc(T** p, size_t count) {
+// Every scratch buffer sits between two guard words of kGuardBytes filled with a pattern; nothing the library
+// launches may write them (cdb_debug_check_guards).  A stand-in for a memory checker on the library's own buffers.
+constexpr size_t kGuardBytes = 256;
+constexpr int kGuardPattern = 0xA5;
+
+template <typename T> cudaError_t dev_alloc(cdb_t* h, T** p, size_t count) {
     *p = nullptr;
-    return cudaMalloc((void**)p, (count ? count : 1) * sizeof(T));
+    const size_t bytes = ((count ? count : 1) * sizeof(T) + 15) / 16 * 16;
+    char* base = nullptr;
+    cudaError_t e = cudaMalloc((void**)&base, bytes + 2 * kGuardBytes);
+    if (e != cudaSuccess) return e;
+    cudaMemset(base, kGuardPattern, kGuardBytes);
+    cudaMemset(base + kGuardBytes + bytes, kGuardPattern, kGuardBytes);
+    if (h->n_allocs < cdb::kMaxAllocs) { h->alloc_base[h->n_allocs] = base; h->alloc_bytes[h->n_allocs] = bytes; ++h->n_allocs; }
+    *p = (T*)(base + kGuardBytes);
+    return cudaSuccess;
 }
 
 int slot_of_loop(int layout, int r) {
@@ -216,13 +229,8 @@ void lm_head(cdb_t* h, int ln, const RowsDev& rows, const float* x, int32_t* tok
 }
 
 void free_all(cdb_t* h) {
-    void* ptrs[] = {h->rope_cos, h->rope_sin, h->g_attn, h->g_mlp, h->g_final, h->gate_S, h->gate_fire,
-                    h->h_prev, h->h_work, h->h_emit, h->logits, h->exit_flag, h->status, h->emit_tmp, h->grid_sync};
-    for (void* p : ptrs) if (p) cudaFree(p);
-    for (Lane& L : h->lane) {
-        void* lp[] = {L.xn, L.qrot, L.attn_o, L.act, L.qkv, L.gu, L.ws, L.attn_part, L.attn_item_start, L.attn_counters, L.pf_tile_rows, L.pf_n_tiles};
-        for (void* p : lp) if (p) cudaFree(p);
-    }
+    for (int i = 0; i < h->n_allocs; ++i) cudaFree(h->alloc_base[i]);     // every scratch buffer (with its guards)
+    h->n_allocs = 0;
     for (int i = 0; i < h->n_tiled; ++i) if (h->tiled[i].tiled) cudaFree(h->tiled[i].tiled);
     h->n_tiled = 0;
     if (h->side) cudaStreamDestroy(h->side);
@@ -284,7 +292,7 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
     const size_t wide = d > F ? d : F;
     const int n_layers = L;
     cudaError_t e = cudaSuccess;
-#define CDB_ALLOC(ptr, type, count) if (e == cudaSuccess) e = dev_alloc<type>((type**)&(ptr), (count))
+#define CDB_ALLOC(ptr, type, count) if (e == cudaSuccess) e = dev_alloc<type>(h, (type**)&(ptr), (count))
     CDB_ALLOC(h->rope_cos, float, (size_t)c.max_position * half);
     CDB_ALLOC(h->rope_sin, float, (size_t)c.max_position * half);
     CDB_ALLOC(h->g_attn, float, (size_t)L * d);
@@ -598,6 +606,21 @@ int cdb_poll_status(cdb_t* h, int32_t* status_host) {
         cudaMemset(h->grid_sync, 0, 3 * sizeof(unsigned int));        // a barrier a timed-out kernel left half way
     }
     return e == cudaSuccess ? CDB_OK : fail_cuda(h, e, "cdb_poll_status");
+}
+
+int cdb_debug_check_guards(cdb_t* h, int32_t* n_clobbered) {
+    if (!h || !n_clobbered) return CDB_ERR_ARG;
+    *n_clobbered = 0;
+    unsigned char host[2 * kGuardBytes];
+    for (int i = 0; i < h->n_allocs; ++i) {
+        cudaError_t e = cudaMemcpy(host, h->alloc_base[i], kGuardBytes, cudaMemcpyDeviceToHost);
+        if (e == cudaSuccess) e = cudaMemcpy(host + kGuardBytes, h->alloc_base[i] + kGuardBytes + h->alloc_bytes[i], kGuardBytes, cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) return fail_cuda(h, e, "cdb_debug_check_guards");
+        bool bad = false;
+        for (size_t k = 0; k < 2 * kGuardBytes; ++k) bad |= host[k] != (unsigned char)kGuardPattern;
+        *n_clobbered += bad ? 1 : 0;
+    }
+    return CDB_OK;
 }
 
 int cdb_profile_begin(cdb_t* h, int32_t record_events) {

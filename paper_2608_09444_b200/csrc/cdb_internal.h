@@ -102,6 +102,11 @@ struct cdb {
     unsigned int* grid_sync;        // [3] per lane: barrier word of the multi-stage layer kernel
     int32_t* emit_tmp;              // [max_rows]
     char err[256];
+    // every cudaMalloc of the handle: base pointers (guard word, buffer, guard word) and buffer sizes
+    static constexpr int kMaxAllocs = 96;
+    char* alloc_base[kMaxAllocs];
+    size_t alloc_bytes[kMaxAllocs];
+    int n_allocs;
 
     // two-stream execution of a loop step: second half-batch on `side`, joined by events
     cudaStream_t side;

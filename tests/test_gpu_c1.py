@@ -68,6 +68,7 @@ def compare(eng, res, ref):
             if res["gates"][s][j]:
                 worst_gate = max(worst_gate, float(np.max(np.abs(np.asarray(res["gates"][s][j]) - np.asarray(p["gate"])))))
     assert worst_state <= TOL and worst_logit <= TOL and worst_gate <= TOL, (worst_state, worst_logit, worst_gate)
+    assert eng.cdb.check_guards() == 0                            # no kernel wrote outside its scratch buffer
 
 
 def test_c1_refill_matches_oracle(oracle_runs):

@@ -41,6 +41,7 @@ def test_c2_full_size_step_matches_oracle_on_sampled_rows():
     wl.step_resident()
     torch.cuda.synchronize()
     assert wl.cdb.poll_status() == 0
+    assert wl.cdb.check_guards() == 0                 # full-size step: nothing wrote outside its scratch buffer
 
     # ---- integer outputs of all rows
     want_s, want_e = O.stable_partition(list(flags), [True] * 256)

@@ -170,3 +170,4 @@ def test_prefill_matches_oracle(H, Dh, dtype, lens, simt):
         page, off = table_np[i, (len(pr) - 1) // 16], (len(pr) - 1) % 16
         got = pool[l, page, 0, :, off, :].float().cpu().numpy()
         assert rel_err(got, cache[l][0][0][len(pr) - 1]) <= tol
+    assert cdb.check_guards() == 0

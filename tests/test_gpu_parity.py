@@ -265,6 +265,7 @@ def test_loop_step_rows_match_oracle(dims, gate_kind, flags):
         mask[:, table_np[i, (ctxs[i] - 1) // 16], :, :, (ctxs[i] - 1) % 16, :] = False
     assert np.array_equal(got_pool[mask], pool_np[mask])
     assert near <= 1
+    assert cdb.check_guards() == 0                                # no kernel wrote outside its scratch buffer
 
 
 def test_two_stream_half_batches_equal_the_single_stream_step():
