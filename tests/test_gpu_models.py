@@ -171,3 +171,43 @@ def test_prefill_matches_oracle(H, Dh, dtype, lens, simt):
         got = pool[l, page, 0, :, off, :].float().cpu().numpy()
         assert rel_err(got, cache[l][0][0][len(pr) - 1]) <= tol
     assert cdb.check_guards() == 0
+
+
+@pytest.mark.parametrize("layout", ["depth_indexed", "first_then_shared"])
+def test_prefill_and_decode_with_depth_slots_bf16(layout):
+    """bf16 prompt processing (tensor-core attention) and a few decode tokens under the depth-aware KV layouts:
+    every loop of the prompt writes its own slot, decode reads slot r-1 (or min(r,2)-1) and copy-on-exit fills
+    the skipped slots.  Logits of the prompt and the K the last core layer holds in every slot against the oracle."""
+    from paper_2608_09444_b200 import binding as B
+    dims = synth.Dims(V=300, d=256, H=2, Dh=128, F=192, L_pre=1, L_core=2, L_coda=1, R=3, dtype="bf16")
+    w = synth.make_weights(dims, 8, std=0.05, gain_jitter=0.1)
+    wn = synth.weights_to_numpy(w)
+    o_layout = {"depth_indexed": O.DEPTH_INDEXED, "first_then_shared": O.FIRST_THEN_SHARED}[layout]
+    b_layout = {"depth_indexed": B.KV_DEPTH_INDEXED, "first_then_shared": B.KV_FIRST_THEN_SHARED}[layout]
+    n_slots = O.n_slots(o_layout, dims.R)
+    lens = [150, 40]
+    prompts = [synth.make_prompts(1, n, dims.V, 50 + i)[0] for i, n in enumerate(lens)]
+    per = (max(lens) + 15) // 16
+    table_np = np.arange(len(lens) * n_slots * per, dtype=np.int32).reshape(len(lens) * n_slots, per)
+    cdb = B.Cdb(dims, {k: v.cuda() for k, v in w.items()}, max_rows=sum(lens), max_seqs=len(lens), max_position=per * 16,
+                gate_kind=B.GATE_NONE, kv_layout=b_layout)
+    pool = torch.full(synth.kv_pool_shape(dims, table_np.size), float("nan"), dtype=torch.bfloat16, device="cuda")
+    cdb.kv_bind(pool)
+    seq = np.concatenate([np.full(m, i) for i, m in enumerate(lens)])
+    pos = np.concatenate([np.arange(m) for m in lens])
+    rows = B.Rows(i32(seq), i32(pos), i32(table_np))
+    token, logits = torch.zeros(len(lens), dtype=torch.int32, device="cuda"), torch.zeros((len(lens), dims.V), device="cuda")
+    cdb.prefill(i32(np.concatenate(prompts)), rows, i32(np.cumsum(lens) - 1), token, logits)
+    torch.cuda.synchronize()
+    assert cdb.poll_status() == 0 and cdb.check_guards() == 0
+    orc = O.Oracle(dims, wn, kv_layout=o_layout, gate_kind=O.GATE_NONE)
+    l = dims.L_pre + dims.L_core - 1
+    for i, pr in enumerate(prompts):
+        cache = orc.new_cache(len(pr))
+        ref = orc.prefill(pr, cache)
+        assert rel_err(logits[i].cpu().numpy(), ref) <= TOL, (i, rel_err(logits[i].cpu().numpy(), ref))
+        t = len(pr) - 1
+        for slot in range(n_slots):
+            page = table_np[i * n_slots + slot, t // 16]
+            got = pool[l, page, 0, :, t % 16, :].float().cpu().numpy()
+            assert rel_err(got, cache[l][slot][0][t]) <= TOL, (i, slot)
