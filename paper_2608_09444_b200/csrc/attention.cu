@@ -323,21 +323,18 @@ static void launch_attention_t(const cdb* h, const AttnParams& p, void* o, cudaS
         // The kernel uses no shared memory; asking for the largest shared-memory carve-out keeps the SM in the
         // configuration the projection kernel needs, so that its CTAs can become resident beside this one.
         cudaFuncSetAttribute(attn_split_kernel<T, DH, LPT, CPL, LAT>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                             getenv("CDB_ATTN_CARVEOUT") ? atoi(getenv("CDB_ATTN_CARVEOUT")) : kAttnSharedCarveoutPct);
+                             tuning_int("CDB_ATTN_CARVEOUT", kAttnSharedCarveoutPct));
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, attn_split_kernel<T, DH, LPT, CPL, LAT>, 128, 0);
         if (blocks_per_sm < 1) blocks_per_sm = 1;
     }
-    int sms = 148;
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = h->sms;
     const int max_items = p.rows.n_rows * p.pool.H * p.max_splits;
     // Warps are independent, so the CTA shape only decides how the block scheduler packs the SMs.
     // Alone: CTAs of 4 warps, as many as fit.  Sharing the GPU with the other half-batch's kernels: one
     // CTA of 4 * cap warps per SM, which leaves registers free on EVERY SM for a projection CTA
     // (small CTAs may be packed unevenly and fill some SMs completely).
     int grid = sms * blocks_per_sm, threads = 128;
-    static const int forced_cap = getenv("CDB_ATTN_CAP") ? atoi(getenv("CDB_ATTN_CAP")) : 0;                  // tuning aid
+    static const int forced_cap = tuning_int("CDB_ATTN_CAP", 0);      // tuning hook
     const int cap = forced_cap > 0 ? forced_cap : h->attn_ctas_per_sm_cap;
     if (cap > 0 && cap < blocks_per_sm) { grid = sms; threads = 128 * cap; }
     const int warps_per_cta = threads / 32;
@@ -361,7 +358,7 @@ void launch_attention(const cdb* h, int ln, int layer, const RowsDev& rows, cons
     p.max_seqs = h->cfg.max_seqs;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)h->cfg.Dh);
     p.part = h->lane[ln].attn_part; p.item_start = h->lane[ln].attn_item_start; p.counter = h->lane[ln].attn_counters + layer; p.status = h->status;
-    static const int force_lat = getenv("CDB_ATTN_LAT") ? atoi(getenv("CDB_ATTN_LAT")) : -1;      // tuning aid
+    static const int force_lat = tuning_int("CDB_ATTN_LAT", -1);      // tuning hook
     // Few (row, head) pairs: the GPU is far from full whatever the contexts are, and a warp's own latency chain
     // sets the pace (measured cross-over: ~64 rows of 16 heads; above it the throughput variant wins by 0-5 %).
     const bool lat = force_lat >= 0 ? force_lat != 0 : p.rows.n_rows * p.pool.H <= 1024;

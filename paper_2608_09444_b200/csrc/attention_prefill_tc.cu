@@ -360,9 +360,7 @@ bool launch_attention_prefill_tc(const cdb* h, int ln, int layer, const RowsDev&
     p.out = (__nv_bfloat16*)o; p.status = h->status;
     const int nch = (Dh + 63) / 64;
     const size_t smem = 1024 + (size_t)(5 * nch + 2) * kChunkBytes;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = h->sms;
     const long long max_items = (long long)rows.n_rows * H;            // at least one row per tile
     const int grid = (int)(max_items < sms ? max_items : sms);
     auto kern = Dh == 128 ? attn_prefill_tc_kernel<128> : Dh == 96 ? attn_prefill_tc_kernel<96> : attn_prefill_tc_kernel<64>;

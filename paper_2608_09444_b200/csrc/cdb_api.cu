@@ -286,6 +286,14 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
     h->w = *w;
     h->elem_size = c.dtype == CDB_FP32 ? 4 : 2;
     h->max_splits = (c.max_position + kSplitTokens - 1) / kSplitTokens;
+    {
+        int dev = 0;
+        h->sms = 148;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || h->sms < 1) {
+            delete h;
+            return CDB_ERR_CUDA;
+        }
+    }
     h->pool.H = c.H;
     h->pool.Dh = c.Dh;
     const size_t R_ = c.max_rows, d = c.d, F = c.F, half = c.Dh / 2;
@@ -644,7 +652,8 @@ int cdb_profile_read(cdb_t* h, cdb_profile_t* out) {
     if (e != cudaSuccess) return fail_cuda(h, e, "cdb_profile_read");
     memset(out, 0, sizeof(*out));
     out->launches = h->launches;
-    if (const char* path = getenv("CDB_PROF_DUMP")) {           // tuning aid: (class, start, end) of every bracketed launch
+#ifdef CDB_TUNING
+    if (const char* path = getenv("CDB_PROF_DUMP")) {           // tuning hook: (class, start, end) of every bracketed launch
         if (FILE* f = fopen(path, "w")) {
             for (int i = 0; i < h->prof_used; ++i) {
                 float a = 0.f, b = 0.f;
@@ -655,6 +664,7 @@ int cdb_profile_read(cdb_t* h, cdb_profile_t* out) {
             fclose(f);
         }
     }
+#endif
     for (int i = 0; i < h->prof_used; ++i) {
         float ms = 0.f;
         if (cudaEventElapsedTime(&ms, h->prof_ev[2 * i], h->prof_ev[2 * i + 1]) != cudaSuccess) continue;

@@ -16,6 +16,16 @@ constexpr int kMaxKSplits = 8;       // most split-K parts of a projection
 constexpr int kWsPerRow = 12;        // workspace floats per row, in units of d: 8 parts of [d] or 3 parts of [3d] fit
 constexpr int kStatusPage = 1, kStatusPosition = 2, kStatusSeq = 3;
 
+// Tuning hooks: a build made with -DCDB_TUNING reads integer overrides from the environment (once per
+// site); the shipped library has none and every hook folds to its default.
+#ifdef CDB_TUNING
+inline int tuning_int(const char* name, int dflt) { const char* v = getenv(name); return v ? atoi(v) : dflt; }
+constexpr bool kTuningBuild = true;
+#else
+constexpr int tuning_int(const char*, int dflt) { return dflt; }
+constexpr bool kTuningBuild = false;
+#endif
+
 enum class Epilogue : int { Store = 0, ResidualAdd = 1 };
 
 // Device view of a row descriptor plus the KV pool, passed by value to kernels.
@@ -76,6 +86,7 @@ struct cdb {
     cdb_weights_t w;
     cdbk::KvPool pool;
     size_t elem_size;               // bytes of the configured dtype
+    int sms;                        // multiprocessors of the device the handle was created on
     int max_splits;                 // ceil(max_position / kSplitTokens)
 
     // library-owned device memory
@@ -142,9 +153,9 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    static const bool no_pdl = getenv("CDB_NO_PDL") != nullptr;      // tuning aid: plain stream-ordered launches
+    static const bool no_pdl = tuning_int("CDB_NO_PDL", 0) != 0;     // tuning hook: plain stream-ordered launches
     cfg.attrs = attr; cfg.numAttrs = no_pdl ? 0 : 1;
-    static const int carve = getenv("CDB_MISC_CARVEOUT") ? atoi(getenv("CDB_MISC_CARVEOUT")) : -2;   // tuning aid
+    static const int carve = tuning_int("CDB_MISC_CARVEOUT", -2);    // tuning hook
     if (carve > -2) cudaFuncSetAttribute((const void*)kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve);
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }

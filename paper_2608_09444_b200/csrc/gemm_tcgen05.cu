@@ -48,7 +48,7 @@ struct GemmParams {
     size_t split_stride;
     uint32_t stage_out_off;     // SwiGLU mode: byte offset (from the ring base) of a [BN][128] bf16 output staging tile
     int32_t* status;
-    unsigned long long* dbg;    // tuning aid: per-CTA phase time stamps (NULL = off)
+    unsigned long long* dbg;    // tuning builds: per-CTA phase time stamps (NULL = off)
 };
 
 __device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t) :: "memory"); return t; }
@@ -186,7 +186,7 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
                 }
                 if (ok && leader) umma_commit(acc_full_bar(acc));     // accumulator complete
             }
-            if (p.dbg && leader) p.dbg[blockIdx.x * 8 + 2] = clock64() - mma_t0;
+            if (kTuningBuild && p.dbg && leader) p.dbg[blockIdx.x * 8 + 2] = clock64() - mma_t0;
         }
         __syncwarp();
     } else {
@@ -199,7 +199,7 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
             const int f = (t % n_ftiles) * BM + q * 32 + lane, r0 = (t / n_ftiles % n_rtiles) * BN;
             const int split = t / (n_ftiles * n_rtiles);
             if (!mbar_wait(acc_full_bar(acc), acc_ph, cx.abortp)) { ok = false; break; }
-            if (p.dbg && it == 0 && warp == 2 && lane == 0) p.dbg[blockIdx.x * 8 + 4] = gtime();
+            if (kTuningBuild && p.dbg && it == 0 && warp == 2 && lane == 0) p.dbg[blockIdx.x * 8 + 4] = gtime();
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t t_addr = cx.tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * acc_cols;
             // 16 columns (= 16 batch rows) of this thread's feature per pass: a small register footprint
@@ -287,7 +287,7 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
-            if (p.dbg && warp == 2 && lane == 0) p.dbg[blockIdx.x * 8 + 6] = gtime();
+            if (kTuningBuild && p.dbg && warp == 2 && lane == 0) p.dbg[blockIdx.x * 8 + 6] = gtime();
             if (lane == 0) mbar_arrive(acc_empty_bar(acc));
         }
     }
@@ -298,18 +298,15 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w2,
                          const __grid_constant__ CUtensorMap map_x, GemmParams p) {
     pdl_trigger();
-    if (p.dbg && threadIdx.x == 0) p.dbg[blockIdx.x * 8 + 0] = gtime();
+    if (kTuningBuild && p.dbg && threadIdx.x == 0) p.dbg[blockIdx.x * 8 + 0] = gtime();
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2 * 8 + 4];          // full[stages], empty[stages], acc_full[2], acc_empty[2]
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int S = p.stages, BN = p.BN;
-    const bool dual = p.mode == kModeSwiGLU;                                 // two weight tiles, two accumulators
-    const uint32_t w_bytes = BM * BK * 2, x_bytes = (uint32_t)BN * BK * 2;
-    const uint32_t x_off = dual ? 2 * w_bytes : w_bytes, stage_bytes = x_off + x_bytes;
-    const uint32_t acc_cols = dual ? 2u * BN : (uint32_t)BN;                 // TMEM columns of one accumulator set
+    const int warp = threadIdx.x >> 5;
+    const int S = p.stages;
+    const uint32_t acc_cols = p.mode == kModeSwiGLU ? 2u * p.BN : (uint32_t)p.BN;   // TMEM columns of one accumulator set (two accumulators for gate/up)
     const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;            // swizzled tiles need 1024-byte alignment
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
@@ -333,7 +330,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_slot;
     volatile int* abortp = &abort_flag;
-    if (p.dbg && threadIdx.x == 0) p.dbg[blockIdx.x * 8 + 1] = gtime();
+    if (kTuningBuild && p.dbg && threadIdx.x == 0) p.dbg[blockIdx.x * 8 + 1] = gtime();
     // Set-up above overlaps the previous kernel's tail.  The weights do not depend on that kernel, so the
     // producer warp starts their copies before it waits (below); every other warp waits here.
     if (warp != 0) pdl_wait();
@@ -581,13 +578,6 @@ void launch_repack_tiled(const void* W, void* Wt, int layers, int N, int K, cuda
     repack_tiled_kernel<<<148 * 8, 256, 0, st>>>((const __nv_bfloat16*)W, (__nv_bfloat16*)Wt, layers, N, K);
 }
 
-static int device_sms() {
-    int sms = 148, dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    return sms;
-}
-
 // Parameters and tensor maps of one projection.  W2 / act only in SwiGLU mode.  k_splits > 1 only with
 // kModeStore (y = workspace).  Returns the number of tiles, 0 on failure.
 static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2, float* y, __nv_bfloat16* act, int n,
@@ -595,7 +585,7 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
                       CUtensorMap* map_w2, CUtensorMap* map_x, size_t* smem) {
     p.y = y; p.act = act; p.n = n; p.N = N; p.K = K; p.mode = mode; p.k_splits = k_splits; p.split_stride = split_stride;
     const int n_ft = (N + BM - 1) / BM;
-    static const int forced_bn = getenv("CDB_GEMM_BN") ? atoi(getenv("CDB_GEMM_BN")) : 0;     // tuning aid
+    static const int forced_bn = tuning_int("CDB_GEMM_BN", 0);       // tuning hook
     const int bn_max = mode == kModeSwiGLU ? 128 : 256;
     // Rows per tile (MMA N): the widest of 64 / 128 / 256 the batch can fill: one tcgen05.mma then does the
     // most work per issue and each weight tile is pulled through L2 the fewest times.
@@ -604,13 +594,13 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
     // prompt processing): narrower row tiles then give more CTAs a share of the weight stream.  The tile
     // width changes which CTA computes an output element, never how it is summed.
     {
-        const int sms = device_sms();
+        const int sms = h->sms;
         auto tiles = [&](int bn) { return n_ft * ((n + bn - 1) / bn) * k_splits; };
         while (p.BN > 64 && tiles(p.BN) * 2 < sms && n > p.BN / 2) p.BN /= 2;
     }
     if ((forced_bn == 64 || forced_bn == 128 || forced_bn == 256) && forced_bn <= bn_max) p.BN = forced_bn;
     const int stage_bytes = (mode == kModeSwiGLU ? 2 : 1) * BM * BK * 2 + p.BN * BK * 2;
-    static const int smem_cap = getenv("CDB_GEMM_SMEM_KB") ? atoi(getenv("CDB_GEMM_SMEM_KB")) * 1024 : kMaxSmem;   // tuning aid
+    static const int smem_cap = tuning_int("CDB_GEMM_SMEM_KB", kMaxSmem / 1024) * 1024;       // tuning hook
     int budget = smem_cap < kMaxSmem ? smem_cap : kMaxSmem;
     if (h->gemm_smem_cap > 0 && h->gemm_smem_cap < budget) budget = h->gemm_smem_cap;
     const int stage_out = mode == kModeSwiGLU ? p.BN * BM * 2 : 0;   // output staging tile of the SwiGLU epilogue
@@ -639,8 +629,8 @@ static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* 
     static bool attr_set = false;
     if (!attr_set) {
         cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-        if (getenv("CDB_GEMM_CARVEOUT"))
-            cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, atoi(getenv("CDB_GEMM_CARVEOUT")));
+        if (tuning_int("CDB_GEMM_CARVEOUT", -2) > -2)           // tuning hook
+            cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, tuning_int("CDB_GEMM_CARVEOUT", -2));
         attr_set = true;
     }
     GemmParams p;
@@ -648,9 +638,12 @@ static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* 
     size_t smem = 0;
     const int n_tiles = setup_gemm(h, x, W, W2, y, act, n, N, K, mode, k_splits, split_stride, p, &map_w, &map_w2, &map_x, &smem);
     if (!n_tiles) return false;
+#ifdef CDB_TUNING
+    // tuning hook: device address of a stamp buffer (8 words per CTA), optionally for one launch kind only
     p.dbg = getenv("CDB_GEMM_DBG") ? (unsigned long long*)strtoull(getenv("CDB_GEMM_DBG"), nullptr, 0) : nullptr;
-    if (getenv("CDB_GEMM_DBG_ONLY") && atoi(getenv("CDB_GEMM_DBG_ONLY")) != mode * 100000 + N) p.dbg = nullptr;   // tuning aid: one launch kind
-    const int sms = device_sms();
+    if (getenv("CDB_GEMM_DBG_ONLY") && atoi(getenv("CDB_GEMM_DBG_ONLY")) != mode * 100000 + N) p.dbg = nullptr;
+#endif
+    const int sms = h->sms;
     const int grid = n_tiles < sms ? n_tiles : sms;
     launch_pdl(gemm_bf16_tcgen05_kernel, dim3(grid), dim3(kThreads), smem, st, map_w, map_w2, map_x, p);
     return true;
@@ -659,8 +652,8 @@ static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* 
 // Part count of a split-K projection.  It depends on the weight's shape alone, never on the number of rows,
 // so that a row's result does not depend on the batch it is computed in: at most one tile per SM for a batch
 // that fills one row tile, and at least four k-blocks per part.
-static int splitk_parts(int N, int K, int max_splits) {
-    const int sms = device_sms();
+static int splitk_parts(const cdb* h, int N, int K, int max_splits) {
+    const int sms = h->sms;
     const int n_ft = (N + BM - 1) / BM, n_kb = (K + BK - 1) / BK;
     int splits = sms / n_ft;                      // rounded down: one tile too many per wave would cost a second wave
     if (splits > n_kb / 4) splits = n_kb / 4;
@@ -681,7 +674,7 @@ bool launch_gate_up_swiglu_tc(const cdb* h, const void* x, const void* Wg, const
 // Split-K: partial products ws[s][n][N] (fp32), s < returned split count; the caller reduces them in
 // split order (deterministic).
 int launch_linear_splitk_tc(const cdb* h, const void* x, const void* W, float* ws, int max_splits, int n, int N, int K, cudaStream_t st) {
-    const int splits = splitk_parts(N, K, max_splits);
+    const int splits = splitk_parts(h, N, K, max_splits);
     return launch_gemm(h, x, W, nullptr, ws, nullptr, n, N, K, kModeStore, splits, (size_t)n * N, st) ? splits : 0;
 }
 
@@ -724,7 +717,7 @@ int launch_layer_tail_tc(const cdb* h, int ln, const RowsDev& rows, float* x, co
         ph.ws = L.ws; ph.splits = splits; ph.split_stride = (size_t)n * d; ph.x = x; ph.gain = gain; ph.out = (__nv_bfloat16*)L.xn;
         ++np;
     };
-    const int s_o = splitk_parts(d, d, kMaxKSplits), s_d = splitk_parts(d, F, kMaxKSplits);
+    const int s_o = splitk_parts(h, d, d, kMaxKSplits), s_d = splitk_parts(h, d, F, kMaxKSplits);
     int s_q = 0;
     if (!projection(L.attn_o, W_o, nullptr, L.ws, nullptr, d, d, kModeStore, s_o)) return -1;
     reduce(s_o, g_mlp);
@@ -732,7 +725,7 @@ int launch_layer_tail_tc(const cdb* h, int ln, const RowsDev& rows, float* x, co
     if (!projection(L.act, W_down, nullptr, L.ws, nullptr, d, F, kModeStore, s_d)) return -1;
     reduce(s_d, next_gain);
     if (W_qkv_next) {
-        s_q = splitk_parts(3 * d, d, kWsPerRow / 3);
+        s_q = splitk_parts(h, 3 * d, d, kWsPerRow / 3);
         if (!projection(L.xn, W_qkv_next, nullptr, L.ws, nullptr, 3 * d, d, kModeStore, s_q)) return -1;
     }
     P.n_phases = np;
@@ -740,14 +733,14 @@ int launch_layer_tail_tc(const cdb* h, int ln, const RowsDev& rows, float* x, co
     for (int i = 3 * np; i < 3 * kTailMaxPhases; ++i) maps.m[i] = maps.m[0];
 
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(device_sms()); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem_max; cfg.stream = st;
+    cfg.gridDim = dim3(h->sms); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem_max; cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeCooperative;
     attr[0].val.cooperative = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    static int with_pdl = getenv("CDB_NO_PDL") ? 0 : 1;
+    static int with_pdl = tuning_int("CDB_NO_PDL", 0) ? 0 : 1;
     cfg.numAttrs = 1 + with_pdl;
     cudaError_t e = cudaLaunchKernelEx(&cfg, layer_tail_tcgen05_kernel, maps, P);
     if (e != cudaSuccess && with_pdl) {            // this driver does not combine the two attributes: plain cooperative launch
