@@ -9,8 +9,9 @@
 //                      shared-memory ring, completion on mbarriers;
 //   warp 1 (one lane)  issues tcgen05.mma (M=128, N=BN, K=16) into one of two TMEM accumulators,
 //                      releases ring stages and publishes accumulators with tcgen05.commit;
-//   warps 2-5          epilogue: tcgen05.ld their 32-lane quarter of the accumulator and store / add
-//                      it to y (lanes = consecutive features -> coalesced rows of y).
+//   warps 2-9          epilogue: tcgen05.ld their 32-lane quarter of the accumulator (warps 2-5 the lower
+//                      half of its columns, warps 6-9 the upper half) and store / add it to y (lanes =
+//                      consecutive features -> coalesced rows of y).
 // CTAs are persistent over (feature tile, row tile) pairs.  Every mbarrier wait is bounded: on
 // expiry the CTA records a status word, lets its outstanding copies land, frees its TMEM and
 // returns.
@@ -31,7 +32,8 @@ using namespace tc;
 constexpr int BM = 128;            // features per tile (MMA M)
 constexpr int BK = 64;             // bf16 elements per k-block = one 128-byte swizzle span
 constexpr int UMMA_K = 16;
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;          // producer warp, MMA warp, eight epilogue warps
+constexpr int kEpiThreads = kThreads - 64;
 constexpr int kMaxSmem = 196 * 1024;    // every launch then asks for the same shared-memory carve-out (no SM reconfiguration between projections)
 
 enum { kModeStore = 0, kModeAccumulate = 1, kModeSwiGLU = 2 };
@@ -203,14 +205,21 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t t_addr = cx.tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * acc_cols;
             // 16 columns (= 16 batch rows) of this thread's feature per pass: a small register footprint
-            const int n_cols = min(BN, p.n - r0);               // columns holding real rows (warp-uniform)
-            if (dual) {
+            const int n_real = min(BN, p.n - r0);               // columns holding real rows (warp-uniform)
+            // two warps share a lane quarter: the first takes columns [0, mid), the second [mid, n_real)
+            const int mid = min(n_real, ((n_real + 1) / 2 + 15) & ~15);
+            const int c_beg = warp < 6 ? 0 : mid, n_cols = warp < 6 ? mid : n_real;
+            if (c_beg >= n_cols && !dual) {
+                // nothing in this warp's share
+            } else if (dual) {
                 // gate and up accumulators side by side; loads of the next 16 columns fly while these are finished
                 uint32_t v[2][16], u[2][16];
-                tmem_ld16(t_addr, v[0]);
-                tmem_ld16(t_addr + (uint32_t)BN, u[0]);
+                if (c_beg < n_cols) {
+                    tmem_ld16(t_addr + (uint32_t)c_beg, v[0]);
+                    tmem_ld16(t_addr + (uint32_t)(BN + c_beg), u[0]);
+                }
 #pragma unroll 1
-                for (int c0 = 0; c0 < n_cols; c0 += 32) {
+                for (int c0 = c_beg; c0 < n_cols; c0 += 32) {
 #pragma unroll
                     for (int hh = 0; hh < 2; ++hh) {
                         const int c = c0 + 16 * hh;
@@ -234,11 +243,11 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
                     }
                 }
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                asm volatile("bar.sync 1, 128;" ::: "memory");              // the four epilogue warps: tile staged
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // the epilogue warps: tile staged
                 {
-                    const int et = threadIdx.x - 64;                         // 0..127 among the epilogue warps
+                    const int et = threadIdx.x - 64;                         // index among the epilogue threads
                     const int f0t = (t % n_ftiles) * BM;
-                    for (int idx = et; idx < n_cols * 16; idx += 128) {      // 16 chunks of 8 features per row
+                    for (int idx = et; idx < n_real * 16; idx += kEpiThreads) {   // 16 chunks of 8 features per row
                         const int row = idx >> 4, ch = idx & 15;
                         const int fc = f0t + ch * 8;
                         uint4 val;
@@ -253,13 +262,13 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
                         }
                     }
                 }
-                asm volatile("bar.sync 1, 128;" ::: "memory");              // staging tile free for the next tile
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // staging tile free for the next tile
             } else {
                 // software pipeline: the TMEM load of the next 16 columns is in flight while these are stored
                 uint32_t v[2][16];
-                tmem_ld16(t_addr, v[0]);
+                tmem_ld16(t_addr + (uint32_t)c_beg, v[0]);
 #pragma unroll 1
-                for (int c0 = 0; c0 < n_cols; c0 += 32) {
+                for (int c0 = c_beg; c0 < n_cols; c0 += 32) {
 #pragma unroll
                     for (int hh = 0; hh < 2; ++hh) {
                         const int c = c0 + 16 * hh;
@@ -318,7 +327,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 4); }
+        for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), kEpiThreads / 32); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -424,7 +433,7 @@ layer_tail_tcgen05_kernel(const __grid_constant__ TailMaps maps, const __grid_co
     constexpr uint32_t tmem_cols = 512;
     auto init_barriers = [&]() {
         for (int s = 0; s < 8; ++s) { mbar_init(bar0 + 8u * s, 1); mbar_init(bar0 + 8u * (8 + s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(bar0 + 8u * (16 + a), 1); mbar_init(bar0 + 8u * (18 + a), 4); }
+        for (int a = 0; a < 2; ++a) { mbar_init(bar0 + 8u * (16 + a), 1); mbar_init(bar0 + 8u * (18 + a), kEpiThreads / 32); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     };
     if (threadIdx.x == 0) { abort_flag = 0; init_barriers(); }
@@ -454,7 +463,7 @@ layer_tail_tcgen05_kernel(const __grid_constant__ TailMaps maps, const __grid_co
                 }
                 if (last_wait && lane == 0) pdl_trigger();
             });
-        } else if (warp >= 2) {
+        } else if (warp >= 2 && warp < 6) {
             const int et = threadIdx.x - 64, q = warp - 2;                // 128 threads share a row
             if (pi > 0) {
                 if (et == 0) grid_wait(P.sync, ticket, abortp);
