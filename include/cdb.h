@@ -115,7 +115,9 @@ typedef struct {
 
 /* Creates a handle for one model on the current CUDA device.  Allocates scratch for max_rows
  * rows and gate state for max_seqs sequences.  CDB_ERR_ARG on inconsistent dims, CDB_ERR_NOMEM /
- * CDB_ERR_CUDA when allocation fails.  Synchronises the device. */
+ * CDB_ERR_CUDA when allocation fails.  Synchronises the device.  The handle belongs to that
+ * device: every later call on it must be made with the same device current (a process may hold
+ * handles on several devices). */
 int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out);
 int cdb_destroy(cdb_t* h);                       /* NULL is allowed */
 const char* cdb_last_error(const cdb_t* h);      /* static / handle-owned string */

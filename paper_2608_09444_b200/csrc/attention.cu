@@ -318,7 +318,8 @@ void launch_attention_plan(const cdb* h, int ln, const RowsDev& rows, cudaStream
 
 template <typename T, int DH, int LPT, int CPL, bool LAT>
 static void launch_attention_t(const cdb* h, const AttnParams& p, void* o, cudaStream_t st) {
-    static int blocks_per_sm = 0;
+    static int per_device[kMaxDevices] = {};
+    int& blocks_per_sm = per_device[h->device];
     if (blocks_per_sm == 0) {
         // The kernel uses no shared memory; asking for the largest shared-memory carve-out keeps the SM in the
         // configuration the projection kernel needs, so that its CTAs can become resident beside this one.

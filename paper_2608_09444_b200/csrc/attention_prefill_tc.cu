@@ -60,7 +60,7 @@ __global__ void __launch_bounds__(kPfThreads, 1)
 attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv, PfParams p) {
     pdl_trigger();
     constexpr int NCH = (DH + 63) / 64;                  // 64-wide slices of the head dimension
-    constexpr uint32_t kQBytes = NCH * kChunkBytes, kKvBytes = NCH * kChunkBytes, kPBytes = 2 * kChunkBytes;
+    constexpr uint32_t kQBytes = NCH * kChunkBytes, kKvBytes = NCH * kChunkBytes;       // P takes two chunks (128 keys)
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[16];
     __shared__ uint32_t tmem_base_slot;
@@ -364,7 +364,8 @@ bool launch_attention_prefill_tc(const cdb* h, int ln, int layer, const RowsDev&
     const long long max_items = (long long)rows.n_rows * H;            // at least one row per tile
     const int grid = (int)(max_items < sms ? max_items : sms);
     auto kern = Dh == 128 ? attn_prefill_tc_kernel<128> : Dh == 96 ? attn_prefill_tc_kernel<96> : attn_prefill_tc_kernel<64>;
-    static bool attr_set[3] = {false, false, false};
+    static bool attr_set_dev[kMaxDevices][3] = {};
+    bool* attr_set = attr_set_dev[h->device];
     const int ki = Dh == 128 ? 0 : Dh == 96 ? 1 : 2;
     if (!attr_set[ki]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;

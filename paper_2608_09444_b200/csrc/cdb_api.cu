@@ -289,10 +289,12 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
     {
         int dev = 0;
         h->sms = 148;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || h->sms < 1) {
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices ||
+            cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || h->sms < 1) {
             delete h;
             return CDB_ERR_CUDA;
         }
+        h->device = dev;
     }
     h->pool.H = c.H;
     h->pool.Dh = c.Dh;

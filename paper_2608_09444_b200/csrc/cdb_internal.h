@@ -15,6 +15,7 @@ constexpr int kSplitTokens = 256;    // attention split length; depends on nothi
 constexpr int kMaxKSplits = 8;       // most split-K parts of a projection
 constexpr int kWsPerRow = 12;        // workspace floats per row, in units of d: 8 parts of [d] or 3 parts of [3d] fit
 constexpr int kStatusPage = 1, kStatusPosition = 2, kStatusSeq = 3;
+constexpr int kMaxDevices = 64;      // one-time per-device kernel set-up is remembered per device ordinal
 
 // Tuning hooks: a build made with -DCDB_TUNING reads integer overrides from the environment (once per
 // site); the shipped library has none and every hook folds to its default.
@@ -86,7 +87,8 @@ struct cdb {
     cdb_weights_t w;
     cdbk::KvPool pool;
     size_t elem_size;               // bytes of the configured dtype
-    int sms;                        // multiprocessors of the device the handle was created on
+    int device;                     // the device that was current in cdb_create: every call on the handle must run there
+    int sms;                        // its multiprocessor count
     int max_splits;                 // ceil(max_position / kSplitTokens)
 
     // library-owned device memory

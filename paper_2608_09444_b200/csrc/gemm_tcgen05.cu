@@ -635,7 +635,8 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
 
 static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* W2, float* y, __nv_bfloat16* act, int n,
                         int N, int K, int mode, int k_splits, size_t split_stride, cudaStream_t st) {
-    static bool attr_set = false;
+    static bool attr_set_dev[kMaxDevices] = {};
+    bool& attr_set = attr_set_dev[h->device];
     if (!attr_set) {
         cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (tuning_int("CDB_GEMM_CARVEOUT", -2) > -2)           // tuning hook
@@ -698,7 +699,8 @@ int launch_layer_tail_tc(const cdb* h, int ln, const RowsDev& rows, float* x, co
     const Lane& L = h->lane[ln];
     const cdb_config_t& c = h->cfg;
     const int n = rows.n_rows, d = c.d, F = c.F;
-    static bool attr_set = false;
+    static bool attr_set_dev[kMaxDevices] = {};
+    bool& attr_set = attr_set_dev[h->device];
     if (!attr_set) {
         if (cudaFuncSetAttribute(layer_tail_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess) return -1;
         attr_set = true;
