@@ -100,6 +100,9 @@ def main():
     ap.add_argument("--min-coda-batch", type=int, default=0, help="exits gathered before a coda call (0: 1 for ouro, 8 for huginn; the offline runs use 32 for huginn)")
     ap.add_argument("--admit-min", type=int, default=1, help="hold arrived requests until this many wait ...")
     ap.add_argument("--admit-wait-ms", type=float, default=0.0, help="... or the oldest has waited this long")
+    ap.add_argument("--first-rate-index", type=int, default=0,
+                    help="position of the first of --rates in the sweep it belongs to (the trace seed follows the position): "
+                         "--rates 2 --first-rate-index 5 repeats the last trace of --rates 64,32,16,8,4,2")
     args = ap.parse_args()
     rank, local_rank, world = D.env_rank()
     if world > 1:
@@ -115,7 +118,7 @@ def main():
         report["b_gate"] = calibrate_gate_bias(dims, w, cal, 24, 2.5)
     else:
         gate_kind = B.GATE_NONE
-    for ri, rate in enumerate(float(x) for x in args.rates.split(",")):
+    for ri, rate in enumerate((float(x) for x in args.rates.split(",")), start=args.first_rate_index):
         arrivals, prompts, out_lens = make_requests(args.requests, rate, seed + 10 * ri, dims.V)
         forced = None
         if args.model == "huginn":       # replayed exit depths: truncated geometric, mean 12
