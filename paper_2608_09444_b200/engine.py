@@ -37,6 +37,8 @@ class Engine:
                  max_prefill_rows: int | None = None, flags: int = 0, record_states: bool = False,
                  record_logits: bool = False, record_ticks: bool = True, use_graphs: bool = True,
                  time_device: bool = False, admit_min: int = 1, admit_wait_s: float = 0.0, device: str = "cuda:0"):
+        if mode not in ("refill", "no_refill", "cb"):
+            raise ValueError(f"unknown scheduling mode {mode!r}: expected 'refill', 'no_refill' or 'cb'")
         self.dims, self.mode, self.lookahead = dims, mode, lookahead
         self.max_batch, self.max_live, self.min_coda_batch = max_batch, max_live, min_coda_batch
         self.dev = torch.device(device)

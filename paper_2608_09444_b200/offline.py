@@ -110,6 +110,9 @@ def main():
                     help="huginn: replayed geometric exit depths, or the convergence criterion with a calibrated threshold")
     ap.add_argument("--time-device", action="store_true", help="bracket every GPU phase with CUDA events and report device_ms")
     args = ap.parse_args()
+    known = {"cb", "refill", "no_refill", "refill_nographs", "cb_pipelined", "refill_pipelined"}
+    if not set(args.modes.split(",")) <= known:
+        raise SystemExit(f"--modes takes a comma-separated subset of {sorted(known)}")
     torch.cuda.set_device(0)
     if args.model == "ouro":
         dims, seed = synth.OURO_1P4B, 2

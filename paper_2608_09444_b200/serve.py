@@ -104,6 +104,9 @@ def main():
                     help="position of the first of --rates in the sweep it belongs to (the trace seed follows the position): "
                          "--rates 2 --first-rate-index 5 repeats the last trace of --rates 64,32,16,8,4,2")
     args = ap.parse_args()
+    known = {"cb", "refill", "no_refill", "cb_pipelined", "refill_pipelined"}
+    if not set(args.modes.split(",")) <= known:
+        raise SystemExit(f"--modes takes a comma-separated subset of {sorted(known)}")
     rank, local_rank, world = D.env_rank()
     if world > 1:
         import torch.distributed as dist
