@@ -27,7 +27,7 @@ from .engine import Engine, _bucket, _static_rows
 
 
 class PipelinedEngine(Engine):
-    def __init__(self, *a, background_prefill=True, **kw):
+    def __init__(self, *a, background_prefill=True, prefill_priority=0, **kw):
         kw.setdefault("mode", "refill")
         kw.setdefault("lookahead", True)
         super().__init__(*a, **kw)
@@ -39,7 +39,8 @@ class PipelinedEngine(Engine):
         # prompts of newly admitted requests are processed on a stream of their own beside the running decode
         # batch (the library gives prompt calls their own scratch); False = drain the pipeline and process them alone
         self.background_prefill = background_prefill
-        self.pstream = torch.cuda.Stream(device=self.dev, priority=0)
+        # (prefill_priority 0 = below the decode streams, -1 = level with them)
+        self.pstream = torch.cuda.Stream(device=self.dev, priority=prefill_priority)
         d = self.dims.d
         self.h_exit2 = [torch.zeros((self.max_rows, d), dtype=torch.float32, device=self.dev) for _ in range(2)]
         self.h_coda_in = torch.zeros((self.cap, d), dtype=torch.float32, device=self.dev)
