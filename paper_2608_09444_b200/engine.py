@@ -73,7 +73,8 @@ class Engine:
         self.tok_out = torch.zeros(max_rows, **i32)
         self.logits = torch.zeros((max_rows, dims.V), **f32) if record_logits else None
         self.record_states, self.record_logits, self.record_ticks = record_states, record_logits, record_ticks
-        self.stats = {"recurrent_steps": 0, "row_steps": 0, "coda_calls": 0, "prefill_calls": 0, "tick_rows": []}
+        self.stats = {"recurrent_steps": 0, "row_steps": 0, "coda_calls": 0, "prefill_calls": 0, "tick_rows": [],
+                      "rows_hist": [0] * ((max_batch + 31) // 32)}      # recurrent steps by row count, 32-row bins
         self.trace_states = {}                                        # (sid, token index) -> exit state
         self.trace_logits = {}
         # Recurrent step as a CUDA graph per row-count bucket (rows padded with seq_id = -1 to a multiple of 32):
@@ -349,6 +350,7 @@ class Engine:
             gv = self.gate_val[:k].cpu().numpy()
             self.stats["recurrent_steps"] += 1
             self.stats["row_steps"] += k
+            self.stats["rows_hist"][(k - 1) // 32] += 1
             if self.record_ticks:
                 self.stats["tick_rows"].append([(s, len(seqs[s].tokens), r) for s, r in rec])
             for i, (s, r) in enumerate(rec):

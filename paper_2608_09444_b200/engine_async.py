@@ -377,6 +377,7 @@ class PipelinedEngine(Engine):
                     depths[s].append(r)
                 self.stats["recurrent_steps"] += 1
                 self.stats["row_steps"] += k
+                self.stats["rows_hist"][(k - 1) // 32] += 1
                 prev = {"parity": parity, "ne": ne, "exits": exits, "G": G}
                 rec = [[rec[int(i)][0], rec[int(i)][1] + 1] for i in surv]
             it += 1

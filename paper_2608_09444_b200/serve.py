@@ -80,6 +80,7 @@ def run(dims, weights, arrivals, prompts, out_lens, *, mode, pipelined, gate_kin
     out = summarize(arrivals, out_lens, eng.stats)
     out["finish_s"], out["first_token_s"] = list(eng.stats["finish_s"]), list(eng.stats["first_token_s"])
     out["mode"] = mode + ("_pipelined" if pipelined else "")
+    out["recurrent_steps_by_rows_32"] = list(eng.stats["rows_hist"])      # this replica's steps by row count, 32-row bins
     out["status"] = eng.cdb.poll_status()
     d = np.concatenate([x for x in res["depths"] if len(x)]) if any(len(x) for x in res["depths"]) else np.zeros(0)
     out["mean_depth"] = float(d.mean()) if d.size else float(dims.R)
