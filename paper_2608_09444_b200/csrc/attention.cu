@@ -338,6 +338,10 @@ static void launch_attention_t(const cdb* h, const AttnParams& p, void* o, cudaS
     static const int forced_cap = tuning_int("CDB_ATTN_CAP", 0);      // tuning hook
     const int cap = forced_cap > 0 ? forced_cap : h->attn_ctas_per_sm_cap;
     if (cap > 0 && cap < blocks_per_sm) { grid = sms; threads = 128 * cap; }
+    // tuning hook (two-stream step only): attention on this many SMs, one CTA of all its warps per SM, so that the
+    // other half-batch's projection CTAs find the remaining SMs empty
+    static const int part_sms = tuning_int("CDB_ATTN_SMS", 0);
+    if (part_sms > 0 && part_sms <= sms && h->attn_ctas_per_sm_cap > 0) { grid = part_sms; threads = 128 * blocks_per_sm; }
     const int warps_per_cta = threads / 32;
     if ((max_items + warps_per_cta - 1) / warps_per_cta < grid) grid = (max_items + warps_per_cta - 1) / warps_per_cta;
     {

@@ -653,7 +653,8 @@ static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* 
     p.dbg = getenv("CDB_GEMM_DBG") ? (unsigned long long*)strtoull(getenv("CDB_GEMM_DBG"), nullptr, 0) : nullptr;
     if (getenv("CDB_GEMM_DBG_ONLY") && atoi(getenv("CDB_GEMM_DBG_ONLY")) != mode * 100000 + N) p.dbg = nullptr;
 #endif
-    const int sms = h->sms;
+    static const int part_sms = tuning_int("CDB_GEMM_SMS", 0);      // tuning hook (two-stream step only): CTA count of a projection
+    const int sms = (part_sms > 0 && part_sms <= h->sms && h->attn_ctas_per_sm_cap > 0) ? part_sms : h->sms;
     const int grid = n_tiles < sms ? n_tiles : sms;
     launch_pdl(gemm_bf16_tcgen05_kernel, dim3(grid), dim3(kThreads), smem, st, map_w, map_w2, map_x, p);
     return true;
