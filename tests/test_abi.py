@@ -54,3 +54,11 @@ def test_kv_footprint_accounting_matches_table1():
         used, reserved = kv_footprint(dims[model], int(slots))
         assert abs(used / 1024 - float(kib)) <= 0.5 and abs(used * 4096 / 2**30 - float(gib)) <= 0.006
         assert reserved >= used and (reserved == used) == (model == "ouro" or int(slots) == 1)
+
+
+def test_engines_reject_unknown_scheduling_modes_before_touching_the_gpu():
+    import pytest
+    from paper_2608_09444_b200 import synth
+    from paper_2608_09444_b200.engine import Engine
+    with pytest.raises(ValueError, match="unknown scheduling mode"):
+        Engine(synth.TINY, None, max_batch=4, max_live=4, max_len=32, n_pages=8, mode="none")
