@@ -75,19 +75,28 @@ def test_huginn_shaped_prelude_step_coda():
     assert all(v <= TOL for v in worst.values()), worst
 
 
-def test_lockstep_replay_of_adaptive_decode_bf16():
+@pytest.mark.parametrize("case", ["small", "ouro_full_size"])
+def test_lockstep_replay_of_adaptive_decode_bf16(case):
+    """small: 6 sequences x 12 tokens on a 3-layer model.  ouro_full_size: the offline-decode configuration's model
+    (Ouro-1.4B shape: 24 core layers, d 2048, vocabulary 49152, learned gate) on a sample of two sequences, prompt
+    processing included - what the oracle can compute token by token in a few seconds."""
     from paper_2608_09444_b200 import binding as B
     from paper_2608_09444_b200.engine import Engine
-    dims = synth.Dims(V=2048, d=512, H=4, Dh=128, F=1408, L_pre=0, L_core=3, L_coda=0, R=4, dtype="bf16")
-    w = synth.make_weights(dims, 6, std=0.03, gate_std=2.0 / np.sqrt(dims.d), b_gate=-0.8)
+    if case == "small":
+        dims = synth.Dims(V=2048, d=512, H=4, Dh=128, F=1408, L_pre=0, L_core=3, L_coda=0, R=4, dtype="bf16")
+        w = synth.make_weights(dims, 6, std=0.03, gate_std=2.0 / np.sqrt(dims.d), b_gate=-0.8)
+        n_seqs, T, max_batch = 6, 12, 4
+    else:
+        dims = synth.OURO_1P4B
+        w = synth.make_weights(dims, 2, device="cuda", gate_std=2.0 / np.sqrt(dims.d), b_gate=0.648)
+        n_seqs, T, max_batch = 2, 4, 2
     wn = synth.weights_to_numpy(w)
-    prompts = synth.make_prompts(6, 24, dims.V, 3)
-    T = 12
+    prompts = synth.make_prompts(n_seqs, 24, dims.V, 3)
     orc = O.Oracle(dims, wn, gate_kind=O.GATE_SIGMOID_CDF, q_or_eps=0.5, lookahead=True)
     ref = [orc.generate(p, T, keep_states=True) for p in prompts]
     depths = np.concatenate([r["depths"] for r in ref])
-    assert depths.min() >= 2 and len(set(depths)) >= 2
-    eng = Engine(dims, {k: v.cuda() for k, v in w.items()}, max_batch=4, max_live=6, max_len=24 + T, n_pages=6 * 3,
+    assert depths.min() >= 2 and (case != "small" or len(set(depths)) >= 2)
+    eng = Engine(dims, {k: v.cuda() for k, v in w.items()}, max_batch=max_batch, max_live=n_seqs, max_len=24 + T, n_pages=n_seqs * 3,
                  gate_kind=B.GATE_SIGMOID_CDF, q_or_eps=0.5, lookahead=True, mode="refill", max_prefill_rows=256,
                  record_states=True, record_logits=True)
     res = eng.generate(list(prompts), T, forced_depths=[list(r["depths"]) for r in ref],
