@@ -36,7 +36,9 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if force or _stale(o, [s] + headers):
             subprocess.check_call([nvcc, *flags, "-c", s, "-o", o])
     if force or _stale(LIB, objs):
-        subprocess.check_call([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB, *objs])
+        tmp = f"{LIB}.{os.getpid()}.tmp"             # link beside the target, then rename: a process that is loading the library never sees half of it
+        subprocess.check_call([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp, *objs])
+        os.replace(tmp, LIB)
     return LIB
 
 
