@@ -437,3 +437,127 @@ def test_truncated_geometric_closed_form():
     assert abs(p - 0.076893) < 2e-6
     d = synth.forced_exit_depths((200000,), 3)
     assert d.min() >= 1 and d.max() == 32 and abs(d.mean() - 12.0) < 0.1
+
+
+# ------------------------------------------------------------------ the step-level entry of the oracle
+
+def _dense_core_kv(orc, cache, r, t):
+    """Per core layer, copies of the dense K and V of the slot loop step r uses, positions 0..t."""
+    dm = orc.dm
+    s = O.kv_slot(orc.layout, r)
+    Ks = [cache[l][s][0][:t + 1].copy() for l in range(dm.L_pre, dm.L_pre + dm.L_core)]
+    Vs = [cache[l][s][1][:t + 1].copy() for l in range(dm.L_pre, dm.L_pre + dm.L_core)]
+    return Ks, Vs
+
+
+@pytest.mark.parametrize("layout", [O.SHARED, O.DEPTH_INDEXED])
+@pytest.mark.parametrize("kind", [O.GATE_SIGMOID_CDF, O.GATE_L2_CONVERGENCE])
+def test_loop_step_row_is_the_step_inside_decode(layout, kind):
+    """Eq. 1: the single-row loop step used for step-level parity must be the very step that the
+    serial decoder (pinned above by the library transformer) takes.  Positions < t of a cache never
+    change once their tokens have left, so the finished run's cache is the cache as it stood before
+    any step of token t, apart from position t itself, which the step rewrites."""
+    dims = SMALL.replace(R=4, L_pre=2)
+    w = small_weights(dims, gate_std=0.3, b_gate=-0.4)
+    orc = O.Oracle(dims, w, kv_layout=layout, gate_kind=kind, q_or_eps=0.5 if kind == O.GATE_SIGMOID_CDF else 0.0)
+    prompt = synth.make_prompts(1, 5, dims.V, 21)[0]
+    forced = [4, 2, 3, 1]
+    out = orc.generate(prompt, 5, forced_depths=forced, keep_states=True)
+    cache = out["cache"]
+    core = range(dims.L_pre, dims.L_pre + dims.L_core)
+    checked = 0
+    for j, rec in enumerate(out["passes"]):
+        t = len(prompt) + j
+        y = int(out["tokens"][j])
+        h = orc.prelude([y], np.array([t]), cache)[0]       # rewrites the prelude layers' entry t with itself
+        S = 1.0
+        for r in range(1, rec["depth"] + 1):
+            Ks, Vs = _dense_core_kv(orc, cache, r, t)
+            for a in Ks + Vs:
+                a[t] = np.nan                               # the step must write position t before reading it
+            h_out, g, fire, S, new_kv = orc.loop_step_row(h, t, r, Ks, Vs, S)
+            assert np.array_equal(h_out, rec["states"][r - 1])
+            assert g == rec["gate"][r - 1] and fire == rec["fire"][r - 1]
+            if layout == O.DEPTH_INDEXED or r == rec["depth"]:
+                s = O.kv_slot(layout, r)
+                for i, l in enumerate(core):
+                    assert np.array_equal(new_kv[i][0], cache[l][s][0][t])
+                    assert np.array_equal(new_kv[i][1], cache[l][s][1][t])
+            h = h_out
+            checked += 1
+    assert checked == sum(forced)
+
+
+def test_convergence_gate_value_and_exit_depths_by_hand():
+    """Appendix C.2: the value is the plain L2 distance of consecutive recurrent states (h_0 = the
+    prelude output), and a token leaves one step after the first r >= 2 whose distance is below
+    the threshold (section 4.3), or after step R."""
+    dims = SMALL.replace(R=6, L_pre=1)
+    w = small_weights(dims, seed=9)                  # a draw whose distances fall from r = 2 on
+    prompt = synth.make_prompts(1, 5, dims.V, 23)[0]
+    free = O.Oracle(dims, w, gate_kind=O.GATE_L2_CONVERGENCE, q_or_eps=0.0)         # never fires
+    out = free.generate(prompt, 2, keep_states=True)
+    rec = out["passes"][0]
+    assert rec["depth"] == dims.R
+    t = len(prompt)
+    h0 = free.prelude([int(out["tokens"][0])], np.array([t]), out["cache"])[0]
+    hs = [h0] + rec["states"]
+    dist = [float(np.linalg.norm(hs[r] - hs[r - 1])) for r in range(1, dims.R + 1)]
+    assert np.allclose(rec["gate"], dist, rtol=1e-13, atol=0)
+    assert len(set(np.round(dist[1:], 9))) == len(dist) - 1                          # the thresholds below separate them
+    # a threshold just above the r-th distance (r >= 2) and below all earlier ones from r = 2 on
+    seen = 0
+    for r in range(2, dims.R + 1):
+        if any(dist[j - 1] <= dist[r - 1] for j in range(2, r)):
+            continue
+        eps = dist[r - 1] * (1 + 1e-9)
+        for lookahead, want in ((True, min(dims.R, r + 1)), (False, r)):
+            orc = O.Oracle(dims, w, gate_kind=O.GATE_L2_CONVERGENCE, q_or_eps=eps, lookahead=lookahead)
+            got = orc.generate(prompt, 2)["depths"][0]
+            assert got == want, (r, lookahead, got)
+        strict = O.Oracle(dims, w, gate_kind=O.GATE_L2_CONVERGENCE, q_or_eps=dist[r - 1], lookahead=False)
+        assert r == dims.R or strict.generate(prompt, 2)["depths"][0] > r             # strict "<"
+        seen += 1
+    assert seen >= 4
+    # the first distance (h_1 against the prelude output) never counts, however small the others are
+    big = O.Oracle(dims, w, gate_kind=O.GATE_L2_CONVERGENCE, q_or_eps=dist[0] * 1e6, lookahead=False)
+    assert big.generate(prompt, 2)["depths"][0] == 2
+
+
+def test_gate_bias_calibration_finds_a_known_step():
+    """The bisection on a stand-in whose mean depth is a known decreasing step function of b."""
+    class Stub:
+        def __init__(self, b):
+            self.b = b
+
+        def generate(self, prompt, T):
+            # depth 4 below b = 1.25, depth 3 up to 2.0, depth 2 above
+            return {"depths": np.full(T - 1, 4 if self.b < 1.25 else 3 if self.b < 2.0 else 2)}
+    b, mean = O.calibrate_gate_bias(Stub, [None, None], 5, 2.5, iters=40, back_off=0.05)
+    assert abs(b - 1.95) < 1e-6 or abs(b - 2.05) < 1e-6          # the crossing of 2.5 is at 2.0; either side is 0.5 off
+    assert mean in (2.0, 3.0)
+    b, mean = O.calibrate_gate_bias(Stub, [None], 5, 3.2, iters=40, back_off=0.05)
+    assert abs(b - 1.30) < 1e-6 and mean == 3.0                  # crossing of 3.2 at 1.25; 3.0 is closer than 4.0
+
+
+def test_golden_gate_bias_reproduces_its_header():
+    """The stored bias of the tiny config is data; its header line states what the oracle gets with it."""
+    lines = open(os.path.join(GOLDEN, "c1_gate_bias.txt")).read().splitlines()
+    b = float(lines[-1])
+    import re
+    m = re.search(r"sequences 0-1: ([\d.]+); of all 8 sequences: ([\d.]+); histogram depth 1..4: \[([\d, ]+)\]", lines[1])
+    mean01, mean_all, hist = float(m.group(1)), float(m.group(2)), [int(x) for x in m.group(3).split(",")]
+    dims = synth.TINY
+    w = synth.weights_to_numpy(synth.make_weights(dims, seed=0, std=0.02))
+    w["b_gate"] = np.array([b], dtype=np.float32)
+    prompts = synth.make_prompts(8, 32, dims.V, seed=0)
+    orc = O.Oracle(dims, w, gate_kind=O.GATE_SIGMOID_CDF, q_or_eps=0.5, lookahead=True)
+    outs = [orc.generate(p, 16, keep_states=False) for p in prompts]
+    depths = np.concatenate([o["depths"] for o in outs])
+    assert abs(depths[:30].mean() - mean01) < 5e-5 and abs(depths.mean() - mean_all) < 5e-5
+    assert np.bincount(depths, minlength=5)[1:].tolist() == hist
+    assert depths.min() >= 2                                     # lookahead: no gate-driven exit below depth 2
+    # every decision is off the threshold by more than fp32 noise (the calibration's back-off)
+    margin = min(abs(g - 0.5) for o in outs for p in o["passes"] for g in p["gate"])
+    print("minimum |gate value - q| over the run:", margin)
+    assert margin > 1e-4
