@@ -77,23 +77,60 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def oracle_sample(wl, row_ids):
-    """Builds the CPU oracle and its inputs for a few rows of the workload (untimed set-up)."""
+def build_oracle(dims, weights_np):
+    """The CPU oracle for the core layers alone (the microbenchmark has no prelude or coda)."""
     import numpy as np
     from oracle import cdb_oracle as O
+    wn = {k: weights_np[k] for k in ("W_qkv", "W_o", "W_gate", "W_up", "W_down", "g_attn", "g_mlp", "w_gate", "b_gate")}
+    wn["g_final"] = np.ones(dims.d, dtype=np.float32)
+    return O.Oracle(dims.replace(L_pre=0, L_coda=0), wn, gate_kind=O.GATE_SIGMOID_CDF, q_or_eps=0.5)
+
+
+def densify(dims, items):
+    """Dense per-layer K, V of each sampled row from its pages (untimed set-up)."""
+    from oracle import cdb_oracle as O
+    for it in items:
+        kv = [O.gather_pages(it["pages"][l], it["table"], it["ctx"]) for l in range(dims.L_core)]
+        it["K"], it["V"] = [k for k, _ in kv], [v for _, v in kv]
+        del it["pages"]
+    return items
+
+
+def oracle_sample(wl, row_ids):
+    """The CPU oracle and its inputs for a few rows of the GPU arm's workload (untimed set-up)."""
     from paper_2608_09444_b200 import synth
     dm = wl.dims
     core = {k: v[dm.L_pre:dm.L_pre + dm.L_core] if v.dim() >= 2 and v.shape[0] == dm.L else v for k, v in wl.weights.items()}
     wn = synth.weights_to_numpy({k: core[k] for k in ("W_qkv", "W_o", "W_gate", "W_up", "W_down", "g_attn", "g_mlp", "w_gate", "b_gate")})
-    wn["g_final"] = np.ones(dm.d, dtype=np.float32)
-    only_core = dm.replace(L_pre=0, L_coda=0)
-    orc = O.Oracle(only_core, wn, gate_kind=O.GATE_SIGMOID_CDF, q_or_eps=0.5)
-    items = wl.oracle_inputs(row_ids)
-    for it in items:
-        kv = [O.gather_pages(it["pages"][l], it["table"], it["ctx"]) for l in range(dm.L_pre, dm.L_pre + dm.L_core)]
-        it["K"], it["V"] = [k for k, _ in kv], [v for _, v in kv]
-        del it["pages"]
-    return orc, items
+    items = [dict(it, pages=it["pages"][dm.L_pre:dm.L_pre + dm.L_core]) for it in wl.oracle_inputs(row_ids)]
+    return build_oracle(dm, wn), densify(dm, items)
+
+
+def host_sample(dims, n_rows, seed, ctx_lo, ctx_hi, row_ids):
+    """The reference arm's inputs, made on the host alone from the same recipe as the GPU arm's workload
+    (same seeded row descriptor; weights, KV pages and row states are fresh draws of the same distributions,
+    since the GPU arm fills those with the device's generator).  Loads nothing of the CUDA library."""
+    import numpy as np
+    import torch
+    from paper_2608_09444_b200 import synth
+    gen = torch.Generator().manual_seed(seed)
+    grid = (lambda t: t.to(torch.bfloat16).to(torch.float32)) if dims.dtype == "bf16" else (lambda t: t)
+    normal = lambda shape, std: grid(torch.empty(shape, dtype=torch.float32).normal_(0.0, std, generator=gen)).numpy()
+    d, F, L = dims.d, dims.F, dims.L_core
+    wn = {"W_qkv": normal((L, 3 * d, d), 0.02), "W_o": normal((L, d, d), 0.02), "W_gate": normal((L, F, d), 0.02),
+          "W_up": normal((L, F, d), 0.02), "W_down": normal((L, d, F), 0.02),
+          "g_attn": np.ones((L, d), np.float32), "g_mlp": np.ones((L, d), np.float32),
+          "w_gate": normal((d,), 2.0 / np.sqrt(d)), "b_gate": np.zeros(1, np.float32)}
+    rows = synth.make_step_rows(n_rows, dims.R, seed, ctx_lo, ctx_hi)
+    items = []
+    for i in row_ids:
+        c = int(rows["position"][i]) + 1
+        n_pages = (c + dims.page_size - 1) // dims.page_size
+        items.append({"row": int(i), "ctx": c, "depth": int(rows["loop_depth"][i]),
+                      "h": torch.empty(d).normal_(0.0, 1.0, generator=gen).numpy(),
+                      "pages": normal((L, n_pages, 2, dims.H, dims.page_size, dims.Dh), 1.0),
+                      "table": np.arange(n_pages)})
+    return build_oracle(dims, wn), densify(dims, items)
 
 
 def oracle_step(orc, items):
@@ -134,11 +171,6 @@ def main():
     if args.impl == "reference" and rank != 0:
         return 0
 
-    import numpy as np
-    import torch
-    import __graft_entry__
-    if local_rank == 0:
-        __graft_entry__.build()
     from paper_2608_09444_b200 import synth
 
     base = synth.OURO_1P4B if args.model == "ouro" else synth.HUGINN_3P5B
@@ -147,20 +179,10 @@ def main():
     config = {"workload": workload, "rows": args.rows, "core_layers": dims.L_core, "page_table": "contiguous" if args.contiguous_pages else "random permutation",
               "l2": "inputs larger than L2 (each step streams the whole KV pool and all core weights)"}
 
-    if world > 1 and args.impl == "cdb":     # the reference arm runs on rank 0 alone: no process group
-        import torch.distributed as dist
-        dist.init_process_group("nccl")
-    torch.cuda.set_device(local_rank)
-    from paper_2608_09444_b200 import binding as B
-    from paper_2608_09444_b200.workloads import LoopStepWorkload
-    wl = LoopStepWorkload(dims, n_rows=args.rows, seed=D.rank_seed(1, rank), ctx_lo=args.ctx_lo, ctx_hi=args.ctx_hi,
-                          permute=not args.contiguous_pages, device=f"cuda:{local_rank}", flags=(B.FLAG_SIMT_GEMM if args.simt_gemm else 0) | (B.FLAG_TWO_STREAM if args.two_stream else 0))
-    alg = wl.algorithmic()
-    cores = len(os.sched_getaffinity(0))
-
     if args.impl == "reference":
+        # host only: the oracle (NumPy) on inputs drawn on the host; neither the CUDA library nor a GPU is touched
         sample_rows = [0, 1]
-        orc, items = oracle_sample(wl, sample_rows)
+        orc, items = host_sample(dims, args.rows, D.rank_seed(1, rank), args.ctx_lo, args.ctx_hi, sample_rows)
         for _ in range(args.warmup):
             oracle_step(orc, items)
         t = sum(oracle_step(orc, items) for _ in range(args.steps))
@@ -174,6 +196,22 @@ def main():
                           "e2e": {"value": value, "unit": "token-loop-steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
                           "gpu_launches": 0}))
         return 0
+
+    import numpy as np
+    import torch
+    import __graft_entry__
+    if local_rank == 0:
+        __graft_entry__.build()
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl")
+    torch.cuda.set_device(local_rank)
+    from paper_2608_09444_b200 import binding as B
+    from paper_2608_09444_b200.workloads import LoopStepWorkload
+    wl = LoopStepWorkload(dims, n_rows=args.rows, seed=D.rank_seed(1, rank), ctx_lo=args.ctx_lo, ctx_hi=args.ctx_hi,
+                          permute=not args.contiguous_pages, device=f"cuda:{local_rank}", flags=(B.FLAG_SIMT_GEMM if args.simt_gemm else 0) | (B.FLAG_TWO_STREAM if args.two_stream else 0))
+    alg = wl.algorithmic()
+    cores = len(os.sched_getaffinity(0))
 
     def barrier():
         if world > 1:

@@ -99,8 +99,8 @@ typedef struct {
     const float* w_gate;  /* [d] fp32, learned exit head (may be NULL when gate_kind != SIGMOID_CDF) */
 } cdb_weights_t;
 
-/* Row descriptor of one call: rows are (sequence, loop depth) items (section 4.1: "recurrent
- * items ready for their next loop step").  Arrays are device int32 [n_rows]. */
+/* Row descriptor of one call: rows are (sequence, loop depth) items, i.e. the entries of the
+ * recurrent queue of section 4.1.  Arrays are device int32 [n_rows]. */
 typedef struct {
     int32_t        n_rows;           /* host: number of rows, pads included; <= max_rows */
     const int32_t* seq_id;           /* -1 = pad */
@@ -110,7 +110,8 @@ typedef struct {
     const int32_t* forced_exit;      /* replayed exit depth, 0 = decided by the gate; may be NULL */
     const int32_t* page_table;       /* device [max_seqs * n_slots][page_table_stride]: physical page
                                         of logical page j of (seq_id, kv_slot), row seq_id*n_slots+kv_slot */
-    int32_t        page_table_stride;
+    int32_t        page_table_stride; /* a row whose position needs logical page >= page_table_stride is skipped
+                                        (no KV write, zero attention output) and reported as status 2 */
 } cdb_rows_t;
 
 /* Creates a handle for one model on the current CUDA device.  Allocates scratch for max_rows
@@ -151,8 +152,8 @@ int cdb_boundary_prelude(cdb_t* h, const int32_t* token_ids, const cdb_rows_t* r
 int cdb_loop_step(cdb_t* h, const cdb_rows_t* rows, float* h_inout, float* gate_val_out,
                   uint8_t* fire_out, void* stream);
 
-/* Exit flag and stable compaction (section 4.1: "the exit decision routes tokens either back to
- * the recurrent queue or out to the coda").  For every non-pad row
+/* Exit flag and stable compaction (section 4.1, exit routing: a token either re-enters the
+ * recurrent queue or leaves for the coda).  For every non-pad row
  *   exit = loop_depth >= R  ||  (forced_exit > 0 ? forced_exit == loop_depth
  *                                               : signal && loop_depth >= r_min)
  * where signal = fire_prev[row] if fire_prev != NULL, else the sequence's stored signal.  With the
@@ -211,7 +212,12 @@ int cdb_linear(cdb_t* h, const void* x, const void* W, float* y, int32_t n, int3
  *   q, o: device [n_rows][H*Dh] of `dtype`;  pool: device [layers][n_phys_pages][2][H][16][Dh];
  *   seq_id, position: device int32 [n_rows] (seq_id < 0 = pad, output row zeroed);
  *   page_table: device int32 [max_seqs][page_table_stride];  max_context: host upper bound on
- *   position + 1 (a row beyond it is skipped and its output zeroed).
+ *   position + 1, at most 16 * page_table_stride (CDB_ERR_ARG otherwise, so that no row can index past
+ *   its table row).
+ * Range errors inside the data are NOT reported by this entry point: it has no handle, so there is no
+ * status word a caller could poll.  A row with position >= max_context or seq_id >= max_seqs is skipped and
+ * its output row zeroed; a page id outside [0, n_phys_pages) is skipped, i.e. the row's output is the
+ * attention over its remaining pages.  Callers that need the report use cdb_paged_attention.
  * Limit: 256 + 4*(n_rows+1) rounded up to 256 + n_rows*H*ceil(max_context/256)*(Dh+2)*4 bytes must fit in
  * 8 MiB (e.g. 64 rows x 16 heads x 2048 context at Dh 128); larger requests return CDB_ERR_CAPACITY and
  * print the sizes to stderr.  The first call on a device looks up the array's device address

@@ -6,9 +6,9 @@ no code with it.
 
 What it computes (paper section 2, Eq. 1): each sequence alone, token by token,
     h0 = P(x_t);  h_{r+1} = R(h_r, K^{(r)}_{<t});  next token = argmax C(h_{r_t})
-with the recurrent core R looped serially to the token's own exit depth r_t.  CDB "executes a
-given exit rule without changing the model's predictions" (section 3), so this serial
-definition is the expected result of any batched / refilled / reordered schedule.
+with the recurrent core R looped serially to the token's own exit depth r_t.  Section 3 states
+that CDB only schedules a given exit rule and leaves the model's outputs as they are, so this
+serial definition is the expected result of any batched / refilled / reordered schedule.
 
 Readings of points the paper leaves open (all fixed here, the CUDA path must agree):
   * block: pre-norm Llama-style layer, two RMSNorms (eps 1e-6), no biases, MHA, causal
@@ -16,7 +16,7 @@ Readings of points the paper leaves open (all fixed here, the CUDA path must agr
     the LM head;
   * RoPE: theta 10000, rotate-half pairing (i, i + Dh/2), absolute position, the same at every
     loop depth;
-  * learned gate (section 3 related work / appendix C.2 describe only "a small head" and a
+  * learned gate (section 3 related work / appendix C.2 describe only a small gating head and a
     threshold q whose increase gives fewer early exits): lambda_r = sigmoid(w_g . n(h_r) + b)
     with n = RMSNorm without gain, survival S_r = prod_{j<=r}(1 - lambda_j), signal fires when
     1 - S_r >= q;

@@ -58,8 +58,12 @@ struct AttnParams {
 };
 
 // splits per row -> exclusive scan; zeroes the per-layer work counters.  One CTA.
+// A row whose position lies outside [0, max_position) or beyond what its page-table row covers gets no split
+// (its output is zeroed by the merge) and latches the status word; the split count never exceeds the partial
+// area's max_splits per (row, head).
 __global__ void __launch_bounds__(1024) attn_plan_kernel(RowsDev rows, int32_t* __restrict__ item_start,
-                                                         int32_t* __restrict__ counters, int n_counters) {
+                                                         int32_t* __restrict__ counters, int n_counters,
+                                                         int max_position, int max_splits, int32_t* __restrict__ status) {
     pdl_trigger();
     pdl_wait();
     __shared__ int warp_tot[32];
@@ -73,7 +77,8 @@ __global__ void __launch_bounds__(1024) attn_plan_kernel(RowsDev rows, int32_t* 
         int ns = 0;
         if (row < rows.n_rows && rows.seq_id[row] >= 0) {
             const int pos = rows.position[row];
-            ns = pos >= 0 ? (pos + kSplitTokens) / kSplitTokens : 0;       // ceil((pos+1)/split)
+            if (pos >= max_position || (pos >= 0 && pos / kPageSize >= rows.page_table_stride)) atomicCAS(status, 0, kStatusPosition);
+            else if (pos >= 0) ns = min((pos + kSplitTokens) / kSplitTokens, max_splits);      // ceil((pos+1)/split)
         }
         int inc = ns;
 #pragma unroll
@@ -265,8 +270,9 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(AttnParams p, T* __rest
     const int row = wid / H, head = wid % H;
     T* o = out + (size_t)row * H * DH + (size_t)head * DH;
     constexpr int PER = (DH + 31) / 32;
-    const int ns = p.item_start[row + 1] - p.item_start[row];
-    if (p.rows.seq_id[row] < 0 || ns <= 0) {
+    const int ns = min(p.item_start[row + 1] - p.item_start[row], p.max_splits);
+    const int sq = p.rows.seq_id[row];
+    if (sq < 0 || sq >= p.max_seqs || ns <= 0) {          // pads and rows the plan or the split kernel skipped
 #pragma unroll
         for (int k = 0; k < PER; ++k) if (lane + 32 * k < DH) o[lane + 32 * k] = T(0.f);
         return;
@@ -313,7 +319,8 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(AttnParams p, T* __rest
 
 void launch_attention_plan(const cdb* h, int ln, const RowsDev& rows, cudaStream_t st) {
     CDB_LAUNCH(h);
-    launch_pdl(attn_plan_kernel, dim3(1), dim3(1024), 0, st, rows, h->lane[ln].attn_item_start, h->lane[ln].attn_counters, h->cfg.L_pre + h->cfg.L_core + h->cfg.L_coda);
+    launch_pdl(attn_plan_kernel, dim3(1), dim3(1024), 0, st, rows, h->lane[ln].attn_item_start, h->lane[ln].attn_counters,
+               h->cfg.L_pre + h->cfg.L_core + h->cfg.L_coda, h->cfg.max_position, h->max_splits, h->status);
 }
 
 template <typename T, int DH, int LPT, int CPL, bool LAT>
@@ -408,8 +415,9 @@ unsigned char* g_static_scratch_addr[kStaticMaxDevices];         // device addre
 
 // Per-row split counts (clamped to the partial area's capacity) -> exclusive scan, and the zeroing of the
 // work counter and status word.  The row count of this variant is small: one thread walks the rows.
-__global__ void attn_static_plan_kernel(RowsDev rows, int max_splits, int max_context, int32_t* __restrict__ item_start,
-                                        int32_t* __restrict__ counter, int32_t* __restrict__ status) {
+__global__ void attn_static_plan_kernel(RowsDev rows, int max_splits, int max_context, int max_seqs,
+                                        int32_t* __restrict__ item_start, int32_t* __restrict__ counter,
+                                        int32_t* __restrict__ status) {
     pdl_trigger();
     pdl_wait();
     if (blockIdx.x != 0 || threadIdx.x != 0) return;
@@ -420,6 +428,7 @@ __global__ void attn_static_plan_kernel(RowsDev rows, int max_splits, int max_co
         item_start[row] = acc;
         const int pos = rows.position[row];
         if (rows.seq_id[row] < 0 || pos < 0) continue;
+        if (rows.seq_id[row] >= max_seqs) { *status = kStatusSeq; continue; } // no table row: skipped, output zeroed
         if (pos >= max_context) { *status = kStatusPosition; continue; }      // beyond the stated bound: row skipped
         const int ns = (pos + kSplitTokens) / kSplitTokens;
         acc += ns < max_splits ? ns : max_splits;
@@ -429,7 +438,7 @@ __global__ void attn_static_plan_kernel(RowsDev rows, int max_splits, int max_co
 
 template <typename T, int DH, int LPT, int CPL>
 void launch_attention_static_t(const AttnParams& p, void* o, int max_context, cudaStream_t st) {
-    launch_pdl(attn_static_plan_kernel, dim3(1), dim3(32), 0, st, p.rows, p.max_splits, max_context, const_cast<int32_t*>(p.item_start), p.counter, p.status);
+    launch_pdl(attn_static_plan_kernel, dim3(1), dim3(32), 0, st, p.rows, p.max_splits, max_context, p.max_seqs, const_cast<int32_t*>(p.item_start), p.counter, p.status);
     const int max_items = p.rows.n_rows * p.pool.H * p.max_splits;
     int grid = 148 * 4;
     if ((max_items + 3) / 4 < grid) grid = (max_items + 3) / 4;
@@ -451,6 +460,11 @@ extern "C" int cdb_paged_attention_static(const void* q, void* o, const void* po
         page_table_stride < 1 || max_seqs < 1 || max_context < 1 || H < 1 || (Dh != 64 && Dh != 96 && Dh != 128) ||
         (dtype != CDB_FP32 && dtype != CDB_BF16))
         return CDB_ERR_ARG;
+    if ((int64_t)max_context > (int64_t)page_table_stride * kPageSize) {            // a row could index past its table row
+        fprintf(stderr, "cdb_paged_attention_static: max_context=%d exceeds the %d tokens a page-table row of %d pages covers\n",
+                max_context, page_table_stride * kPageSize, page_table_stride);
+        return CDB_ERR_ARG;
+    }
     const int max_splits = (max_context + kSplitTokens - 1) / kSplitTokens;
     const size_t head = 256;                                                        // status word, work counter
     const size_t scan = (((size_t)n_rows + 1) * sizeof(int32_t) + 255) / 256 * 256;
@@ -582,7 +596,7 @@ __global__ void __launch_bounds__(128) attn_prefill_kernel(AttnParams p, const i
     const int slot = p.rows.slot_of(row0);
     const int pos = p.rows.position[row];
     const int pos_last = p.rows.position[row0 + nq - 1];
-    if (seq < 0 || seq >= p.max_seqs || slot < 0 || slot >= p.rows.n_slots || pos_last < 0) {
+    if (seq < 0 || seq >= p.max_seqs || slot < 0 || slot >= p.rows.n_slots || pos_last < 0 || pos_last / kPageSize >= p.rows.page_table_stride) {
         if (threadIdx.x == 0) atomicCAS(p.status, 0, kStatusSeq);
         return;
     }

@@ -152,7 +152,10 @@ __global__ void __launch_bounds__(256) rope_kv_write_kernel(const float* __restr
     const int slot = rows.slot_of(row);
     if (seq < 0) return;
     if (seq >= max_seqs || slot < 0 || slot >= rows.n_slots) { if (threadIdx.x == 0) atomicCAS(status, 0, kStatusSeq); return; }
-    if (pos < 0 || pos >= max_position) { if (threadIdx.x == 0) atomicCAS(status, 0, kStatusPosition); return; }
+    if (pos < 0 || pos >= max_position || pos / kPageSize >= rows.page_table_stride) {
+        if (threadIdx.x == 0) atomicCAS(status, 0, kStatusPosition);
+        return;
+    }
     const int page = rows.page_table[((size_t)seq * rows.n_slots + slot) * rows.page_table_stride + pos / kPageSize];
     if (page < 0 || page >= pool.n_phys_pages) { if (threadIdx.x == 0) atomicCAS(status, 0, kStatusPage); return; }
     // four consecutive pair indices per thread: float4 loads of each split-K part, 8- or 16-byte stores
@@ -434,7 +437,7 @@ void launch_argmax(const cdb* h, const float* logits, int n_rows, int32_t* token
 // Last-exited cache: k, v of the row's position in slot exit_depth-1 -> slots exit_depth..R-1.
 template <typename T>
 __global__ void __launch_bounds__(256) copy_on_exit_kernel(KvPool pool, RowsDev rows, const int32_t* __restrict__ exit_depth,
-                                                           int layer0, int R, int max_seqs, int32_t* status) {
+                                                           int layer0, int R, int max_seqs, int max_position, int32_t* status) {
     pdl_trigger();
     pdl_wait();
     const int row = blockIdx.x, layer = layer0 + blockIdx.y;
@@ -442,6 +445,11 @@ __global__ void __launch_bounds__(256) copy_on_exit_kernel(KvPool pool, RowsDev 
     if (seq < 0 || seq >= max_seqs) return;
     const int pos = rows.position[row], rt = exit_depth[row];
     if (rt < 1 || rt >= R) return;
+    if (rt > rows.n_slots) { if (threadIdx.x == 0) atomicCAS(status, 0, kStatusSeq); return; }
+    if (pos < 0 || pos >= max_position || pos / kPageSize >= rows.page_table_stride) {
+        if (threadIdx.x == 0) atomicCAS(status, 0, kStatusPosition);
+        return;
+    }
     const size_t trow = (size_t)seq * rows.n_slots;
     const int src_page = rows.page_table[(trow + rt - 1) * rows.page_table_stride + pos / kPageSize];
     if (src_page < 0 || src_page >= pool.n_phys_pages) { if (threadIdx.x == 0) atomicCAS(status, 0, kStatusPage); return; }
@@ -464,9 +472,9 @@ void launch_copy_on_exit(const cdb* h, const RowsDev& rows, const int32_t* exit_
     if (rows.n_rows <= 0 || h->cfg.L_core <= 0) return;
     dim3 grid(rows.n_rows, h->cfg.L_core);
     if (h->cfg.dtype == CDB_FP32)
-        launch_pdl(copy_on_exit_kernel<float>, dim3(grid), dim3(256), 0, st, h->pool, rows, exit_depth, h->cfg.L_pre, h->cfg.R, h->cfg.max_seqs, h->status);
+        launch_pdl(copy_on_exit_kernel<float>, dim3(grid), dim3(256), 0, st, h->pool, rows, exit_depth, h->cfg.L_pre, h->cfg.R, h->cfg.max_seqs, h->cfg.max_position, h->status);
     else
-        launch_pdl(copy_on_exit_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, st, h->pool, rows, exit_depth, h->cfg.L_pre, h->cfg.R, h->cfg.max_seqs, h->status);
+        launch_pdl(copy_on_exit_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, st, h->pool, rows, exit_depth, h->cfg.L_pre, h->cfg.R, h->cfg.max_seqs, h->cfg.max_position, h->status);
 }
 
 }  // namespace cdbk

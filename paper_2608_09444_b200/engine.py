@@ -76,6 +76,7 @@ class Engine:
         self.stats = {"recurrent_steps": 0, "row_steps": 0, "coda_calls": 0, "prefill_calls": 0, "tick_rows": [],
                       "rows_hist": [0] * ((max_batch + 31) // 32)}      # recurrent steps by row count, 32-row bins
         self.trace_states = {}                                        # (sid, token index) -> exit state
+        self.trace_step_states = {}                                   # (sid, token index, loop depth) -> state after that loop step
         self.trace_logits = {}
         # Recurrent step as a CUDA graph per row-count bucket (rows padded with seq_id = -1 to a multiple of 32):
         # the descriptor lives in fixed device arrays refreshed by one host-to-device copy per step.
@@ -355,6 +356,12 @@ class Engine:
                 self.stats["tick_rows"].append([(s, len(seqs[s].tokens), r) for s, r in rec])
             for i, (s, r) in enumerate(rec):
                 seqs[s].cur_gates.append(float(gv[i]))
+            if self.record_states:                                    # survivors now lead h_rec, exits fill h_exit
+                hs, he = self.h_rec[:ns].cpu().numpy(), self.h_exit[:ne].cpu().numpy()
+                for j, i in enumerate(surv):
+                    self.trace_step_states[(rec[int(i)][0], len(seqs[rec[int(i)][0]].tokens), rec[int(i)][1])] = hs[j]
+                for j, i in enumerate(ex):
+                    self.trace_step_states[(rec[int(i)][0], len(seqs[rec[int(i)][0]].tokens), rec[int(i)][1])] = he[j]
             if ne:
                 slots = [coda_free.pop() for _ in range(ne)]
                 self.h_coda.index_copy_(0, torch.tensor(slots, dtype=torch.int64, device=self.dev), self.h_exit[:ne])

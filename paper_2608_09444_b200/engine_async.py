@@ -82,8 +82,9 @@ class PipelinedEngine(Engine):
 
     # ------------------------------------------------------------------ generation
     def generate(self, prompts, T, forced_depths=None, teacher_tokens=None, arrivals=None):
-        """Same contract as Engine.generate (teacher tokens are not supported: sampled tokens stay on the
-        device and feed the prelude directly).  Gate values are not read back."""
+        """Same contract as Engine.generate.  Sampled tokens stay on the device and feed the prelude directly;
+        with teacher_tokens (lock-step replay) the given tokens are fed instead, while the sampled ones are
+        still returned.  Gate values are not read back."""
         caller = torch.cuda.current_stream(self.dev)
         self.main.wait_stream(caller)
         with torch.cuda.stream(self.main):
@@ -92,8 +93,6 @@ class PipelinedEngine(Engine):
         return out
 
     def _generate(self, prompts, T, forced_depths, teacher_tokens, arrivals):
-        if teacher_tokens is not None:
-            raise ValueError("lock-step replay needs the synchronous engine")
         dims, cdb, dev = self.dims, self.cdb, self.dev
         main, side = torch.cuda.current_stream(dev), self.side
         n = len(prompts)
@@ -130,6 +129,12 @@ class PipelinedEngine(Engine):
             if forced_depths is not None and forced_depths[s] is not None:
                 return int(forced_depths[s][gen[s] - 1])
             return 0
+
+        def fed_back(sids, sampled):
+            """input tokens of the next pass of sequences sids: the sampled ones (device), or the teacher's"""
+            if teacher_tokens is None:
+                return sampled
+            return i32([teacher_tokens[s][gen[s] - 1] for s in sids])
 
         def drain_tokens(block):
             while pending_tokens and (block or pending_tokens[0][0].query()):
@@ -214,7 +219,7 @@ class PipelinedEngine(Engine):
                     cont.append(j)
             if cont:                                     # boundary calls share one scratch lane: all of them on the side stream
                 with torch.cuda.stream(side):
-                    enqueue_prelude([batch[j] for j in cont], i32(vals[cont]), side, it)
+                    enqueue_prelude([batch[j] for j in cont], fed_back([batch[j] for j in cont], i32(vals[cont])), side, it)
 
         def admit():
             """prompt processing of waiting requests while live slots and pages are free (drains the pipeline)"""
@@ -253,7 +258,7 @@ class PipelinedEngine(Engine):
                     else:
                         cont.append(j)
                 if cont:
-                    enqueue_prelude([batch[j] for j in cont], tok_dev[:m][i64(cont)].contiguous(), main, -1)
+                    enqueue_prelude([batch[j] for j in cont], fed_back([batch[j] for j in cont], tok_dev[:m][i64(cont)].contiguous()), main, -1)
             torch.cuda.synchronize(dev)
 
         def boundary_for(prev, it, force):
@@ -297,7 +302,7 @@ class PipelinedEngine(Engine):
                     else:
                         cont.append(j)
                 if cont:
-                    enqueue_prelude([sids[j] for j in cont], tok_dev[:m][i64(cont)].contiguous(), side, it)
+                    enqueue_prelude([sids[j] for j in cont], fed_back([sids[j] for j in cont], tok_dev[:m][i64(cont)].contiguous()), side, it)
 
         rec, prev, it = [], None, 0
         while True:

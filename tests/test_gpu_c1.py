@@ -249,7 +249,7 @@ def test_c1_fixed_depth_on_the_pipelined_engine_equals_continuous_batching(oracl
 @pytest.mark.parametrize("pipelined", [False, True])
 def test_c1_kv_pool_smaller_than_the_live_set(oracle_runs, pipelined):
     """Eight live slots but pages for only four sequences: admission has to wait for finished sequences to hand
-    their pages back ("prefill up to a KV-cache limit", section 4.1); everything still completes with the oracle's
+    their pages back (section 4.1 admits prompts only while the KV cache has room); everything still completes with the oracle's
     tokens and every page returns to the free list."""
     from paper_2608_09444_b200 import binding as B
     from paper_2608_09444_b200.engine import Engine
