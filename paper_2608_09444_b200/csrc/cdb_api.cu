@@ -138,16 +138,32 @@ void layer_forward_tc(cdb_t* h, int ln, int layer, const RowsDev& rows, float* x
     const size_t d = c.d, F = c.F;
     int& qkv_parts = h->qkv_parts_ready[ln];                    // > 0: the previous layer's launch already left this layer's QKV parts in L.ws
     if (!xn_ready) { launch_rmsnorm(h, x, h->g_attn + (size_t)layer * d, L.xn, rows, st); qkv_parts = 0; }
+    // Split-K parts are summed inside thread-block clusters where that is the faster form (CDB_FLAG_WORKSPACE_PARTS:
+    // always through a workspace and a row-wise kernel; same sums in the same order either way, so a row's result
+    // does not depend on which form its batch took).  Measured on the 2048-wide model: the QKV projection with RoPE
+    // and the KV page write in its epilogue wins up to 128 rows (one launch fewer), the in-cluster residual sums up
+    // to 64 rows (-4 % step time at 64 rows, -7.5 % at 16); at 256 rows the exchange through distributed shared
+    // memory costs as much as the workspace round trip it replaces and the step is 1 % slower.
+    const bool in_cluster = !(c.flags & (CDB_FLAG_WORKSPACE_PARTS | CDB_FLAG_FUSED_STAGES));
+    static const int cluster_mask = tuning_int("CDB_CLUSTER_MASK", 7);       // tuning hook: 1 QKV, 2 output, 4 down projection
+    static const int cluster_rows_qkv = tuning_int("CDB_CLUSTER_ROWS_QKV", 128), cluster_rows_res = tuning_int("CDB_CLUSTER_ROWS_RES", 64);
     {
         ProfScope ps(h, kProfLinear, st);
         int s = qkv_parts;
-        if (!s) {
-            CDB_LAUNCH(h);
-            s = launch_linear_splitk_tc(h, L.xn, layer_ptr(h, h->w.W_qkv, layer, 3 * d * d), L.ws, kWsPerRow / 3, n, 3 * c.d, c.d, st);
-            if (!s) h->launch_error = 1;
+        bool done = false;
+        if (!s && in_cluster && (cluster_mask & 1) && n <= cluster_rows_qkv && !h->prefill_attention) {       // projection, RoPE and KV page write in one launch
+            done = launch_qkv_rope_cluster_tc(h, ln, layer, L.xn, layer_ptr(h, h->w.W_qkv, layer, 3 * d * d), rows, kWsPerRow / 3, st);
+            if (done) CDB_LAUNCH(h);
+        }
+        if (!done) {
+            if (!s) {
+                CDB_LAUNCH(h);
+                s = launch_linear_splitk_tc(h, L.xn, layer_ptr(h, h->w.W_qkv, layer, 3 * d * d), L.ws, kWsPerRow / 3, n, 3 * c.d, c.d, st);
+                if (!s) h->launch_error = 1;
+            }
+            launch_rope_kv_write(h, ln, layer, L.ws, s, (size_t)n * 3 * d, rows, st);      // sums the parts
         }
         qkv_parts = 0;
-        launch_rope_kv_write(h, ln, layer, L.ws, s, (size_t)n * 3 * d, rows, st);      // sums the parts
     }
     if (attn_after) cudaStreamWaitEvent(st, attn_after, 0);      // the other half-batch's attention goes first
     h->attn_split_done = attn_done;
@@ -169,9 +185,12 @@ void layer_forward_tc(cdb_t* h, int ln, int layer, const RowsDev& rows, float* x
     {
         ProfScope ps(h, kProfLinear, st);
         CDB_LAUNCH(h);
-        const int s = launch_linear_splitk_tc(h, L.attn_o, layer_ptr(h, h->w.W_o, layer, d * d), L.ws, kMaxKSplits, n, c.d, c.d, st);
-        if (!s) h->launch_error = 1;
-        launch_reduce_residual_norm(h, L.ws, s, (size_t)n * d, x, h->g_mlp + (size_t)layer * d, L.xn, rows, st);
+        int s = 0;
+        if (!(in_cluster && (cluster_mask & 2) && n <= cluster_rows_res && launch_linear_cluster_residual_tc(h, L.attn_o, layer_ptr(h, h->w.W_o, layer, d * d), x, n, c.d, c.d, kMaxKSplits, st))) {
+            s = launch_linear_splitk_tc(h, L.attn_o, layer_ptr(h, h->w.W_o, layer, d * d), L.ws, kMaxKSplits, n, c.d, c.d, st);
+            if (!s) h->launch_error = 1;
+        }
+        launch_reduce_residual_norm(h, L.ws, s, (size_t)n * d, x, h->g_mlp + (size_t)layer * d, L.xn, rows, st);   // s == 0: the norm alone
     }
     {
         ProfScope ps(h, kProfLinear, st);
@@ -183,9 +202,12 @@ void layer_forward_tc(cdb_t* h, int ln, int layer, const RowsDev& rows, float* x
     {
         ProfScope ps(h, kProfLinear, st);
         CDB_LAUNCH(h);
-        const int s = launch_linear_splitk_tc(h, L.act, layer_ptr(h, h->w.W_down, layer, d * F), L.ws, kMaxKSplits, n, c.d, c.F, st);
-        if (!s) h->launch_error = 1;
-        launch_reduce_residual_norm(h, L.ws, s, (size_t)n * d, x, next_gain, L.xn, rows, st);
+        int s = 0;
+        if (!(in_cluster && (cluster_mask & 4) && n <= cluster_rows_res && launch_linear_cluster_residual_tc(h, L.act, layer_ptr(h, h->w.W_down, layer, d * F), x, n, c.d, c.F, kMaxKSplits, st))) {
+            s = launch_linear_splitk_tc(h, L.act, layer_ptr(h, h->w.W_down, layer, d * F), L.ws, kMaxKSplits, n, c.d, c.F, st);
+            if (!s) h->launch_error = 1;
+        }
+        if (s || next_gain) launch_reduce_residual_norm(h, L.ws, s, (size_t)n * d, x, next_gain, L.xn, rows, st);
     }
 }
 

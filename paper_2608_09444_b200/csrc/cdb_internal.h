@@ -145,6 +145,11 @@ namespace cdbk {
 // still draining; it runs its set-up, then pdl_wait() blocks until the predecessor has completed and
 // its writes are visible.  Every kernel of the library calls pdl_trigger() first (lets ITS successor
 // be scheduled early) and pdl_wait() before its first global-memory access.
+// Rotation of one rotate-half pair (x_i, x_{i+Dh/2}) by the position's angle, with the roundings spelled out so
+// that every kernel that rotates gives the same bits.
+__device__ __forceinline__ float rope_lo(float a1, float a2, float c, float s) { return __fmaf_rn(a1, c, -__fmul_rn(a2, s)); }
+__device__ __forceinline__ float rope_hi(float a1, float a2, float c, float s) { return __fmaf_rn(a2, c, __fmul_rn(a1, s)); }
+
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
@@ -210,6 +215,8 @@ void launch_repack_tiled(const void* W, void* Wt, int layers, int N, int K, cuda
 bool linear_tc_supported(const cdb* h, int n, int N, int K);
 bool launch_gate_up_swiglu_tc(const cdb* h, const void* x, const void* Wg, const void* Wu, void* act, int n, int F, int K, cudaStream_t st);
 int launch_linear_splitk_tc(const cdb* h, const void* x, const void* W, float* ws, int max_splits, int n, int N, int K, cudaStream_t st);
+bool launch_linear_cluster_residual_tc(const cdb* h, const void* xin, const void* W, float* x, int n, int N, int K, int max_splits, cudaStream_t st);
+bool launch_qkv_rope_cluster_tc(const cdb* h, int ln, int layer, const void* xin, const void* W_qkv, const RowsDev& rows, int max_splits, cudaStream_t st);
 int launch_layer_tail_tc(const cdb* h, int ln, const RowsDev& rows, float* x, const void* W_o, const float* g_mlp,
                          const void* W_gate, const void* W_up, const void* W_down, const float* next_gain,
                          const void* W_qkv_next, cudaStream_t st);

@@ -15,6 +15,7 @@
 // CTAs are persistent over (feature tile, row tile) pairs.  Every mbarrier wait is bounded: on
 // expiry the CTA records a status word, lets its outstanding copies land, frees its TMEM and
 // returns.
+#include <cstdio>
 #include <cstdlib>
 
 #include <cuda.h>
@@ -358,6 +359,271 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
 }
 
 // ------------------------------------------------------------------------------------------------------
+// Split-K projection whose parts are summed INSIDE a thread-block cluster.  The k_splits CTAs of a cluster
+// work on the same [128 features x BN rows] output tile, each on its own share of K (the same shares as the
+// split-K launches above, so every part is the same number bit for bit).  Instead of writing fp32 parts to
+// a workspace that a row-wise kernel reads back, the CTAs exchange them through distributed shared memory:
+// the tile's columns (batch rows) are dealt out in chunks of 16 to the CTAs of the cluster, every CTA stores
+// each chunk of its part into the owner's shared memory, and the owner adds the parts in part order.  What
+// the owner does with the finished sums is the mode:
+//   kClusterResidual  x[row][f] += sum            (output and down projections; x + part 0 + part 1 + ...)
+//   kClusterRope      the tile is one head of q, k or v (Dh = 128): q and k are rotated at the row's position,
+//                     q goes to the rotated-query buffer, k and v into the row's KV page (RoPE + KV write)
+// One tile per CTA (no persistence: the cluster is the scheduling unit).  The cluster barriers are reached
+// by every thread on every path (a bounded wait that runs out only skips work), so they cannot hang.
+constexpr int kClusterResidual = 0, kClusterRope = 1;
+
+struct ClusterParams {
+    float* x;                   // residual mode: [n][N] fp32, updated in place
+    int n, N, K, BN, stages, k_splits, w_tiled, mode;
+    // RoPE mode
+    void* qrot;                 // [n][d] bf16
+    KvPool pool;
+    RowsDev rows;
+    int layer, d, max_position, max_seqs;
+    const float* rope_cos;
+    const float* rope_sin;
+    int32_t* status;
+    unsigned long long* dbg;    // tuning builds: per-CTA phase time stamps (NULL = off)
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, uint32_t v) {
+    asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ float4 ld_shared_f4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint2 pack_bf16x4(float a, float b, float c, float d) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+    uint2 v;
+    v.x = *reinterpret_cast<const uint32_t*>(&lo);
+    v.y = *reinterpret_cast<const uint32_t*>(&hi);
+    return v;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, ClusterParams p) {
+    pdl_trigger();
+    auto stamp = [&](int k) { if (kTuningBuild && p.dbg && threadIdx.x == 64) p.dbg[blockIdx.x * 8 + k] = gtime(); };
+    stamp(0);
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bars[2 * 8 + 1];          // full[stages], empty[stages], acc_full
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int S = p.stages, BN = p.BN, KS = p.k_splits;
+    const uint32_t rank = cluster_ctarank();
+    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (8 + s); };
+    const uint32_t acc_full = bar0 + 8u * 16;
+    const uint32_t w_bytes = BM * BK * 2, x_bytes = (uint32_t)BN * BK * 2, stage_bytes = w_bytes + x_bytes;
+    const uint32_t tmem_cols = (uint32_t)BN;
+
+    const int n_ftiles = (p.N + BM - 1) / BM;
+    const int tile = blockIdx.x / KS;
+    const int f0 = (tile % n_ftiles) * BM, r0 = (tile / n_ftiles) * BN;
+    const int n_kb = (p.K + BK - 1) / BK;
+    const int kb0 = (int)((long long)rank * n_kb / KS), nk = (int)((long long)(rank + 1) * n_kb / KS) - kb0;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(acc_full, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+    if (warp != 0) pdl_wait();
+    stamp(1);
+
+    if (warp == 0) {
+        // TMA producer: the weight tiles of the first ring fill go out before the wait for the previous kernel
+        const bool leader = elect_one();
+        const int n_pre = nk < S ? nk : S;
+        auto w_coord = [&](int kb, int& wc, int& wr) { wc = p.w_tiled ? 0 : kb * BK; wr = p.w_tiled ? ((f0 / BM) * n_kb + kb) * BM : f0; };
+        // the k-blocks of a part are taken in the same rotated order as by the workspace form of this projection
+        // (a function of the feature tile only), so that both forms accumulate every part in the same order
+        const int rot = ((tile % n_ftiles) * 7) % nk;
+        auto kb_of = [&](int g) { return kb0 + (g + rot) % nk; };
+        for (int g = 0; g < n_pre; ++g) {
+            int wc, wr; w_coord(kb_of(g), wc, wr);
+            if (leader) { mbar_expect_tx(full_bar(g), stage_bytes); tma_load_2d(ring + (uint32_t)g * stage_bytes, &map_w, full_bar(g), wc, wr); }
+        }
+        __syncwarp();
+        pdl_wait();
+        for (int g = 0; g < n_pre; ++g)
+            if (leader) tma_load_2d(ring + (uint32_t)g * stage_bytes + w_bytes, &map_x, full_bar(g), kb_of(g) * BK, r0);
+        __syncwarp();
+        int s = n_pre % S; uint32_t ph = n_pre == S ? 1u : 0u;
+        for (int g = n_pre; g < nk; ++g) {
+            if (!mbar_wait(empty_bar(s), ph ^ 1u, abortp)) break;
+            int wc, wr; w_coord(kb_of(g), wc, wr);
+            const uint32_t dst = ring + (uint32_t)s * stage_bytes;
+            if (leader) {
+                mbar_expect_tx(full_bar(s), stage_bytes);
+                tma_load_2d(dst, &map_w, full_bar(s), wc, wr);
+                tma_load_2d(dst + w_bytes, &map_x, full_bar(s), kb_of(g) * BK, r0);
+            }
+            __syncwarp();
+            if (++s == S) { s = 0; ph ^= 1u; }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        const bool leader = elect_one();
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+        int s = 0; uint32_t ph = 0;
+        bool ok = true;
+        for (int g = 0; g < nk; ++g) {
+            if (!mbar_wait(full_bar(s), ph, abortp)) { ok = false; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a_addr = ring + (uint32_t)s * stage_bytes;
+            const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(a_addr + w_bytes);
+#pragma unroll
+            for (int k = 0; k < BK / UMMA_K; ++k) {
+                const uint64_t adv = (uint64_t)(k * UMMA_K * 2 >> 4);
+                if (leader) umma_bf16(tmem_base, a_desc + adv, b_desc + adv, idesc, (g > 0 || k > 0) ? 1u : 0u);
+            }
+            __syncwarp();
+            if (leader) umma_commit(empty_bar(s));
+            if (++s == S) { s = 0; ph ^= 1u; }
+        }
+        if (ok && leader) umma_commit(acc_full);
+        __syncwarp();
+    } else {
+        mbar_wait(acc_full, 0u, abortp);                   // this CTA's part is complete in TMEM (or the wait gave up)
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        stamp(2);
+    }
+    __syncwarp();
+    // Every CTA of the cluster has finished reading its ring: the rings now serve as receive buffers.
+    cluster_sync_all();
+    stamp(3);
+
+    const int n_real = min(BN, p.n - r0);                   // columns of the tile that hold real rows
+    const int n_chunks = (n_real + 15) / 16;                // 16-column chunks; chunk i belongs to CTA i % KS
+    const bool healthy = *abortp == 0;
+    if (warp >= 2 && healthy) {
+        const int q = warp & 3, half = (warp - 2) >> 2;     // TMEM lane quarter; even or odd chunks
+        const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+        const uint32_t f_off = (uint32_t)(q * 32 + lane) * 4u;
+        uint32_t v[2][16];                                 // the next chunk's TMEM load flies while this one is sent
+        if (half < n_chunks) tmem_ld16(t_addr + (uint32_t)(half * 16), v[0]);
+#pragma unroll 1
+        for (int i0 = half; i0 < n_chunks; i0 += 4) {
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const int i = i0 + 2 * hh;
+                if (i >= n_chunks) break;
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (i + 2 < n_chunks) tmem_ld16(t_addr + (uint32_t)((i + 2) * 16), v[hh ^ 1]);
+                const uint32_t owner = (uint32_t)(i % KS), li = (uint32_t)(i / KS);
+                const uint32_t dst = map_to_cta(ring + ((li * (uint32_t)KS + rank) * 16u) * (BM * 4u) + f_off, owner);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) st_cluster_f32(dst + (uint32_t)j * (BM * 4u), v[hh][j]);
+            }
+        }
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+    __syncwarp();
+    stamp(4);
+    // All parts have arrived in their owners' shared memory.
+    cluster_sync_all();
+    stamp(5);
+
+    if (warp >= 2 && healthy) {
+        const int et = threadIdx.x - 64;                    // 0..255
+        for (int i = (int)rank; i < n_chunks; i += KS) {
+            const uint32_t li = (uint32_t)(i / KS);
+            const uint32_t chunk = ring + (li * (uint32_t)KS * 16u) * (BM * 4u);      // [part][16 columns][128 features]
+            if (p.mode == kClusterResidual) {
+                for (int idx = et; idx < 16 * (BM / 4); idx += kEpiThreads) {
+                    const int j = idx / (BM / 4), f4 = idx % (BM / 4);
+                    const int row = r0 + 16 * i + j, f = f0 + 4 * f4;
+                    if (row >= p.n || f >= p.N) continue;
+                    float4* dst = reinterpret_cast<float4*>(p.x + (size_t)row * p.N + f);
+                    float4 a = __ldcg(dst);
+                    for (int sp = 0; sp < KS; ++sp) {         // fixed order: x + part 0 + part 1 + ...
+                        const float4 b = ld_shared_f4(chunk + (((uint32_t)sp * 16u + (uint32_t)j) * BM + 4u * (uint32_t)f4) * 4u);
+                        a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+                    }
+                    *dst = a;
+                }
+            } else {
+                // the tile is head `hd` of q (which = 0), k (1) or v (2); pairs (i, i + 64) are rotated
+                const int which = f0 / p.d, hd = (f0 % p.d) / BM;
+                for (int idx = et; idx < 16 * 16; idx += kEpiThreads) {
+                    const int j = idx / 16, i4 = (idx % 16) * 4;
+                    const bool reporter = i4 == 0 && hd == 0;
+                    const int row = r0 + 16 * i + j;
+                    if (row >= p.n) continue;
+                    const int seq = p.rows.seq_id[row];
+                    if (seq < 0) continue;
+                    const int pos = p.rows.position[row], slot = p.rows.slot_of(row);
+                    if (seq >= p.max_seqs || slot < 0 || slot >= p.rows.n_slots) { if (reporter && which == 0) atomicCAS(p.status, 0, kStatusSeq); continue; }
+                    if (pos < 0 || pos >= p.max_position || pos / kPageSize >= p.rows.page_table_stride) {
+                        if (reporter && which == 0) atomicCAS(p.status, 0, kStatusPosition);
+                        continue;
+                    }
+                    const uint32_t at = chunk + ((uint32_t)j * BM + (uint32_t)i4) * 4u;
+                    float4 a1 = ld_shared_f4(at), a2 = ld_shared_f4(at + 64u * 4u);
+                    for (int sp = 1; sp < KS; ++sp) {         // fixed order: part 0 + part 1 + ...
+                        const float4 b1 = ld_shared_f4(at + (uint32_t)sp * 16u * BM * 4u), b2 = ld_shared_f4(at + (uint32_t)sp * 16u * BM * 4u + 64u * 4u);
+                        a1.x += b1.x; a1.y += b1.y; a1.z += b1.z; a1.w += b1.w;
+                        a2.x += b2.x; a2.y += b2.y; a2.z += b2.z; a2.w += b2.w;
+                    }
+                    __nv_bfloat16* dst;
+                    if (which == 0) {
+                        dst = (__nv_bfloat16*)p.qrot + (size_t)row * p.d + (size_t)hd * BM;
+                    } else {
+                        const int page = p.rows.page_table[((size_t)seq * p.rows.n_slots + slot) * p.rows.page_table_stride + pos / kPageSize];
+                        if (page < 0 || page >= p.pool.n_phys_pages) { if (reporter && which == 1) atomicCAS(p.status, 0, kStatusPage); continue; }
+                        dst = (__nv_bfloat16*)p.pool.base + p.pool.tile_offset(p.layer, page, which - 1, hd) + (size_t)(pos % kPageSize) * BM;
+                    }
+                    if (which < 2) {
+                        const float4 c = *reinterpret_cast<const float4*>(p.rope_cos + (size_t)pos * 64 + i4);
+                        const float4 sv = *reinterpret_cast<const float4*>(p.rope_sin + (size_t)pos * 64 + i4);
+                        *reinterpret_cast<uint2*>(dst + i4) = pack_bf16x4(rope_lo(a1.x, a2.x, c.x, sv.x), rope_lo(a1.y, a2.y, c.y, sv.y), rope_lo(a1.z, a2.z, c.z, sv.z), rope_lo(a1.w, a2.w, c.w, sv.w));
+                        *reinterpret_cast<uint2*>(dst + 64 + i4) = pack_bf16x4(rope_hi(a1.x, a2.x, c.x, sv.x), rope_hi(a1.y, a2.y, c.y, sv.y), rope_hi(a1.z, a2.z, c.z, sv.z), rope_hi(a1.w, a2.w, c.w, sv.w));
+                    } else {
+                        *reinterpret_cast<uint2*>(dst + i4) = pack_bf16x4(a1.x, a1.y, a1.z, a1.w);
+                        *reinterpret_cast<uint2*>(dst + 64 + i4) = pack_bf16x4(a2.x, a2.y, a2.z, a2.w);
+                    }
+                }
+            }
+        }
+    }
+    stamp(6);
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag) atomicCAS(p.status, 0, kStatusTimeout);
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------
 // Several dependent stages of a layer in ONE launch (opt-in, CDB_FLAG_FUSED_STAGES): projections (as above)
 // and the row-wise "sum the split-K parts + residual + RMSNorm" step, separated by grid-wide barriers instead
 // of kernel boundaries; the producer warp starts the NEXT projection's weight copies before it waits at the
@@ -650,7 +916,7 @@ static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* 
     if (!n_tiles) return false;
 #ifdef CDB_TUNING
     // tuning hook: device address of a stamp buffer (8 words per CTA), optionally for one launch kind only
-    p.dbg = getenv("CDB_GEMM_DBG") ? (unsigned long long*)strtoull(getenv("CDB_GEMM_DBG"), nullptr, 0) : nullptr;
+    p.dbg = getenv("CDB_GEMM_DBG") && !getenv("CDB_GEMM_DBG_CLUSTER") ? (unsigned long long*)strtoull(getenv("CDB_GEMM_DBG"), nullptr, 0) : nullptr;
     if (getenv("CDB_GEMM_DBG_ONLY") && atoi(getenv("CDB_GEMM_DBG_ONLY")) != mode * 100000 + N) p.dbg = nullptr;
 #endif
     static const int part_sms = tuning_int("CDB_GEMM_SMS", 0);      // tuning hook (two-stream step only): CTA count of a projection
@@ -660,9 +926,35 @@ static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* 
     return true;
 }
 
-// Part count of a split-K projection.  It depends on the weight's shape alone, never on the number of rows,
-// so that a row's result does not depend on the batch it is computed in: at most one tile per SM for a batch
-// that fills one row tile, and at least four k-blocks per part.
+// How many clusters of `size` CTAs of the cluster projection kernel can be resident at once on the handle's device
+// (each CTA takes a whole SM, and a cluster must fit inside one GPC); 0 when such clusters cannot be launched.
+// Asked once per device and size.
+static int cluster_fit(const cdb* h, int size) {
+    static int fit[kMaxDevices][kMaxKSplits + 1] = {};          // 0 = not asked yet, -1 = unavailable
+    if (size < 1 || size > kMaxKSplits) return 0;
+    int& f = fit[h->device][size];
+    if (f == 0) {
+        f = -1;
+        if (cudaFuncSetAttribute(gemm_splitk_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) == cudaSuccess) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(size * 64); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = kMaxSmem;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = size; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr; cfg.numAttrs = 1;
+            int nc = 0;
+            if (cudaOccupancyMaxActiveClusters(&nc, gemm_splitk_cluster_kernel, &cfg) == cudaSuccess && nc > 0) f = nc;
+            else cudaGetLastError();
+            if (kTuningBuild) fprintf(stderr, "cluster projection: %d clusters of %d fit\n", nc, size);
+        }
+    }
+    return f > 0 ? f : 0;
+}
+
+// Part count of a split-K projection.  It depends on the weight's shape (and the device) alone, never on the
+// number of rows, so that a row's result does not depend on the batch it is computed in: at most one tile per SM
+// for a batch that fills one row tile, at least four k-blocks per part, and - so that the parts can be summed
+// inside thread-block clusters - no more parts than let one cluster per feature tile be resident at once.
 static int splitk_parts(const cdb* h, int N, int K, int max_splits) {
     const int sms = h->sms;
     const int n_ft = (N + BM - 1) / BM, n_kb = (K + BK - 1) / BK;
@@ -670,6 +962,8 @@ static int splitk_parts(const cdb* h, int N, int K, int max_splits) {
     if (splits > n_kb / 4) splits = n_kb / 4;
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
+    if (!(h->cfg.flags & CDB_FLAG_FUSED_STAGES))
+        while (splits > 1 && cluster_fit(h, splits) > 0 && cluster_fit(h, splits) < n_ft) --splits;
     return splits;
 }
 
@@ -687,6 +981,68 @@ bool launch_gate_up_swiglu_tc(const cdb* h, const void* x, const void* Wg, const
 int launch_linear_splitk_tc(const cdb* h, const void* x, const void* W, float* ws, int max_splits, int n, int N, int K, cudaStream_t st) {
     const int splits = splitk_parts(h, N, K, max_splits);
     return launch_gemm(h, x, W, nullptr, ws, nullptr, n, N, K, kModeStore, splits, (size_t)n * N, st) ? splits : 0;
+}
+
+// ---- split-K projections summed inside thread-block clusters -------------------------------------------
+namespace {
+
+// Fills the shape-dependent fields and launches.  false: the cluster form is not available for this shape on
+// this device (the caller then takes the workspace path); nothing was launched.
+bool launch_cluster_gemm(const cdb* h, const void* xin, const void* W, int n, int N, int K, int max_splits, ClusterParams& p, cudaStream_t st) {
+    if (n < 1 || N % 4 != 0) return false;
+    const int KS = splitk_parts(h, N, K, max_splits);
+    if (KS < 1 || KS > kMaxKSplits) return false;
+    p.n = n; p.N = N; p.K = K; p.k_splits = KS;
+    p.BN = n <= 64 ? 64 : n <= 128 ? 128 : 256;
+    // every cluster of the launch resident at once, or the workspace form (whose CTAs are persistent) does it
+    if (((N + BM - 1) / BM) * ((n + p.BN - 1) / p.BN) > cluster_fit(h, KS)) return false;
+    const int stage_bytes = BM * BK * 2 + p.BN * BK * 2;
+    p.stages = (kMaxSmem - 1024) / stage_bytes;
+    if (p.stages > 8) p.stages = 8;
+    // the ring doubles as the receive buffer: [chunks owned][parts][16 columns][128 features] fp32
+    const int chunks = p.BN / 16, owned = (chunks + KS - 1) / KS;
+    if ((size_t)owned * KS * 16 * BM * 4 > (size_t)p.stages * stage_bytes) return false;
+    p.status = h->status;
+    const int n_ft = (N + BM - 1) / BM, n_kb = (K + BK - 1) / BK;
+    const void* Wt = find_tiled(h, W, N, K);
+    p.w_tiled = Wt ? 1 : 0;
+    CUtensorMap map_w, map_x;
+    if (Wt ? !make_map(&map_w, Wt, n_ft * n_kb * BM, BK, BM) : !make_map(&map_w, W, N, K, BM)) return false;
+    if (!make_map(&map_x, xin, n, K, p.BN)) return false;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_ft * ((n + p.BN - 1) / p.BN) * KS); cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = (size_t)p.stages * stage_bytes + 1024; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = KS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 2;
+#ifdef CDB_TUNING
+    p.dbg = getenv("CDB_GEMM_DBG") ? (unsigned long long*)strtoull(getenv("CDB_GEMM_DBG"), nullptr, 0) : nullptr;
+#endif
+    return cudaLaunchKernelEx(&cfg, gemm_splitk_cluster_kernel, map_w, map_x, p) == cudaSuccess;
+}
+
+}  // namespace
+
+// x[n][N] += xin[n][K] . W[N][K]^T, the split-K parts added in part order on top of x.
+bool launch_linear_cluster_residual_tc(const cdb* h, const void* xin, const void* W, float* x, int n, int N, int K, int max_splits, cudaStream_t st) {
+    ClusterParams p = {};
+    p.mode = kClusterResidual;
+    p.x = x;
+    return launch_cluster_gemm(h, xin, W, n, N, K, max_splits, p, st);
+}
+
+// QKV projection of one layer with RoPE and the KV page write in its epilogue (heads of 128 only).
+bool launch_qkv_rope_cluster_tc(const cdb* h, int ln, int layer, const void* xin, const void* W_qkv, const RowsDev& rows, int max_splits, cudaStream_t st) {
+    const cdb_config_t& c = h->cfg;
+    if (c.Dh != BM || c.d % BM != 0 || c.dtype != CDB_BF16) return false;
+    ClusterParams p = {};
+    p.mode = kClusterRope;
+    p.qrot = h->lane[ln].qrot; p.pool = h->pool; p.rows = rows; p.layer = layer; p.d = c.d;
+    p.max_position = c.max_position; p.max_seqs = c.max_seqs; p.rope_cos = h->rope_cos; p.rope_sin = h->rope_sin;
+    return launch_cluster_gemm(h, xin, W_qkv, rows.n_rows, 3 * c.d, c.d, max_splits, p, st);
 }
 
 // Everything of a layer after its attention in one cooperative launch: output projection (split-K) ->

@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(256) reduce_residual_norm_kernel(const float* 
                 const float4 b = __ldcg(reinterpret_cast<const float4*>(ws + (size_t)s * split_stride) + at);
                 a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
             }
-            reinterpret_cast<float4*>(x)[at] = a;
+            if (splits > 0) reinterpret_cast<float4*>(x)[at] = a;
             v[k] = a;
             ss = fmaf(a.x, a.x, fmaf(a.y, a.y, fmaf(a.z, a.z, fmaf(a.w, a.w, ss))));
         }
@@ -177,12 +177,12 @@ __global__ void __launch_bounds__(256) rope_kv_write_kernel(const float* __restr
         const int e = hd * Dh + i;
         const float4 q1 = val4(e), q2 = val4(e + half), k1 = val4(d + e), k2 = val4(d + e + half);
         const float4 v1 = val4(2 * d + e), v2 = val4(2 * d + e + half);
-        store4<T>(qrot + (size_t)row * d + e, q1.x * c.x - q2.x * s.x, q1.y * c.y - q2.y * s.y, q1.z * c.z - q2.z * s.z, q1.w * c.w - q2.w * s.w);
-        store4<T>(qrot + (size_t)row * d + e + half, q2.x * c.x + q1.x * s.x, q2.y * c.y + q1.y * s.y, q2.z * c.z + q1.z * s.z, q2.w * c.w + q1.w * s.w);
+        store4<T>(qrot + (size_t)row * d + e, rope_lo(q1.x, q2.x, c.x, s.x), rope_lo(q1.y, q2.y, c.y, s.y), rope_lo(q1.z, q2.z, c.z, s.z), rope_lo(q1.w, q2.w, c.w, s.w));
+        store4<T>(qrot + (size_t)row * d + e + half, rope_hi(q1.x, q2.x, c.x, s.x), rope_hi(q1.y, q2.y, c.y, s.y), rope_hi(q1.z, q2.z, c.z, s.z), rope_hi(q1.w, q2.w, c.w, s.w));
         T* kt = base + pool.tile_offset(layer, page, 0, hd) + (size_t)(pos % kPageSize) * Dh;
         T* vt = base + pool.tile_offset(layer, page, 1, hd) + (size_t)(pos % kPageSize) * Dh;
-        store4<T>(kt + i, k1.x * c.x - k2.x * s.x, k1.y * c.y - k2.y * s.y, k1.z * c.z - k2.z * s.z, k1.w * c.w - k2.w * s.w);
-        store4<T>(kt + i + half, k2.x * c.x + k1.x * s.x, k2.y * c.y + k1.y * s.y, k2.z * c.z + k1.z * s.z, k2.w * c.w + k1.w * s.w);
+        store4<T>(kt + i, rope_lo(k1.x, k2.x, c.x, s.x), rope_lo(k1.y, k2.y, c.y, s.y), rope_lo(k1.z, k2.z, c.z, s.z), rope_lo(k1.w, k2.w, c.w, s.w));
+        store4<T>(kt + i + half, rope_hi(k1.x, k2.x, c.x, s.x), rope_hi(k1.y, k2.y, c.y, s.y), rope_hi(k1.z, k2.z, c.z, s.z), rope_hi(k1.w, k2.w, c.w, s.w));
         store4<T>(vt + i, v1.x, v1.y, v1.z, v1.w);
         store4<T>(vt + i + half, v2.x, v2.y, v2.z, v2.w);
     }

@@ -120,7 +120,7 @@ def main():
         dims, seed = synth.HUGINN_3P5B, 3
     if args.layers:
         dims = dims.replace(L_core=args.layers)
-    w = synth.make_weights(dims, seed, device="cuda:0", gate_std=2.0 / np.sqrt(dims.d))
+    w = synth.make_weights(dims, seed, device="cuda:0", std=synth.width_scaled_std(dims.d), gate_std=2.0 / np.sqrt(dims.d))
     prompts = list(synth.make_prompts(args.seqs, args.prompt, dims.V, seed))
     report = {"model": args.model, "dims": {"d": dims.d, "H": dims.H, "Dh": dims.Dh, "F": dims.F, "V": dims.V,
                                             "layers": [dims.L_pre, dims.L_core, dims.L_coda], "R": dims.R},

@@ -117,7 +117,7 @@ def main():
         dist.init_process_group("nccl")
     torch.cuda.set_device(local_rank)
     dims, seed = (synth.OURO_1P4B, 4) if args.model == "ouro" else (synth.HUGINN_3P5B, 5)
-    w = synth.make_weights(dims, seed, device=f"cuda:{local_rank}", gate_std=2.0 / np.sqrt(dims.d))
+    w = synth.make_weights(dims, seed, device=f"cuda:{local_rank}", std=synth.width_scaled_std(dims.d), gate_std=2.0 / np.sqrt(dims.d))
     report = {"model": args.model, "requests": args.requests, "runs": []}
     if args.model == "ouro":
         gate_kind = B.GATE_SIGMOID_CDF

@@ -56,7 +56,7 @@ def sweep(dims, batches, lengths, *, pool_tokens, warmup=3, steps=10, seed=7, de
     max_rows, max_len = max(batches), max(lengths)
     width = (max_len + dims.page_size - 1) // dims.page_size
     n_pages = (pool_tokens + dims.page_size - 1) // dims.page_size
-    weights = synth.make_weights(dims, seed, device=str(dev), std=0.02, gate_std=2.0 / np.sqrt(dims.d))
+    weights = synth.make_weights(dims, seed, device=str(dev), std=synth.width_scaled_std(dims.d), gate_std=2.0 / np.sqrt(dims.d))
     cdb = B.Cdb(dims, weights, max_rows=max_rows, max_seqs=max_rows, max_position=width * dims.page_size,
                 gate_kind=B.GATE_SIGMOID_CDF, q_or_eps=0.5, flags=flags)
     dt = torch.float32 if dims.dtype == "fp32" else torch.bfloat16

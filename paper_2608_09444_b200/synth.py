@@ -114,6 +114,12 @@ def make_weights(dims: Dims, seed: int, device: str = "cpu", std: float = 0.02,
     return out
 
 
+def width_scaled_std(d: int, base: float = 0.02, base_width: int = 2048) -> float:
+    """Weight scale that keeps the gain of a layer (std * sqrt(d)) at that of a `base_width`-wide layer drawn at
+    `base`: random-init stand-in for models wider than the 2048-wide one."""
+    return base * math.sqrt(base_width / d)
+
+
 def weights_to_numpy(w: dict[str, torch.Tensor]) -> dict[str, np.ndarray]:
     """Host fp32 copies (exact for bf16 storage) for the CPU oracle."""
     return {k: v.detach().to("cpu", torch.float32).numpy() for k, v in w.items()}

@@ -16,10 +16,10 @@ from . import synth
 
 class LoopStepWorkload:
     def __init__(self, dims=synth.OURO_1P4B, n_rows=256, seed=1, ctx_lo=128, ctx_hi=2048, permute=True,
-                 p_fire=0.3, device="cuda:0", flags=0, weight_std=0.02):
+                 p_fire=0.3, device="cuda:0", flags=0, weight_std=None):
         self.dims, self.n_rows, self.dev = dims, n_rows, torch.device(device)
         torch.cuda.set_device(self.dev)
-        self.weights = synth.make_weights(dims, seed, device=str(self.dev), std=weight_std, gate_std=2.0 / np.sqrt(dims.d))
+        self.weights = synth.make_weights(dims, seed, device=str(self.dev), std=weight_std or synth.width_scaled_std(dims.d), gate_std=2.0 / np.sqrt(dims.d))
         self.rows_np = synth.make_step_rows(n_rows, dims.R, seed, ctx_lo, ctx_hi, p_fire)
         self.ctx = self.rows_np["position"].astype(np.int64) + 1
         self.table_np, self.n_pages = synth.make_page_table(self.ctx, dims.page_size, seed, permute=permute)

@@ -106,7 +106,7 @@ def test_range_errors_are_reported_not_faulted():
     assert "max_rows" in str(e.value) or "rows" in str(e.value)
 
 
-@pytest.mark.parametrize("flags,extra", [(0, 0), (4, 0), (0, 70), (0, 200), (16, 0), (16, 200)])
+@pytest.mark.parametrize("flags,extra", [(0, 0), (4, 0), (0, 70), (0, 200), (16, 0), (16, 200), (32, 0), (32, 200)])
 def test_a_rows_result_does_not_depend_on_its_batch(flags, extra):
     """Run nine rows together, then three of them alone, as a pair in another order and among pads: hidden
     states, gate values, exit signals and the K/V written must be identical bit for bit (shape-only split-K
@@ -149,6 +149,59 @@ def test_a_rows_result_does_not_depend_on_its_batch(flags, extra):
             assert np.array_equal(hh, full[i][0]), (subset, i)
             assert np.array_equal(gg, full[i][1]) and ff == full[i][2], (subset, i)
             assert np.array_equal(kv, full[i][3]), (subset, i)
+
+
+WIDE = synth.Dims(V=64, d=1024, H=8, Dh=128, F=2816, L_pre=0, L_core=2, L_coda=0, R=4, dtype="bf16")
+
+
+@pytest.mark.parametrize("n_rows", [9, 79, 209, 300])
+def test_in_cluster_sums_equal_workspace_sums_and_do_not_depend_on_the_batch(n_rows):
+    """A model wide enough for real split-K (4 parts for the QKV and output projections, 8 for the down projection).
+    Default flow: the parts are summed inside thread-block clusters, with RoPE and the KV page write in the QKV
+    projection's epilogue.  Cross-check flow (flag 32): the parts go through a workspace and row-wise kernels.
+    Both add the same parts in the same order, so states, gate values, exit signals and the K/V written must agree
+    bit for bit - between the flows, and between a full batch (one to two 256-row tiles, ragged) and subsets."""
+    ctxs = [1, 16, 17, 40, 255, 256, 257, 300, 33] + [int(c) for c in np.random.default_rng(2).integers(1, 90, n_rows - 9)]
+    n = len(ctxs)
+    rng = np.random.default_rng(1)
+    h_np = rng.standard_normal((n, WIDE.d)).astype(np.float32)
+    depth = rng.integers(1, WIDE.R + 1, n)
+    results = {}
+    for flags in (0, 32):
+        B, cdb, _, table_np, pool, pool_np = setup(ctxs, max_rows=n, dims=WIDE, flags=flags)
+        table = dev(table_np)
+
+        def run(idx):
+            pool.copy_(dev(pool_np, torch.bfloat16))
+            seq = [int(i) if i >= 0 else -1 for i in idx]
+            pos = [ctxs[i] - 1 if i >= 0 else 0 for i in idx]
+            dep = [int(depth[i]) if i >= 0 else 1 for i in idx]
+            rows = B.Rows(i32(seq), i32(pos), table, loop_depth=i32(dep), kv_slot=i32([0] * len(idx)))
+            cdb.boundary_embed(i32([0] * len(idx)), rows, torch.zeros((len(idx), WIDE.d), device="cuda"))
+            h = dev(np.stack([h_np[i] if i >= 0 else np.zeros(WIDE.d, np.float32) for i in idx]))
+            gate, fire = torch.zeros(len(idx), device="cuda"), torch.zeros(len(idx), dtype=torch.uint8, device="cuda")
+            cdb.loop_step(rows, h, gate, fire)
+            torch.cuda.synchronize()
+            assert cdb.poll_status() == 0 and cdb.check_guards() == 0
+            out = {}
+            pl = pool.view(torch.int16).cpu().numpy()
+            for j, i in enumerate(idx):
+                if i >= 0:
+                    page, off = table_np[i, (ctxs[i] - 1) // 16], (ctxs[i] - 1) % 16
+                    out[i] = (h[j].cpu().numpy().view(np.int32), gate[j].cpu().numpy().view(np.int32), int(fire[j]),
+                              pl[:, page, :, :, off, :].copy())
+            return out
+
+        results[flags] = [run(list(range(n)))] + [run(sub) for sub in ([4], [7, 4], [-1, 5, -1, 2], list(range(8, min(n, 75))))]
+        cdb.destroy()
+    full = results[0][0]
+    assert all(np.isfinite(v[0].view(np.float32)).all() for v in full.values())
+    for flags in (0, 32):
+        for part in results[flags]:
+            for i, (hh, gg, ff, kv) in part.items():
+                assert np.array_equal(kv, full[i][3]), (flags, i, "K/V")
+                assert np.array_equal(hh, full[i][0]), (flags, i, "state")
+                assert np.array_equal(gg, full[i][1]) and ff == full[i][2], (flags, i, "gate")
 
 
 def test_host_checks_refuse_bad_calls_with_an_error_code():
