@@ -114,6 +114,11 @@ typedef struct {
                                         of logical page j of (seq_id, kv_slot), row seq_id*n_slots+kv_slot */
     int32_t        page_table_stride; /* a row whose position needs logical page >= page_table_stride is skipped
                                         (no KV write, zero attention output) and reported as status 2 */
+    const int32_t* n_rows_dev;       /* device int32 [1] or NULL.  When given, only the first *n_rows_dev rows are live:
+                                        every row at an index >= *n_rows_dev is a pad whatever its seq_id says.  n_rows
+                                        stays the host-side capacity of the call (launch shapes follow it), so one
+                                        recorded launch sequence - a CUDA graph - serves every batch size up to n_rows
+                                        (the static shapes of section 4.3) */
 } cdb_rows_t;
 
 /* Creates a handle for one model on the current CUDA device.  Allocates scratch for max_rows

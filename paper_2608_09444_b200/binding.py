@@ -50,7 +50,7 @@ class Weights(C.Structure):
 class RowsStruct(C.Structure):
     _fields_ = [("n_rows", C.c_int32), ("seq_id", C.c_void_p), ("loop_depth", C.c_void_p), ("position", C.c_void_p),
                 ("kv_slot", C.c_void_p), ("forced_exit", C.c_void_p), ("page_table", C.c_void_p),
-                ("page_table_stride", C.c_int32)]
+                ("page_table_stride", C.c_int32), ("n_rows_dev", C.c_void_p)]
 
 
 class Profile(C.Structure):
@@ -118,15 +118,17 @@ def paged_attention_static(q, o, pool, layer, seq_id, position, page_table, max_
 class Rows:
     """Row descriptor of one call: device int32 tensors (see cdb_rows_t)."""
 
-    def __init__(self, seq_id, position, page_table, loop_depth=None, kv_slot=None, forced_exit=None, n_rows=None):
+    def __init__(self, seq_id, position, page_table, loop_depth=None, kv_slot=None, forced_exit=None, n_rows=None,
+                 n_rows_dev=None):
         self.seq_id, self.position, self.page_table = seq_id, position, page_table
         self.loop_depth, self.kv_slot, self.forced_exit = loop_depth, kv_slot, forced_exit
+        self.n_rows_dev = n_rows_dev                    # device int32 [1]: live rows (the rest are pads), or None
         self.n_rows = int(seq_id.shape[0]) if n_rows is None else int(n_rows)
-        for t in (seq_id, position, page_table, loop_depth, kv_slot, forced_exit):
+        for t in (seq_id, position, page_table, loop_depth, kv_slot, forced_exit, n_rows_dev):
             if t is not None and t.dtype != torch.int32:
                 raise TypeError("row descriptor tensors must be int32")
         self.struct = RowsStruct(self.n_rows, _ptr(seq_id), _ptr(loop_depth), _ptr(position), _ptr(kv_slot),
-                                 _ptr(forced_exit), _ptr(page_table), int(page_table.shape[-1]))
+                                 _ptr(forced_exit), _ptr(page_table), int(page_table.shape[-1]), _ptr(n_rows_dev))
 
     @property
     def ref(self):

@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(1024) attn_plan_kernel(RowsDev rows, int32_t* 
     for (int start = 0; start < rows.n_rows; start += 1024) {
         const int row = start + threadIdx.x;
         int ns = 0;
-        if (row < rows.n_rows && rows.seq_id[row] >= 0) {
+        if (row < rows.n_rows && rows.seq_of(row) >= 0) {
             const int pos = rows.position[row];
             if (pos >= max_position || (pos >= 0 && pos / kPageSize >= rows.page_table_stride)) atomicCAS(status, 0, kStatusPosition);
             else if (pos >= 0) ns = min((pos + kSplitTokens) / kSplitTokens, max_splits);      // ceil((pos+1)/split)
@@ -129,7 +129,7 @@ __global__ void __maxnreg__(LAT ? 208 : 96) attn_split_kernel(AttnParams p) {
         int lo = 0, hi = n_rows;                 // last row with item_start[row] <= pair
         while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (p.item_start[mid] <= pair) lo = mid; else hi = mid; }
         const int row = lo, split = pair - p.item_start[lo];
-        const int seq = p.rows.seq_id[row];
+        const int seq = p.rows.seq_of(row);
         const int slot = p.rows.slot_of(row);
         const int ctx = p.rows.position[row] + 1;
         float* part = p.part + ((size_t)(row * H + head) * p.max_splits + split) * (DH + 2);
@@ -271,7 +271,7 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(AttnParams p, T* __rest
     T* o = out + (size_t)row * H * DH + (size_t)head * DH;
     constexpr int PER = (DH + 31) / 32;
     const int ns = min(p.item_start[row + 1] - p.item_start[row], p.max_splits);
-    const int sq = p.rows.seq_id[row];
+    const int sq = p.rows.seq_of(row);
     if (sq < 0 || sq >= p.max_seqs || ns <= 0) {          // pads and rows the plan or the split kernel skipped
 #pragma unroll
         for (int k = 0; k < PER; ++k) if (lane + 32 * k < DH) o[lane + 32 * k] = T(0.f);
@@ -427,7 +427,7 @@ __global__ void attn_static_plan_kernel(RowsDev rows, int max_splits, int max_co
     for (int row = 0; row < rows.n_rows; ++row) {
         item_start[row] = acc;
         const int pos = rows.position[row];
-        if (rows.seq_id[row] < 0 || pos < 0) continue;
+        if (rows.seq_of(row) < 0 || pos < 0) continue;
         if (rows.seq_id[row] >= max_seqs) { *status = kStatusSeq; continue; } // no table row: skipped, output zeroed
         if (pos >= max_context) { *status = kStatusPosition; continue; }      // beyond the stated bound: row skipped
         const int ns = (pos + kSplitTokens) / kSplitTokens;
@@ -488,7 +488,7 @@ extern "C" int cdb_paged_attention_static(const void* q, void* o, const void* po
     p.pool.base = const_cast<void*>(pool); p.pool.n_phys_pages = n_phys_pages; p.pool.H = H; p.pool.Dh = Dh;
     p.rows.n_rows = n_rows; p.rows.seq_id = seq_id; p.rows.loop_depth = nullptr; p.rows.position = position;
     p.rows.kv_slot = nullptr; p.rows.forced_exit = nullptr; p.rows.page_table = page_table;
-    p.rows.page_table_stride = page_table_stride; p.rows.n_slots = 1; p.rows.slot_override = 0;
+    p.rows.page_table_stride = page_table_stride; p.rows.n_slots = 1; p.rows.slot_override = 0; p.rows.n_live = nullptr;
     p.layer = layer; p.max_splits = max_splits; p.max_seqs = max_seqs;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)Dh);
     p.status = (int32_t*)base; p.counter = (int32_t*)(base + 4);
@@ -536,12 +536,12 @@ __global__ void __launch_bounds__(1024) prefill_plan_kernel(RowsDev rows, int ti
         const int r = base + tid;
         bool valid = false, start = false;
         if (r < rows.n_rows) {
-            const int sq = rows.seq_id[r];
+            const int sq = rows.seq_of(r);
             valid = sq >= 0;
             if (valid) {
                 start = r == 0;
                 if (!start) {
-                    const int sp = rows.seq_id[r - 1];
+                    const int sp = rows.seq_of(r - 1);
                     start = sp != sq || rows.position[r] != rows.position[r - 1] + 1;
                 }
             }
@@ -592,7 +592,7 @@ __global__ void __launch_bounds__(128) attn_prefill_kernel(AttnParams p, const i
     const int qi = threadIdx.x >> 2, part = threadIdx.x & 3;           // query in tile, quarter of the head dim
     const bool active = qi < nq;
     const int row = row0 + (active ? qi : 0);
-    const int seq = p.rows.seq_id[row0];
+    const int seq = p.rows.seq_of(row0);
     const int slot = p.rows.slot_of(row0);
     const int pos = p.rows.position[row];
     const int pos_last = p.rows.position[row0 + nq - 1];

@@ -106,7 +106,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
             const int tile = item_tile(it), head = it % H;
             const int row0 = p.tiles[tile], nq = p.tile_rows[tile];
-            const int seq = p.rows.seq_id[row0], slot = p.rows.slot_of(row0);
+            const int seq = p.rows.seq_of(row0), slot = p.rows.slot_of(row0);
             const int pos_last = p.rows.position[row0 + nq - 1];
             if (seq < 0 || seq >= p.max_seqs || slot < 0 || slot >= p.rows.n_slots || pos_last < 0 || pos_last / kPageSize >= p.rows.page_table_stride) continue;   // flagged by the softmax warps
             const int32_t* table = p.rows.page_table + ((size_t)seq * p.rows.n_slots + slot) * p.rows.page_table_stride;
@@ -170,7 +170,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
             const int tile = item_tile(it);
             const int row0 = p.tiles[tile], nq = p.tile_rows[tile];
-            const int seq = p.rows.seq_id[row0], slot = p.rows.slot_of(row0);
+            const int seq = p.rows.seq_of(row0), slot = p.rows.slot_of(row0);
             const int pos_last = p.rows.position[row0 + nq - 1];
             if (seq < 0 || seq >= p.max_seqs || slot < 0 || slot >= p.rows.n_slots || pos_last < 0 || pos_last / kPageSize >= p.rows.page_table_stride) continue;
             const int n_kt = pos_last / kKT + 1;
@@ -213,7 +213,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
             const int tile = item_tile(it), head = it % H;
             const int row0 = p.tiles[tile], nq = p.tile_rows[tile];
-            const int seq = p.rows.seq_id[row0], slot = p.rows.slot_of(row0);
+            const int seq = p.rows.seq_of(row0), slot = p.rows.slot_of(row0);
             const int pos_last = p.rows.position[row0 + nq - 1];
             if (seq < 0 || seq >= p.max_seqs || slot < 0 || slot >= p.rows.n_slots || pos_last < 0 || pos_last / kPageSize >= p.rows.page_table_stride) {
                 if (r == 0) atomicCAS(p.status, 0, kStatusSeq);

@@ -81,6 +81,7 @@ int make_rows(cdb_t* h, const cdb_rows_t* rows, RowsDev* out, bool need_depth) {
     out->page_table_stride = rows->page_table_stride;
     out->n_slots = h->cfg.n_slots;
     out->slot_override = -1;
+    out->n_live = rows->n_rows_dev;
     return CDB_OK;
 }
 
@@ -476,7 +477,7 @@ int cdb_loop_step(cdb_t* h, const cdb_rows_t* rows, float* h_inout, float* gate_
     if (c.gate_kind == CDB_GATE_L2_CONVERGENCE)
         cudaMemcpyAsync(h->h_prev, h_inout, (size_t)rd.n_rows * c.d * sizeof(float), cudaMemcpyDeviceToDevice, st);
     const int n0 = (rd.n_rows + 1) / 2;
-    const bool split = (c.flags & CDB_FLAG_TWO_STREAM) && h->side && rd.n_rows >= kMinSplitRows;
+    const bool split = (c.flags & CDB_FLAG_TWO_STREAM) && h->side && rd.n_rows >= kMinSplitRows && !rd.n_live;   // (a half-batch view cannot shift a device-side count)
     if (!split) {
         h->attn_ctas_per_sm_cap = 0;
         launch_attention_plan(h, 0, rd, st);
@@ -590,6 +591,7 @@ int cdb_prefill(cdb_t* h, const int32_t* token_ids, const cdb_rows_t* rows, cons
         RowsDev re = rd;
         re.n_rows = n_emit;
         re.seq_id = nullptr;
+        re.n_live = nullptr;
         lm_head(h, kPrefillLane, re, h->h_emit, token_out, logits_out, st);
     }
     return check_launch(h, "cdb_prefill");

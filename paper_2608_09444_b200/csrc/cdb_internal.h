@@ -41,7 +41,13 @@ struct RowsDev {
     int32_t page_table_stride;
     int32_t n_slots;
     int32_t slot_override;   // >= 0: use this KV slot for every row (prelude / coda layers, prefill)
+    const int32_t* n_live;   // device count of live rows or NULL: rows at an index >= *n_live are pads
     __device__ __forceinline__ int slot_of(int row) const { return slot_override >= 0 ? slot_override : kv_slot[row]; }
+    // sequence id of a row, -1 for pads (0 when the call carries no sequence ids: LM head of gathered rows)
+    __device__ __forceinline__ int seq_of(int row) const {
+        if (n_live != nullptr && row >= *n_live) return -1;
+        return seq_id != nullptr ? seq_id[row] : 0;
+    }
 };
 
 struct KvPool {

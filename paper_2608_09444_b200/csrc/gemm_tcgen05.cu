@@ -578,7 +578,7 @@ gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
                     const bool reporter = i4 == 0 && hd == 0;
                     const int row = r0 + 16 * i + j;
                     if (row >= p.n) continue;
-                    const int seq = p.rows.seq_id[row];
+                    const int seq = p.rows.seq_of(row);
                     if (seq < 0) continue;
                     const int pos = p.rows.position[row], slot = p.rows.slot_of(row);
                     if (seq >= p.max_seqs || slot < 0 || slot >= p.rows.n_slots) { if (reporter && which == 0) atomicCAS(p.status, 0, kStatusSeq); continue; }
@@ -650,6 +650,7 @@ struct TailParams {
     int n_phases;
     TailPhase ph[kTailMaxPhases];
     const int32_t* seq_id;             // pads (< 0) are skipped by the row-wise stage
+    const int32_t* n_live;             // device count of live rows or NULL
     int n_rows, d;
     float eps;
     unsigned int* sync;                // grid barrier word (top bit flips once per barrier)
@@ -739,7 +740,7 @@ layer_tail_tcgen05_kernel(const __grid_constant__ TailMaps maps, const __grid_co
             constexpr int MAXV = 12;                                      // float4 chunks per thread: d <= 12 * 4 * 128
             const int d4 = P.d / 4;
             for (int row = blockIdx.x; row < P.n_rows; row += gridDim.x) {
-                if (P.seq_id != nullptr && P.seq_id[row] < 0) {
+                if (P.seq_id != nullptr && (P.seq_id[row] < 0 || (P.n_live != nullptr && row >= *P.n_live))) {
                     if (ph.gain)
                         for (int i = et; i < d4; i += 128) *reinterpret_cast<uint2*>(ph.out + (size_t)row * P.d + 4 * i) = make_uint2(0u, 0u);
                     continue;
@@ -1097,7 +1098,7 @@ int launch_layer_tail_tc(const cdb* h, int ln, const RowsDev& rows, float* x, co
         if (!projection(L.xn, W_qkv_next, nullptr, L.ws, nullptr, 3 * d, d, kModeStore, s_q)) return -1;
     }
     P.n_phases = np;
-    P.seq_id = rows.seq_id; P.n_rows = n; P.d = d; P.eps = c.eps; P.sync = h->grid_sync + ln; P.status = h->status;
+    P.seq_id = rows.seq_id; P.n_live = rows.n_live; P.n_rows = n; P.d = d; P.eps = c.eps; P.sync = h->grid_sync + ln; P.status = h->status;
     for (int i = 3 * np; i < 3 * kTailMaxPhases; ++i) maps.m[i] = maps.m[0];
 
     cudaLaunchConfig_t cfg = {};

@@ -46,13 +46,12 @@ template <int NT> __device__ __forceinline__ float block_sum(float v, float* sme
 // out[row] = x[row] * rsqrt(mean(x^2) + eps) * gain, rounded to T.  Pad rows get zeros.
 template <typename T>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain,
-                                                      T* __restrict__ out, const int32_t* __restrict__ seq_id,
-                                                      int d, float eps) {
+                                                      T* __restrict__ out, RowsDev rows, int d, float eps) {
     pdl_trigger();
     pdl_wait();
     __shared__ float red[8];
     const int row = blockIdx.x;
-    const bool pad = seq_id != nullptr && seq_id[row] < 0;
+    const bool pad = rows.seq_of(row) < 0;
     const float* xr = x + (size_t)row * d;
     T* orow = out + (size_t)row * d;
     if (pad) {
@@ -70,9 +69,9 @@ void launch_rmsnorm(const cdb* h, const float* x, const float* gain, void* out, 
     CDB_LAUNCH(h);
     if (rows.n_rows <= 0) return;
     if (h->cfg.dtype == CDB_FP32)
-        launch_pdl(rmsnorm_kernel<float>, dim3(rows.n_rows), dim3(256), 0, st, x, gain, (float*)out, rows.seq_id, h->cfg.d, h->cfg.eps);
+        launch_pdl(rmsnorm_kernel<float>, dim3(rows.n_rows), dim3(256), 0, st, x, gain, (float*)out, rows, h->cfg.d, h->cfg.eps);
     else
-        launch_pdl(rmsnorm_kernel<__nv_bfloat16>, dim3(rows.n_rows), dim3(256), 0, st, x, gain, (__nv_bfloat16*)out, rows.seq_id, h->cfg.d, h->cfg.eps);
+        launch_pdl(rmsnorm_kernel<__nv_bfloat16>, dim3(rows.n_rows), dim3(256), 0, st, x, gain, (__nv_bfloat16*)out, rows, h->cfg.d, h->cfg.eps);
 }
 
 // ------------------------------------------------------------------------------- split-K reduce + residual + RMSNorm
@@ -81,15 +80,14 @@ void launch_rmsnorm(const cdb* h, const float* x, const float* gain, void* out, 
 template <typename T>
 __global__ void __launch_bounds__(256) reduce_residual_norm_kernel(const float* __restrict__ ws, int splits, size_t split_stride,
                                                                    float* __restrict__ x, const float* __restrict__ gain,
-                                                                   T* __restrict__ out, const int32_t* __restrict__ seq_id,
-                                                                   int d, float eps) {
+                                                                   T* __restrict__ out, RowsDev rows, int d, float eps) {
     pdl_trigger();
     pdl_wait();
     __shared__ float red[8];
     constexpr int MAXV = 6;                                    // float4 chunks per thread: d <= 6 * 4 * 256
     const int row = blockIdx.x;
     const int d4 = d / 4;
-    if (seq_id != nullptr && seq_id[row] < 0) {
+    if (rows.seq_of(row) < 0) {
         if (gain) for (int i = threadIdx.x; i < d4; i += 256) store4<T>(out + (size_t)row * d + 4 * i, 0.f, 0.f, 0.f, 0.f);
         return;
     }
@@ -128,9 +126,9 @@ void launch_reduce_residual_norm(const cdb* h, const float* ws, int splits, size
     if (rows.n_rows <= 0) return;
     CDB_LAUNCH(h);
     if (h->cfg.dtype == CDB_FP32)
-        launch_pdl(reduce_residual_norm_kernel<float>, dim3(rows.n_rows), dim3(256), 0, st, ws, splits, split_stride, x, gain, (float*)out, rows.seq_id, h->cfg.d, h->cfg.eps);
+        launch_pdl(reduce_residual_norm_kernel<float>, dim3(rows.n_rows), dim3(256), 0, st, ws, splits, split_stride, x, gain, (float*)out, rows, h->cfg.d, h->cfg.eps);
     else
-        launch_pdl(reduce_residual_norm_kernel<__nv_bfloat16>, dim3(rows.n_rows), dim3(256), 0, st, ws, splits, split_stride, x, gain, (__nv_bfloat16*)out, rows.seq_id, h->cfg.d, h->cfg.eps);
+        launch_pdl(reduce_residual_norm_kernel<__nv_bfloat16>, dim3(rows.n_rows), dim3(256), 0, st, ws, splits, split_stride, x, gain, (__nv_bfloat16*)out, rows, h->cfg.d, h->cfg.eps);
 }
 
 // ------------------------------------------------------------------------------- RoPE + KV write
@@ -147,7 +145,7 @@ __global__ void __launch_bounds__(256) rope_kv_write_kernel(const float* __restr
     pdl_wait();
     const int row = blockIdx.x;
     // the three descriptor loads go out together, then the page-table load: two memory latencies instead of four
-    const int seq = rows.seq_id[row];
+    const int seq = rows.seq_of(row);
     const int pos = rows.position[row];
     const int slot = rows.slot_of(row);
     if (seq < 0) return;
@@ -228,13 +226,13 @@ void launch_swiglu(const cdb* h, int ln, int n_rows, cudaStream_t st) {
 // ------------------------------------------------------------------------------- embedding
 template <typename T>
 __global__ void __launch_bounds__(256) embed_kernel(const T* __restrict__ table, const int32_t* __restrict__ tokens,
-                                                    const int32_t* __restrict__ seq_id, float* __restrict__ out, int d,
+                                                    RowsDev rows, float* __restrict__ out, int d,
                                                     int V, int max_seqs, float* gate_S, uint8_t* gate_fire, int reset,
                                                     int32_t* status) {
     pdl_trigger();
     pdl_wait();
     const int row = blockIdx.x;
-    const int seq = seq_id ? seq_id[row] : 0;
+    const int seq = rows.seq_of(row);
     float* o = out + (size_t)row * d;
     const int tok = tokens[row];
     if (seq < 0 || tok < 0 || tok >= V || seq >= max_seqs) {
@@ -251,10 +249,10 @@ void launch_embed(const cdb* h, const int32_t* tokens, const RowsDev& rows, floa
     CDB_LAUNCH(h);
     if (rows.n_rows <= 0) return;
     if (h->cfg.dtype == CDB_FP32)
-        launch_pdl(embed_kernel<float>, dim3(rows.n_rows), dim3(256), 0, st, (const float*)h->w.embed, tokens, rows.seq_id, out, h->cfg.d,
+        launch_pdl(embed_kernel<float>, dim3(rows.n_rows), dim3(256), 0, st, (const float*)h->w.embed, tokens, rows, out, h->cfg.d,
             h->cfg.V, h->cfg.max_seqs, h->gate_S, h->gate_fire, reset_gate ? 1 : 0, h->status);
     else
-        launch_pdl(embed_kernel<__nv_bfloat16>, dim3(rows.n_rows), dim3(256), 0, st, (const __nv_bfloat16*)h->w.embed, tokens, rows.seq_id, out,
+        launch_pdl(embed_kernel<__nv_bfloat16>, dim3(rows.n_rows), dim3(256), 0, st, (const __nv_bfloat16*)h->w.embed, tokens, rows, out,
             h->cfg.d, h->cfg.V, h->cfg.max_seqs, h->gate_S, h->gate_fire, reset_gate ? 1 : 0, h->status);
 }
 
@@ -269,7 +267,7 @@ __global__ void __launch_bounds__(256) gate_kernel(const float* __restrict__ x, 
     pdl_wait();
     __shared__ float red[8];
     const int row = blockIdx.x;
-    const int seq = rows.seq_id[row];
+    const int seq = rows.seq_of(row);
     if (seq < 0 || seq >= max_seqs) {
         if (threadIdx.x == 0) { if (gate_val_out) gate_val_out[row] = 0.f; if (fire_out) fire_out[row] = 0; }
         return;
@@ -332,7 +330,7 @@ __global__ void __launch_bounds__(1024) compact_kernel(RowsDev rows, const uint8
         const int row = start + threadIdx.x;
         int s = 0, e = 0;
         if (row < rows.n_rows) {
-            const int seq = rows.seq_id[row];
+            const int seq = rows.seq_of(row);
             if (seq >= 0 && seq < max_seqs) {
                 const int depth = rows.loop_depth[row];
                 const int forced = rows.forced_exit ? rows.forced_exit[row] : 0;
@@ -441,7 +439,7 @@ __global__ void __launch_bounds__(256) copy_on_exit_kernel(KvPool pool, RowsDev 
     pdl_trigger();
     pdl_wait();
     const int row = blockIdx.x, layer = layer0 + blockIdx.y;
-    const int seq = rows.seq_id[row];
+    const int seq = rows.seq_of(row);
     if (seq < 0 || seq >= max_seqs) return;
     const int pos = rows.position[row], rt = exit_depth[row];
     if (rt < 1 || rt >= R) return;

@@ -28,7 +28,7 @@ def test_struct_sizes_match_the_header():
     from paper_2608_09444_b200 import binding
     assert ctypes.sizeof(binding.Config) == 18 * 4 + 4 * 4 + 4
     assert ctypes.sizeof(binding.Weights) == 11 * 8
-    assert ctypes.sizeof(binding.RowsStruct) == 4 + 4 + 6 * 8 + 4 + 4     # int, pad, six pointers, int, pad
+    assert ctypes.sizeof(binding.RowsStruct) == 4 + 4 + 6 * 8 + 4 + 4 + 8 # int, pad, six pointers, int, pad, pointer
 
 
 def test_null_handle_is_an_error_not_a_crash():

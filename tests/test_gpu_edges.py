@@ -151,6 +151,70 @@ def test_a_rows_result_does_not_depend_on_its_batch(flags, extra):
             assert np.array_equal(kv, full[i][3]), (subset, i)
 
 
+def test_device_side_row_count_masks_the_tail_and_serves_one_graph_for_every_batch_size():
+    """Static shapes (section 4.3): the call's capacity is fixed on the host, the number of live rows is read from
+    device memory.  Rows beyond the count are pads although their descriptor looks like a real row: their state and
+    their KV pages stay untouched and they appear in neither compaction list; the live rows get, bit for bit, what a
+    call of exactly that many rows gives.  One captured CUDA graph is replayed with three different counts."""
+    ctxs = [1, 16, 17, 40, 255, 256, 257, 300, 33, 70, 12, 90]
+    cap = len(ctxs)
+    B, cdb, _, table_np, pool, pool_np = setup(ctxs, max_rows=cap)
+    table = dev(table_np)
+    rng = np.random.default_rng(4)
+    h_np = rng.standard_normal((cap, DIMS.d)).astype(np.float32)
+    depth = rng.integers(1, DIMS.R + 1, cap)
+    seq, pos, dep, slot = i32(np.arange(cap)), i32(np.asarray(ctxs) - 1), i32(depth), i32(np.zeros(cap))
+    fire_prev = dev((rng.random(cap) < 0.4).astype(np.uint8))
+
+    def fresh():
+        pool.copy_(dev(pool_np, torch.bfloat16))
+        cdb.boundary_embed(i32([0] * cap), B.Rows(seq, pos, table), torch.zeros((cap, DIMS.d), device="cuda"))   # gate state reset
+        return dev(h_np.copy())
+
+    def exact(k):                                            # a call of exactly k rows
+        h = fresh()
+        rows = B.Rows(seq[:k], pos[:k], table, loop_depth=dep[:k], kv_slot=slot[:k])
+        gate = torch.zeros(k, device="cuda")
+        surv, ex, cnt = i32(np.zeros(k)), i32(np.zeros(k)), i32(np.zeros(2))
+        cdb.compact(rows, surv, ex, cnt, fire_prev=fire_prev[:k])
+        cdb.loop_step(rows, h[:k], gate)
+        torch.cuda.synchronize()
+        c = cnt.cpu().numpy()
+        return h.cpu().numpy(), gate.cpu().numpy(), surv.cpu().numpy()[:c[0]], ex.cpu().numpy()[:c[1]], pool.view(torch.int16).cpu().numpy()
+
+    n_live = i32([0])
+    rows = B.Rows(seq, pos, table, loop_depth=dep, kv_slot=slot, n_rows_dev=n_live)
+    h_g = torch.zeros((cap, DIMS.d), device="cuda")
+    gate_g = torch.zeros(cap, device="cuda")
+    surv_g, ex_g, cnt_g = i32(np.zeros(cap)), i32(np.zeros(cap)), i32(np.zeros(2))
+
+    def body():
+        cdb.compact(rows, surv_g, ex_g, cnt_g, fire_prev=fire_prev)
+        cdb.loop_step(rows, h_g, gate_g)
+
+    h_g.copy_(fresh())
+    body()                                                   # warm-up with a count of 0: nothing may change
+    torch.cuda.synchronize()
+    assert np.array_equal(h_g.cpu().numpy(), h_np) and cnt_g.cpu().tolist() == [0, 0]
+    assert np.array_equal(pool.float().cpu().numpy(), pool_np)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        body()
+    for k in (5, 12, 1):
+        want_h, want_gate, want_s, want_e, want_pool = exact(k)
+        h_g.copy_(fresh())
+        n_live.fill_(k)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert cdb.poll_status() == 0
+        c = cnt_g.cpu().numpy()
+        assert np.array_equal(surv_g.cpu().numpy()[:c[0]], want_s) and np.array_equal(ex_g.cpu().numpy()[:c[1]], want_e)
+        assert np.array_equal(h_g.cpu().numpy().view(np.int32), want_h.view(np.int32))          # live rows equal, dead rows untouched
+        assert np.array_equal(gate_g.cpu().numpy()[:k].view(np.int32), want_gate.view(np.int32))
+        assert np.array_equal(pool.view(torch.int16).cpu().numpy(), want_pool)                  # dead rows wrote no K/V
+    assert cdb.check_guards() == 0
+
+
 WIDE = synth.Dims(V=64, d=1024, H=8, Dh=128, F=2816, L_pre=0, L_core=2, L_coda=0, R=4, dtype="bf16")
 
 
