@@ -136,6 +136,17 @@ const char* cdb_last_error(const cdb_t* h);      /* static / handle-owned string
  * expressed through cdb_rows_t.page_table.  CDB_ERR_ARG if `bytes` is too small. */
 int cdb_kv_bind(cdb_t* h, void* pool_device, size_t bytes, int32_t n_phys_pages);
 
+/* Optional, before cdb_kv_bind: a page space of their own for the prelude and coda layers.  Those layers cache one
+ * k, v per token whatever the depth layout (appendix C.1, Table 1 counts L_pre + L_coda + slots * L_core vectors), so
+ * with more than one depth slot they should not share page ids with the core layers, whose every slot owns pages.
+ *   pool_device[layer in [0, L_pre + L_coda)][physical page][K / V][head][token in page][Dh]   (prelude layers first)
+ *   page_table: device int32 [max_seqs][page_table_stride], row seq_id; caller-owned, must stay valid and may be
+ *   updated in place between calls (like cdb_rows_t.page_table).
+ * The pool given to cdb_kv_bind afterwards holds the L_core core layers alone, layer index 0 = first core layer.
+ * CDB_ERR_STATE for a model without boundary layers or when cdb_kv_bind was already called. */
+int cdb_kv_bind_boundary(cdb_t* h, void* pool_device, size_t bytes, int32_t n_phys_pages, const int32_t* page_table,
+                         int32_t page_table_stride);
+
 /* Changes the learned gate's bias and the exit threshold (host values). */
 int cdb_set_gate(cdb_t* h, float b_gate, float q_or_eps);
 

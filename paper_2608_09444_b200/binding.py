@@ -31,7 +31,8 @@ FLAG_WORKSPACE_PARTS = 32
 EXPORTS = ["cdb_create", "cdb_destroy", "cdb_last_error", "cdb_kv_bind", "cdb_set_gate", "cdb_boundary_embed",
            "cdb_boundary_prelude", "cdb_loop_step", "cdb_compact", "cdb_gather_rows", "cdb_boundary_coda_lmhead",
            "cdb_prefill", "cdb_kv_copy_on_exit", "cdb_paged_attention", "cdb_linear", "cdb_poll_status",
-           "cdb_profile_begin", "cdb_profile_read", "cdb_paged_attention_static", "cdb_debug_check_guards"]
+           "cdb_profile_begin", "cdb_profile_read", "cdb_paged_attention_static", "cdb_debug_check_guards",
+           "cdb_kv_bind_boundary"]
 
 
 class Config(C.Structure):
@@ -63,6 +64,7 @@ lib.cdb_destroy.argtypes = [_P]
 lib.cdb_last_error.argtypes = [_P]
 lib.cdb_last_error.restype = C.c_char_p
 lib.cdb_kv_bind.argtypes = [_P, _P, C.c_size_t, C.c_int32]
+lib.cdb_kv_bind_boundary.argtypes = [_P, _P, C.c_size_t, C.c_int32, _P, C.c_int32]
 lib.cdb_set_gate.argtypes = [_P, C.c_float, C.c_float]
 lib.cdb_boundary_embed.argtypes = [_P, _P, C.POINTER(RowsStruct), _P, _P]
 lib.cdb_boundary_prelude.argtypes = [_P, _P, C.POINTER(RowsStruct), _P, _P]
@@ -184,6 +186,12 @@ class Cdb:
     def kv_bind(self, pool: torch.Tensor):
         self._pool = pool
         self._check(lib.cdb_kv_bind(self.h, _ptr(pool), pool.numel() * pool.element_size(), int(pool.shape[1])))
+
+    def kv_bind_boundary(self, pool: torch.Tensor, page_table: torch.Tensor):
+        """Page space of the prelude and coda layers (call before kv_bind; the main pool then holds the core layers)."""
+        self._pool_b, self._table_b = pool, page_table
+        self._check(lib.cdb_kv_bind_boundary(self.h, _ptr(pool), pool.numel() * pool.element_size(), int(pool.shape[1]),
+                                             _ptr(page_table), int(page_table.shape[-1])))
 
     def set_gate(self, b_gate: float, q_or_eps: float):
         self._check(lib.cdb_set_gate(self.h, b_gate, q_or_eps))

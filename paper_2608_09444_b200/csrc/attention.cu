@@ -366,7 +366,8 @@ static void launch_attention_t(const cdb* h, const AttnParams& p, void* o, cudaS
 void launch_attention(const cdb* h, int ln, int layer, const RowsDev& rows, const void* q, void* o, cudaStream_t st) {
     if (rows.n_rows <= 0) return;
     AttnParams p;
-    p.q = q; p.pool = h->pool; p.rows = rows; p.layer = layer; p.max_splits = h->max_splits;
+    const LayerKv kv = layer_kv(h, layer, rows);
+    p.q = q; p.pool = kv.pool; p.rows = kv.rows; p.layer = kv.layer; p.max_splits = h->max_splits;
     p.max_seqs = h->cfg.max_seqs;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)h->cfg.Dh);
     p.part = h->lane[ln].attn_part; p.item_start = h->lane[ln].attn_item_start; p.counter = h->lane[ln].attn_counters + layer; p.status = h->status;
@@ -719,7 +720,8 @@ void launch_attention_prefill(const cdb* h, int ln, int layer, const RowsDev& ro
     if (rows.n_rows <= 0) return;
     if (!(h->cfg.flags & CDB_FLAG_SIMT_PREFILL) && launch_attention_prefill_tc(h, ln, layer, rows, q, o, st)) return;
     AttnParams p;
-    p.q = q; p.pool = h->pool; p.rows = rows; p.layer = layer; p.max_splits = h->max_splits;
+    const LayerKv kv = layer_kv(h, layer, rows);
+    p.q = q; p.pool = kv.pool; p.rows = kv.rows; p.layer = kv.layer; p.max_splits = h->max_splits;
     p.max_seqs = h->cfg.max_seqs;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)h->cfg.Dh);
     p.part = nullptr; p.item_start = nullptr; p.counter = nullptr; p.status = h->status;

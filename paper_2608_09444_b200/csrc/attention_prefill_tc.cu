@@ -345,16 +345,17 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
 bool launch_attention_prefill_tc(const cdb* h, int ln, int layer, const RowsDev& rows, const void* q, void* o, cudaStream_t st) {
     const int Dh = h->cfg.Dh, H = h->cfg.H;
     if (h->cfg.dtype != CDB_BF16 || (Dh != 64 && Dh != 96 && Dh != 128) || encode_fn() == nullptr) return false;
-    const long long kv_rows = (long long)(h->cfg.L_pre + h->cfg.L_core + h->cfg.L_coda) * h->pool.n_phys_pages * 2 * H * kPageSize;
+    const LayerKv kv = layer_kv(h, layer, rows);
+    const long long kv_rows = (long long)kv.n_layers * kv.pool.n_phys_pages * 2 * H * kPageSize;
     if (kv_rows >= (1LL << 31)) return false;
     CUtensorMap map_q, map_kv;
-    if (!make_map(&map_q, q, rows.n_rows, H * Dh, kQT) || !make_map(&map_kv, h->pool.base, (int)kv_rows, Dh, kPageSize)) return false;
+    if (!make_map(&map_q, q, rows.n_rows, H * Dh, kQT) || !make_map(&map_kv, kv.pool.base, (int)kv_rows, Dh, kPageSize)) return false;
     const Lane& L = h->lane[ln];
     // pads first: rows the tiles do not cover keep a zero output
     cudaMemsetAsync(o, 0, (size_t)rows.n_rows * H * Dh * sizeof(__nv_bfloat16), st);
     launch_prefill_plan(h, ln, rows, kQT, st);
     PfParams p;
-    p.rows = rows; p.pool = h->pool; p.layer = layer; p.max_seqs = h->cfg.max_seqs;
+    p.rows = kv.rows; p.pool = kv.pool; p.layer = kv.layer; p.max_seqs = h->cfg.max_seqs;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)Dh);
     p.tiles = L.attn_item_start; p.tile_rows = L.pf_tile_rows; p.n_tiles = L.pf_n_tiles;
     p.out = (__nv_bfloat16*)o; p.status = h->status;

@@ -422,12 +422,32 @@ const char* cdb_last_error(const cdb_t* h) { return h ? h->err : "invalid handle
 int cdb_kv_bind(cdb_t* h, void* pool_device, size_t bytes, int32_t n_phys_pages) {
     if (!h) return CDB_ERR_ARG;
     if (!pool_device || n_phys_pages < 1) return fail(h, CDB_ERR_ARG, "pool is NULL or has no pages");
-    const size_t L = h->cfg.L_pre + h->cfg.L_core + h->cfg.L_coda;
+    // with a boundary page space bound, this pool holds the core layers alone
+    const size_t L = h->pool_b.base ? h->cfg.L_core : h->cfg.L_pre + h->cfg.L_core + h->cfg.L_coda;
     const size_t need = L * n_phys_pages * 2 * h->cfg.H * kPageSize * h->cfg.Dh * h->elem_size;
-    if (bytes < need) return fail(h, CDB_ERR_ARG, "pool is smaller than [L][pages][2][H][16][Dh]");
+    if (bytes < need) return fail(h, CDB_ERR_ARG, "pool is smaller than [layers][pages][2][H][16][Dh]");
     if ((uintptr_t)pool_device % 16) return fail(h, CDB_ERR_ARG, "pool must be 16-byte aligned");
     h->pool.base = pool_device;
     h->pool.n_phys_pages = n_phys_pages;
+    return CDB_OK;
+}
+
+int cdb_kv_bind_boundary(cdb_t* h, void* pool_device, size_t bytes, int32_t n_phys_pages, const int32_t* page_table,
+                         int32_t page_table_stride) {
+    if (!h) return CDB_ERR_ARG;
+    const size_t Lb = h->cfg.L_pre + h->cfg.L_coda;
+    if (Lb == 0) return fail(h, CDB_ERR_STATE, "the model has no prelude or coda layers");
+    if (h->pool.base) return fail(h, CDB_ERR_STATE, "bind the boundary page space before cdb_kv_bind");
+    if (!pool_device || n_phys_pages < 1 || !page_table || page_table_stride < 1) return fail(h, CDB_ERR_ARG, "pool / page table is NULL or empty");
+    const size_t need = Lb * n_phys_pages * 2 * h->cfg.H * kPageSize * h->cfg.Dh * h->elem_size;
+    if (bytes < need) return fail(h, CDB_ERR_ARG, "boundary pool is smaller than [L_pre + L_coda][pages][2][H][16][Dh]");
+    if ((uintptr_t)pool_device % 16) return fail(h, CDB_ERR_ARG, "pool must be 16-byte aligned");
+    h->pool_b.base = pool_device;
+    h->pool_b.n_phys_pages = n_phys_pages;
+    h->pool_b.H = h->cfg.H;
+    h->pool_b.Dh = h->cfg.Dh;
+    h->table_b = page_table;
+    h->table_b_stride = page_table_stride;
     return CDB_OK;
 }
 

@@ -92,6 +92,9 @@ struct cdb {
     cdb_config_t cfg;
     cdb_weights_t w;
     cdbk::KvPool pool;
+    cdbk::KvPool pool_b;            // page space of the prelude and coda layers (base NULL: they share `pool`)
+    const int32_t* table_b;         // its page table [max_seqs][table_b_stride] (device, caller-owned)
+    int32_t table_b_stride;
     size_t elem_size;               // bytes of the configured dtype
     int device;                     // the device that was current in cdb_create: every call on the handle must run there
     int sms;                        // its multiprocessor count
@@ -175,6 +178,27 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 }  // namespace cdbk
 
 namespace cdbk {
+// What a layer's KV kernels see.  Without a boundary page space every layer lives in `pool` ([L] layers, page ids
+// shared by all layers).  With one, the prelude and coda layers live in pool_b ([L_pre + L_coda] layers, one slot per
+// sequence, their own page table) and `pool` holds the core layers alone ([L_core] layers): a depth slot then
+// reserves pages in the core layers only, which is what the paper's Table 1 counts.
+struct LayerKv { KvPool pool; int layer; int n_layers; RowsDev rows; };
+inline LayerKv layer_kv(const cdb* h, int layer, const RowsDev& rows) {
+    const int Lp = h->cfg.L_pre, Lc = h->cfg.L_core, Lo = h->cfg.L_coda;
+    LayerKv k;
+    k.pool = h->pool; k.layer = layer; k.n_layers = Lp + Lc + Lo; k.rows = rows;
+    if (h->pool_b.base) {
+        if (layer < Lp || layer >= Lp + Lc) {
+            k.pool = h->pool_b; k.layer = layer < Lp ? layer : layer - Lc; k.n_layers = Lp + Lo;
+            k.rows.page_table = h->table_b; k.rows.page_table_stride = h->table_b_stride;
+            k.rows.n_slots = 1; k.rows.slot_override = 0;
+        } else {
+            k.layer = layer - Lp; k.n_layers = Lc;
+        }
+    }
+    return k;
+}
+
 constexpr int kProfCap = 8192;
 enum { kProfAttention = 0, kProfLinear = 1, kProfClasses = 2 };
 // Brackets the kernels launched during its lifetime with an event pair when profiling is on.

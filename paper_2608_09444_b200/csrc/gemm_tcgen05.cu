@@ -1041,7 +1041,8 @@ bool launch_qkv_rope_cluster_tc(const cdb* h, int ln, int layer, const void* xin
     if (c.Dh != BM || c.d % BM != 0 || c.dtype != CDB_BF16) return false;
     ClusterParams p = {};
     p.mode = kClusterRope;
-    p.qrot = h->lane[ln].qrot; p.pool = h->pool; p.rows = rows; p.layer = layer; p.d = c.d;
+    const LayerKv kv = layer_kv(h, layer, rows);
+    p.qrot = h->lane[ln].qrot; p.pool = kv.pool; p.rows = kv.rows; p.layer = kv.layer; p.d = c.d;
     p.max_position = c.max_position; p.max_seqs = c.max_seqs; p.rope_cos = h->rope_cos; p.rope_sin = h->rope_sin;
     return launch_cluster_gemm(h, xin, W_qkv, rows.n_rows, 3 * c.d, c.d, max_splits, p, st);
 }

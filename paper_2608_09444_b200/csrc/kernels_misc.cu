@@ -190,13 +190,14 @@ void launch_rope_kv_write(const cdb* h, int ln, int layer, const float* qkv_part
                           const RowsDev& rows, cudaStream_t st) {
     CDB_LAUNCH(h);
     if (rows.n_rows <= 0) return;
+    const LayerKv kv = layer_kv(h, layer, rows);
     if (h->cfg.dtype == CDB_FP32)
         launch_pdl(rope_kv_write_kernel<float>, dim3(rows.n_rows), dim3(256), 0, st, qkv_parts, parts, part_stride,
-                   (float*)h->lane[ln].qrot, h->pool, rows, layer, h->rope_cos, h->rope_sin, h->cfg.d, h->cfg.max_position,
+                   (float*)h->lane[ln].qrot, kv.pool, kv.rows, kv.layer, h->rope_cos, h->rope_sin, h->cfg.d, h->cfg.max_position,
                    h->cfg.max_seqs, h->status);
     else
         launch_pdl(rope_kv_write_kernel<__nv_bfloat16>, dim3(rows.n_rows), dim3(256), 0, st, qkv_parts, parts, part_stride,
-                   (__nv_bfloat16*)h->lane[ln].qrot, h->pool, rows, layer, h->rope_cos, h->rope_sin, h->cfg.d,
+                   (__nv_bfloat16*)h->lane[ln].qrot, kv.pool, kv.rows, kv.layer, h->rope_cos, h->rope_sin, h->cfg.d,
                    h->cfg.max_position, h->cfg.max_seqs, h->status);
 }
 
@@ -469,10 +470,11 @@ void launch_copy_on_exit(const cdb* h, const RowsDev& rows, const int32_t* exit_
     CDB_LAUNCH(h);
     if (rows.n_rows <= 0 || h->cfg.L_core <= 0) return;
     dim3 grid(rows.n_rows, h->cfg.L_core);
+    const int layer0 = layer_kv(h, h->cfg.L_pre, rows).layer;          // first core layer's index inside the core layers' pool
     if (h->cfg.dtype == CDB_FP32)
-        launch_pdl(copy_on_exit_kernel<float>, dim3(grid), dim3(256), 0, st, h->pool, rows, exit_depth, h->cfg.L_pre, h->cfg.R, h->cfg.max_seqs, h->cfg.max_position, h->status);
+        launch_pdl(copy_on_exit_kernel<float>, dim3(grid), dim3(256), 0, st, h->pool, rows, exit_depth, layer0, h->cfg.R, h->cfg.max_seqs, h->cfg.max_position, h->status);
     else
-        launch_pdl(copy_on_exit_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, st, h->pool, rows, exit_depth, h->cfg.L_pre, h->cfg.R, h->cfg.max_seqs, h->cfg.max_position, h->status);
+        launch_pdl(copy_on_exit_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, st, h->pool, rows, exit_depth, layer0, h->cfg.R, h->cfg.max_seqs, h->cfg.max_position, h->status);
 }
 
 }  // namespace cdbk

@@ -36,7 +36,8 @@ class Engine:
                  r_min: int = 1, lookahead: bool = True, mode: str = "refill", min_coda_batch: int = 1,
                  max_prefill_rows: int | None = None, flags: int = 0, record_states: bool = False,
                  record_logits: bool = False, record_ticks: bool = True, use_graphs: bool = True,
-                 time_device: bool = False, admit_min: int = 1, admit_wait_s: float = 0.0, device: str = "cuda:0"):
+                 time_device: bool = False, admit_min: int = 1, admit_wait_s: float = 0.0, device: str = "cuda:0",
+                 boundary_pages: int | None = None):
         if mode not in ("refill", "no_refill", "cb"):
             raise ValueError(f"unknown scheduling mode {mode!r}: expected 'refill', 'no_refill' or 'cb'")
         self.dims, self.mode, self.lookahead = dims, mode, lookahead
@@ -50,7 +51,18 @@ class Engine:
         self.n_slots = self.cdb.n_slots
         self.kv_layout = kv_layout
         dt = torch.float32 if dims.dtype == "fp32" else torch.bfloat16
-        self.pool = torch.zeros((dims.L, n_pages, 2, dims.H, dims.page_size, dims.Dh), dtype=dt, device=self.dev)
+        # A model with prelude / coda layers and more than one depth slot gets a page space of its own for those layers:
+        # they cache one k, v per token whatever the layout, so only the core layers' pool pays for the slots (Table 1).
+        # boundary_pages: pages of that space (default: the main pool's share of one slot); 0 = one shared page space.
+        self.split_kv = self.n_slots > 1 and dims.L_pre + dims.L_coda > 0 and boundary_pages != 0
+        if self.split_kv:
+            self.n_pages_b = boundary_pages or max(1, n_pages // self.n_slots)
+            self.pool_b = torch.zeros((dims.L_pre + dims.L_coda, self.n_pages_b, 2, dims.H, dims.page_size, dims.Dh), dtype=dt, device=self.dev)
+            self.free_pages_b = list(range(self.n_pages_b - 1, -1, -1))
+            self.page_table_b_host = np.full((max_live, self.max_pages), -1, dtype=np.int32)
+            self.page_table_b = torch.from_numpy(self.page_table_b_host.copy()).to(self.dev)
+            self.cdb.kv_bind_boundary(self.pool_b, self.page_table_b)
+        self.pool = torch.zeros((dims.L_core if self.split_kv else dims.L, n_pages, 2, dims.H, dims.page_size, dims.Dh), dtype=dt, device=self.dev)
         self.cdb.kv_bind(self.pool)
         self.n_pages = n_pages
         self.free_pages = list(range(n_pages - 1, -1, -1))            # pop() hands out the lowest id first
@@ -81,8 +93,8 @@ class Engine:
         # Recurrent step as a CUDA graph per row-count bucket (rows padded with seq_id = -1 to a multiple of 32):
         # the descriptor lives in fixed device arrays refreshed by one host-to-device copy per step.
         self.use_graphs = use_graphs
-        self.desc_host = torch.zeros((5, max_rows), dtype=torch.int32).pin_memory()
-        self.desc_dev = torch.zeros((5, max_rows), **i32)
+        self.desc_host = torch.zeros((6, max_rows), dtype=torch.int32).pin_memory()    # five descriptor rows; [5, 0] = live rows
+        self.desc_dev = torch.zeros((6, max_rows), **i32)
         self.graphs = {}
         # optional accounting of device time: CUDA-event pairs around every GPU phase the engine enqueues
         self.time_device = time_device
@@ -138,6 +150,12 @@ class Engine:
         need = (n_tokens + self.dims.page_size - 1) // self.dims.page_size
         if need * self.n_slots > len(self.free_pages) or need > self.max_pages:
             return False
+        if self.split_kv:
+            if need > len(self.free_pages_b):
+                return False
+            for j in range(need):
+                self.page_table_b_host[slot_id, j] = self.free_pages_b.pop()
+            self.page_table_b[slot_id].copy_(torch.from_numpy(self.page_table_b_host[slot_id]))
         for s in range(self.n_slots):
             row = slot_id * self.n_slots + s
             for j in range(need):
@@ -147,6 +165,11 @@ class Engine:
         return True
 
     def _release_pages(self, slot_id: int):
+        if self.split_kv:
+            used = self.page_table_b_host[slot_id][self.page_table_b_host[slot_id] >= 0]
+            for p in reversed(used):
+                self.free_pages_b.append(int(p))
+            self.page_table_b_host[slot_id] = -1
         for s in reversed(range(self.n_slots)):
             row = slot_id * self.n_slots + s
             used = self.page_table_host[row][self.page_table_host[row] >= 0]
@@ -411,16 +434,16 @@ class Engine:
                 "gates": [s.gates for s in seqs]}
 
 
-def kv_footprint(dims, n_slots: int) -> tuple[int, int]:
-    """KV bytes per cached token: (in use, reserved by this library's pool).  In use is what the paper's
-    Table 1 counts: one K and one V vector per layer, the core layers once per depth slot.  The pool gives
-    every (sequence, slot) pair its own pages in ALL layers (page ids are shared by the layers), so the
-    prelude and coda layers' share of the pages of slots > 0 stays empty: reserved >= in use, equal for
-    fully looped models and for the shared layout."""
+def kv_footprint(dims, n_slots: int, split_kv: bool = True) -> tuple[int, int]:
+    """KV bytes per cached token: (in use, reserved by the engine's page pools).  In use is what the paper's
+    Table 1 counts: one K and one V vector per layer, the core layers once per depth slot.  With a page space of
+    their own for the prelude and coda layers (the engines' default for more than one slot) exactly that is
+    reserved.  With ONE page space shared by all layers every (sequence, slot) pair owns pages in ALL layers, so the
+    boundary layers' share of the pages of slots > 0 stays empty: reserved >= in use."""
     eb = 4 if dims.dtype == "fp32" else 2
     per_layer = 2 * dims.H * dims.Dh * eb
     used = (dims.L_pre + dims.L_coda + dims.L_core * n_slots) * per_layer
-    reserved = (dims.L_pre + dims.L_coda + dims.L_core) * n_slots * per_layer
+    reserved = used if split_kv else (dims.L_pre + dims.L_coda + dims.L_core) * n_slots * per_layer
     return used, reserved
 
 
@@ -430,7 +453,9 @@ def _bucket(k: int, cap: int) -> int:
 
 def _static_rows(eng: "Engine", nb: int) -> B.Rows:
     d = eng.desc_dev
-    return B.Rows(d[0, :nb], d[2, :nb], eng.page_table, loop_depth=d[1, :nb], kv_slot=d[3, :nb], forced_exit=d[4, :nb])
+    # rows beyond the device-side count d[5, 0] are pads: a bucket's graph serves every batch size up to nb
+    return B.Rows(d[0, :nb], d[2, :nb], eng.page_table, loop_depth=d[1, :nb], kv_slot=d[3, :nb], forced_exit=d[4, :nb],
+                  n_rows_dev=d[5, :1])
 
 
 def _step_body(eng: "Engine", rows: B.Rows, nb: int):
@@ -456,18 +481,17 @@ def _run_step(eng: "Engine", k: int, seq, depth, pos, slot, forced):
     dh[2, :k] = torch.as_tensor(np.asarray(pos, dtype=np.int32))
     dh[3, :k] = torch.as_tensor(np.asarray(slot, dtype=np.int32))
     dh[4, :k] = torch.as_tensor(np.asarray(forced, dtype=np.int32))
-    dh[0, k:nb] = -1
-    dh[1:, k:nb] = 0
+    dh[5, 0] = k
     if not eng.use_graphs:
         eng.desc_dev.copy_(dh, non_blocking=True)
         _step_body(eng, _static_rows(eng, nb), nb)
         return
     if nb not in eng.graphs:
-        # Warm-up on an all-pad descriptor, then capture.  Pads touch neither the KV pool nor the gate state, but
-        # the body ends by moving the (empty) survivor list to the front of h_rec, which would overwrite the
-        # rows waiting there for this very step: keep them aside.
+        # Warm-up with a live count of zero (every row a pad), then capture.  Pads touch neither the KV pool nor the
+        # gate state, but the body ends by moving the (empty) survivor list to the front of h_rec, which would
+        # overwrite the rows waiting there for this very step: keep them aside.
         saved = eng.h_rec[:nb].clone()
-        eng.desc_dev[0, :nb].fill_(-1)
+        eng.desc_dev[5, 0].fill_(0)
         rows = _static_rows(eng, nb)
         _step_body(eng, rows, nb)
         torch.cuda.synchronize(eng.dev)

@@ -66,7 +66,7 @@ class PipelinedEngine(Engine):
             for parity in (0, 1):
                 if (nb, parity) in self.pgraphs:
                     continue
-                self.desc_dev[0, :nb].fill_(-1)                   # all pads: the warm-up touches no model state
+                self.desc_dev[5, 0].fill_(0)                      # live count 0, all pads: the warm-up touches no model state
                 rows = _static_rows(self, nb)
                 self.cdb.compact(rows, self.surv_idx, self.exit_idx, self.counts)
                 self._body(rows, nb, parity)
@@ -107,7 +107,7 @@ class PipelinedEngine(Engine):
         ready, ready_free = [], list(range(self.cap - 1, -1, -1))     # (sid, slot in h_ready, event, iteration)
         coda_q, coda_free = [], list(range(self.cap - 1, -1, -1))     # (sid, depth, slot in h_coda)
         pending_tokens, pending_release = [], []
-        ring = [torch.zeros((5, self.max_rows), dtype=torch.int32).pin_memory() for _ in range(4)]
+        ring = [torch.zeros((6, self.max_rows), dtype=torch.int32).pin_memory() for _ in range(4)]
         tok_ring = [torch.zeros(self.cap, dtype=torch.int32).pin_memory() for _ in range(16)]
         tok_dev = torch.zeros(self.cap, dtype=torch.int32, device=dev)
         tokp_dev = torch.zeros(self.cap, dtype=torch.int32, device=dev)      # first tokens of a prompt call
@@ -347,8 +347,7 @@ class PipelinedEngine(Engine):
                 dh[2, :k] = torch.as_tensor(np.asarray([P[s] + gen[s] - 1 for s, _ in rec], dtype=np.int32))
                 dh[3, :k] = torch.as_tensor(np.asarray([self._slot(r) for _, r in rec], dtype=np.int32))
                 dh[4, :k] = torch.as_tensor(np.asarray([forced_for(s) for s, _ in rec], dtype=np.int32))
-                dh[0, k:nb] = -1
-                dh[1:, k:nb] = 0
+                dh[5, 0] = k                                # device-side live count: the rows behind it are pads
                 with self._phase("recurrent"):
                     self.desc_dev.copy_(dh, non_blocking=True)
                     g, rows = self.pgraphs[(nb, parity)]

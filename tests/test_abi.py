@@ -40,8 +40,9 @@ def test_null_handle_is_an_error_not_a_crash():
 
 
 def test_kv_footprint_accounting_matches_table1():
-    """The driver's KV accounting against the sizes printed in the paper's Table 1 (appendix C.1), and the
-    pool's own reservation, which exceeds them only for models with boundary layers and more than one slot."""
+    """The driver's KV accounting against the sizes printed in the paper's Table 1 (appendix C.1): what the page
+    pools reserve per cached token equals the table in every row once the prelude and coda layers have a page space
+    of their own; with one page space for all layers it exceeds the table for boundary layers with several slots."""
     import os
     from paper_2608_09444_b200 import synth
     from paper_2608_09444_b200.engine import kv_footprint
@@ -53,7 +54,9 @@ def test_kv_footprint_accounting_matches_table1():
         model, slots, kib, gib = line.split()
         used, reserved = kv_footprint(dims[model], int(slots))
         assert abs(used / 1024 - float(kib)) <= 0.5 and abs(used * 4096 / 2**30 - float(gib)) <= 0.006
-        assert reserved >= used and (reserved == used) == (model == "ouro" or int(slots) == 1)
+        assert reserved == used
+        used1, reserved1 = kv_footprint(dims[model], int(slots), split_kv=False)
+        assert used1 == used and reserved1 >= used and (reserved1 == used) == (model == "ouro" or int(slots) == 1)
 
 
 def test_engines_reject_unknown_scheduling_modes_before_touching_the_gpu():

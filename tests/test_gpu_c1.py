@@ -143,6 +143,16 @@ def test_c1_depth_aware_kv_layouts(layout):
     for s in range(8):
         assert np.array_equal(pres["tokens"][s], ref[s]["tokens"]), s
         assert np.array_equal(pres["depths"][s], ref[s]["depths"]), s
+    # Both engines gave the prelude and coda layers a page space of their own (several slots, boundary layers present):
+    # per cached token the pools hold what Table 1 counts, and every page of both spaces came back.
+    for e in (eng, peng):
+        assert e.split_kv and e.pool.shape[0] == dims.L_core and e.pool_b.shape[0] == dims.L_pre + dims.L_coda
+        assert sorted(e.free_pages) == list(range(e.n_pages)) and sorted(e.free_pages_b) == list(range(e.n_pages_b))
+        assert np.all(e.page_table_host == -1) and np.all(e.page_table_b_host == -1)
+    # ... and one page space shared by all layers (the other way to bind the pool) gives the same tokens
+    eng1, res1 = run_engine("refill", n_slots=n_slots, kv_layout=b_layout, boundary_pages=0)
+    assert not eng1.split_kv and eng1.pool.shape[0] == dims.L
+    compare(eng1, res1, ref)
 
 
 def test_c1_graph_replay_equals_direct_launches(oracle_runs):
