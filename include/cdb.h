@@ -82,8 +82,10 @@ enum { CDB_FLAG_SIMT_GEMM = 1,         /* run bf16 projections on the plain-FMA 
        CDB_FLAG_SIMT_PREFILL = 8,      /* prompt attention of bf16 pools on the plain-FMA kernel instead of the tensor cores (cross-check) */
        CDB_FLAG_FUSED_STAGES = 16,     /* everything of a layer after its attention as ONE cooperative launch with grid barriers between
                                          * the stages (experimental: measured slower than the separate, programmatically chained launches) */
-       CDB_FLAG_WORKSPACE_PARTS = 32 };/* split-K parts of the decode projections through a workspace and a row-wise kernel instead of being
+       CDB_FLAG_WORKSPACE_PARTS = 32,  /* split-K parts of the decode projections through a workspace and a row-wise kernel instead of being
                                          * summed inside thread-block clusters (cross-check: the sums and their order are the same) */
+       CDB_FLAG_CTA_PAIRS = 64 };      /* projections on 128 rows and more run as CTA pairs (one 256-feature MMA over two SMs, each CTA loading
+                                         * its own weights and half of the activation tile); same results bit for bit, measured no faster */
 
 /* Row-major [out_features, in_features] ("K-major") weights of the configured dtype, layers
  * stacked in the order prelude, core, coda (L = L_pre + L_core + L_coda).  All device pointers. */

@@ -67,13 +67,20 @@ struct CtaCtx {
 // is called by the producer warp after it has started the weight copies of its first ring fill and before
 // its first copy of an activation tile: it must return once the activations (and the output buffers) may
 // be touched.
-template <typename WaitInputs>
+// PAIR: the CTA is one of a pair (cluster of two) that shares every activation tile: tile = 2 x 128 features x BN rows,
+// this CTA loads its own 128 features' weights and its own half of the BN activation rows; the even CTA's MMA warp
+// issues for both (see tc_common.cuh).  map_x then has a box of BN / 2 rows.  The pair walks the same tile sequence.
+template <bool PAIR, typename WaitInputs>
 __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUtensorMap* map_w2, const CUtensorMap* map_x,
                                            const GemmParams& p, const CtaCtx& cx, WaitInputs wait_inputs) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int S = p.stages, BN = p.BN;
     const bool dual = p.mode == kModeSwiGLU;                                 // two weight tiles, two accumulators
-    const uint32_t w_bytes = BM * BK * 2, x_bytes = (uint32_t)BN * BK * 2;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+    const int cta = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x, n_cta = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    constexpr int FT = PAIR ? 2 * BM : BM;                                   // features per tile
+    const int XR = PAIR ? BN / 2 : BN;                                       // activation rows this CTA loads per tile
+    const uint32_t w_bytes = BM * BK * 2, x_bytes = (uint32_t)XR * BK * 2;
     const uint32_t x_off = dual ? 2 * w_bytes : w_bytes, stage_bytes = x_off + x_bytes;
     const uint32_t acc_cols = dual ? 2u * BN : (uint32_t)BN;                 // TMEM columns of one accumulator set
     const uint32_t ring = cx.ring, bar0 = cx.bar0;
@@ -81,8 +88,14 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
     auto empty_bar = [&](int s) { return bar0 + 8u * (8 + s); };
     auto acc_full_bar = [&](int a) { return bar0 + 8u * (16 + a); };
     auto acc_empty_bar = [&](int a) { return bar0 + 8u * (18 + a); };
-    const int n_ftiles = (p.N + BM - 1) / BM, n_rtiles = (p.n + BN - 1) / BN;
+    const int n_ftiles = (p.N + FT - 1) / FT, n_rtiles = (p.n + BN - 1) / BN;
     const int n_tiles = n_ftiles * n_rtiles * p.k_splits;                   // tile t = (split, row tile, feature tile)
+    // the barrier the loads of a stage report to (a shared::cluster address: in a pair, the even CTA's)
+    auto load_bar = [&](int s) { return PAIR ? map_to_cta(full_bar(s), 0u) : full_bar(s); };
+    auto load = [&](uint32_t dst, const CUtensorMap* m, int s, int c0, int c1) {
+        if (PAIR) tma_load_2d_pair(dst, m, load_bar(s), c0, c1); else tma_load_2d(dst, m, full_bar(s), c0, c1);
+    };
+    const uint32_t tx_bytes = PAIR ? 2u * stage_bytes : stage_bytes;         // both CTAs' shares arrive on one barrier
     const int n_kb = (p.K + BK - 1) / BK;
     auto kb_begin = [&](int t) { return (int)((long long)(t / (n_ftiles * n_rtiles)) * n_kb / p.k_splits); };
     auto kb_end = [&](int t) { return (int)((long long)(t / (n_ftiles * n_rtiles) + 1) * n_kb / p.k_splits); };
@@ -100,11 +113,13 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
             for (int pass = 0; pass < 2; ++pass) {
                 if (pass == 1) wait_inputs();
                 int g = 0;                                   // position in this CTA's (tile, k-block) sequence
-                for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-                    const int f0 = (t % n_ftiles) * BM, r0 = (t / n_ftiles % n_rtiles) * BN;
-                    // Every CTA walks its k-blocks from a different starting point (a function of its feature
-                    // tile only), so that the CTAs do not all pull the same activation lines from L2 at once.
-                    const int kb0 = kb_begin(t), nk = kb_end(t) - kb0, rot = ((t % n_ftiles) * 7) % nk;
+                for (int t = cta; t < n_tiles && ok; t += n_cta) {
+                    const int f0 = (t % n_ftiles) * FT + (int)rank * BM, r0 = (t / n_ftiles % n_rtiles) * BN + (int)rank * XR;
+                    // Every CTA walks its k-blocks from a different starting point, so that the CTAs do not all pull
+                    // the same activation lines from L2 at once.  The starting point is a function of the 256-feature
+                    // group alone: the same in every form of the kernel (alone, in a pair, in a split-K cluster), so
+                    // that a part is accumulated in the same order whichever form computes it.
+                    const int kb0 = kb_begin(t), nk = kb_end(t) - kb0, rot = (((t % n_ftiles) * FT / (2 * BM)) * 7) % nk;
                     if (pass == 0 && g >= S) break;
                     for (int j = 0; j < nk; ++j, ++g) {
                         if (pass == 0 && g >= S) break;
@@ -113,16 +128,16 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
                         if (pass == 0) {                     // ring is empty: stage g is free
                             const uint32_t dst = ring + (uint32_t)g * stage_bytes;
                             if (leader) {
-                                mbar_expect_tx(full_bar(g), stage_bytes);
-                                tma_load_2d(dst, map_w, full_bar(g), wc, wr);
-                                if (dual) tma_load_2d(dst + w_bytes, map_w2, full_bar(g), wc, wr);
+                                if (rank == 0) mbar_expect_tx(full_bar(g), tx_bytes);
+                                load(dst, map_w, g, wc, wr);
+                                if (dual) load(dst + w_bytes, map_w2, g, wc, wr);
                             }
                             __syncwarp();
                             n_pre = g + 1;
                             continue;
                         }
                         if (g < n_pre) {
-                            if (leader) tma_load_2d(ring + (uint32_t)g * stage_bytes + x_off, map_x, full_bar(g), kb * BK, r0);
+                            if (leader) load(ring + (uint32_t)g * stage_bytes + x_off, map_x, g, kb * BK, r0);
                             __syncwarp();
                             if (++s == S) { s = 0; ph ^= 1u; }
                             continue;
@@ -130,10 +145,10 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
                         if (!mbar_wait(empty_bar(s), ph ^ 1u, cx.abortp)) { ok = false; break; }
                         const uint32_t dst = ring + (uint32_t)s * stage_bytes;
                         if (leader) {
-                            mbar_expect_tx(full_bar(s), stage_bytes);
-                            tma_load_2d(dst, map_w, full_bar(s), wc, wr);
-                            if (dual) tma_load_2d(dst + w_bytes, map_w2, full_bar(s), wc, wr);
-                            tma_load_2d(dst + x_off, map_x, full_bar(s), kb * BK, r0);
+                            if (rank == 0) mbar_expect_tx(full_bar(s), tx_bytes);
+                            load(dst, map_w, s, wc, wr);
+                            if (dual) load(dst + w_bytes, map_w2, s, wc, wr);
+                            load(dst + x_off, map_x, s, kb * BK, r0);
                         }
                         __syncwarp();
                         if (++s == S) { s = 0; ph ^= 1u; }
@@ -155,15 +170,15 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
         }
         __syncwarp();
     } else if (warp == 1) {
-        {
+        if (!PAIR || rank == 0) {
             const bool leader = elect_one();
-            // instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, N = BN, M = 128
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            // instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, N = BN, M = 128 (256 over a pair)
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(FT >> 4) << 24);
             int s = 0; uint32_t ph = 0;
             int it = 0;
             bool ok = true;
             const long long mma_t0 = clock64();
-            for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
+            for (int t = cta; t < n_tiles && ok; t += n_cta, ++it) {
                 const int acc = it & 1;
                 const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
                 if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, cx.abortp)) { ok = false; break; }
@@ -180,14 +195,19 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
                     for (int k = 0; k < BK / UMMA_K; ++k) { // advance 32 bytes inside the swizzle span per UMMA_K
                         const uint64_t adv = (uint64_t)(k * UMMA_K * 2 >> 4);
                         const uint32_t accum = (kb > kb0 || k > 0) ? 1u : 0u;
-                        if (leader) umma_bf16(d_tmem, a_desc + adv, b_desc + adv, idesc, accum);
-                        if (leader && dual) umma_bf16(d_tmem + (uint32_t)BN, a2_desc + adv, b_desc + adv, idesc, accum);
+                        if (PAIR) {
+                            if (leader) umma_bf16_pair(d_tmem, a_desc + adv, b_desc + adv, idesc, accum);
+                            if (leader && dual) umma_bf16_pair(d_tmem + (uint32_t)BN, a2_desc + adv, b_desc + adv, idesc, accum);
+                        } else {
+                            if (leader) umma_bf16(d_tmem, a_desc + adv, b_desc + adv, idesc, accum);
+                            if (leader && dual) umma_bf16(d_tmem + (uint32_t)BN, a2_desc + adv, b_desc + adv, idesc, accum);
+                        }
                     }
                     __syncwarp();
-                    if (leader) umma_commit(empty_bar(s));  // stage is free once these MMAs have read it
+                    if (leader) { if (PAIR) umma_commit_pair(empty_bar(s)); else umma_commit(empty_bar(s)); }   // stage is free once these MMAs have read it
                     if (++s == S) { s = 0; ph ^= 1u; }
                 }
-                if (ok && leader) umma_commit(acc_full_bar(acc));     // accumulator complete
+                if (ok && leader) { if (PAIR) umma_commit_pair(acc_full_bar(acc)); else umma_commit(acc_full_bar(acc)); }   // accumulator complete
             }
             if (kTuningBuild && p.dbg && leader) p.dbg[blockIdx.x * 8 + 2] = clock64() - mma_t0;
         }
@@ -196,10 +216,10 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
         const int q = warp & 3;                             // TMEM lane quarter this warp may read
         int it = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
+        for (int t = cta; t < n_tiles && ok; t += n_cta, ++it) {
             const int acc = it & 1;
             const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
-            const int f = (t % n_ftiles) * BM + q * 32 + lane, r0 = (t / n_ftiles % n_rtiles) * BN;
+            const int f = (t % n_ftiles) * FT + (int)rank * BM + q * 32 + lane, r0 = (t / n_ftiles % n_rtiles) * BN;
             const int split = t / (n_ftiles * n_rtiles);
             if (!mbar_wait(acc_full_bar(acc), acc_ph, cx.abortp)) { ok = false; break; }
             if (kTuningBuild && p.dbg && it == 0 && warp == 2 && lane == 0) p.dbg[blockIdx.x * 8 + 4] = gtime();
@@ -247,7 +267,7 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
                 asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // the epilogue warps: tile staged
                 {
                     const int et = threadIdx.x - 64;                         // index among the epilogue threads
-                    const int f0t = (t % n_ftiles) * BM;
+                    const int f0t = (t % n_ftiles) * FT + (int)rank * BM;
                     for (int idx = et; idx < n_real * 16; idx += kEpiThreads) {   // 16 chunks of 8 features per row
                         const int row = idx >> 4, ch = idx & 15;
                         const int fc = f0t + ch * 8;
@@ -298,12 +318,14 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (kTuningBuild && p.dbg && warp == 2 && lane == 0) p.dbg[blockIdx.x * 8 + 6] = gtime();
-            if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+            // the accumulator may be overwritten once BOTH CTAs of a pair have drained their halves: all arrive at the issuing CTA
+            if (lane == 0) { if (PAIR && rank != 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(acc), 0u)); else mbar_arrive(acc_empty_bar(acc)); }
         }
     }
 
 }
 
+template <bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w2,
                          const __grid_constant__ CUtensorMap map_x, GemmParams p) {
@@ -328,15 +350,21 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), kEpiThreads / 32); }
+        for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), (PAIR ? 2 : 1) * (kEpiThreads / 32)); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if (PAIR) cluster_sync_all();                 // the peer's barriers exist before anything arrives on them
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_slot;
     volatile int* abortp = &abort_flag;
@@ -347,14 +375,16 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
 
     CtaCtx cx;
     cx.ring = ring; cx.bar0 = bar0; cx.tmem_base = tmem_base; cx.abortp = abortp;
-    gemm_roles(&map_w, &map_w2, &map_x, p, cx, [] { pdl_wait(); });
+    gemm_roles<PAIR>(&map_w, &map_w2, &map_x, p, cx, [] { pdl_wait(); });
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if (PAIR) cluster_sync_all();                 // nothing of the peer reads or signals this CTA's shared memory any more
     if (threadIdx.x == 0 && abort_flag) atomicCAS(p.status, 0, kStatusTimeout);
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+        if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
     }
 }
 
@@ -387,15 +417,6 @@ struct ClusterParams {
     unsigned long long* dbg;    // tuning builds: per-CTA phase time stamps (NULL = off)
 };
 
-__device__ __forceinline__ uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
-    return r;
-}
 __device__ __forceinline__ void st_cluster_f32(uint32_t addr, uint32_t v) {
     asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
@@ -464,7 +485,7 @@ gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
         auto w_coord = [&](int kb, int& wc, int& wr) { wc = p.w_tiled ? 0 : kb * BK; wr = p.w_tiled ? ((f0 / BM) * n_kb + kb) * BM : f0; };
         // the k-blocks of a part are taken in the same rotated order as by the workspace form of this projection
         // (a function of the feature tile only), so that both forms accumulate every part in the same order
-        const int rot = ((tile % n_ftiles) * 7) % nk;
+        const int rot = (((tile % n_ftiles) / 2) * 7) % nk;
         auto kb_of = [&](int g) { return kb0 + (g + rot) % nk; };
         for (int g = 0; g < n_pre; ++g) {
             int wc, wr; w_coord(kb_of(g), wc, wr);
@@ -720,7 +741,7 @@ layer_tail_tcgen05_kernel(const __grid_constant__ TailMaps maps, const __grid_co
         const TailPhase& ph = P.ph[pi];
         const bool last_wait = pi + 1 == P.n_phases;        // whoever passes the last barrier lets the next kernel launch
         if (ph.kind == kPhaseProjection) {
-            gemm_roles(&maps.m[ph.map_w], &maps.m[ph.map_w2], &maps.m[ph.map_x], ph.g, cx, [&] {
+            gemm_roles<false>(&maps.m[ph.map_w], &maps.m[ph.map_w2], &maps.m[ph.map_x], ph.g, cx, [&] {
                 if (pi == 0) {
                     pdl_wait();
                 } else {
@@ -858,7 +879,7 @@ void launch_repack_tiled(const void* W, void* Wt, int layers, int N, int K, cuda
 // kModeStore (y = workspace).  Returns the number of tiles, 0 on failure.
 static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2, float* y, __nv_bfloat16* act, int n,
                       int N, int K, int mode, int k_splits, size_t split_stride, GemmParams& p, CUtensorMap* map_w,
-                      CUtensorMap* map_w2, CUtensorMap* map_x, size_t* smem) {
+                      CUtensorMap* map_w2, CUtensorMap* map_x, size_t* smem, bool* pair = nullptr) {
     p.y = y; p.act = act; p.n = n; p.N = N; p.K = K; p.mode = mode; p.k_splits = k_splits; p.split_stride = split_stride;
     const int n_ft = (N + BM - 1) / BM;
     static const int forced_bn = tuning_int("CDB_GEMM_BN", 0);       // tuning hook
@@ -873,9 +894,29 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
         const int sms = h->sms;
         auto tiles = [&](int bn) { return n_ft * ((n + bn - 1) / bn) * k_splits; };
         while (p.BN > 64 && tiles(p.BN) * 2 < sms && n > p.BN / 2) p.BN /= 2;
+        // ... or when the tiles of the last wave would keep a few CTAs busy while the others idle (192 tiles of 256
+        // rows on 148 SMs take two full tile times; 384 tiles of 128 rows take three half ones).  Cost of a width =
+        // waves x (rows of a tile + a per-tile overhead worth ~32 rows); the widest of the cheapest widths wins.
+        static const int quant = tuning_int("CDB_GEMM_WAVES", 1);     // tuning hook: 0 = off
+        if (quant && tiles(p.BN) > sms) {
+            auto cost = [&](int bn) { return ((tiles(bn) + sms - 1) / sms) * (bn + 32); };
+            int best = p.BN;
+            for (int bn = p.BN / 2; bn >= 64; bn /= 2)
+                if (cost(bn) * 10 < cost(best) * 9) best = bn;
+            p.BN = best;
+        }
     }
     if ((forced_bn == 64 || forced_bn == 128 || forced_bn == 256) && forced_bn <= bn_max) p.BN = forced_bn;
-    const int stage_bytes = (mode == kModeSwiGLU ? 2 : 1) * BM * BK * 2 + p.BN * BK * 2;
+    // CTA pairs (CDB_FLAG_CTA_PAIRS): two CTAs share every activation tile of 128 or 256 rows, each loads half of it.
+    // Same sums in the same order as the single-CTA form.  Measured on the 2048-wide model it halves a CTA's activation
+    // traffic and changes the step time by -0.8 % (1024 rows) to +0.7 % (256 rows): at these sizes the main loop waits
+    // for the tensor pipe and the per-k-block hand-shake, not for L2, so the flag is off by default.
+    static const int pair_mask = tuning_int("CDB_GEMM_PAIR", 7);      // tuning hook: 1 store / split-K, 2 SwiGLU, 4 residual epilogue
+    const int pair_bit = mode == kModeSwiGLU ? 2 : mode == kModeAccumulate ? 4 : 1;
+    const bool use_pair = pair != nullptr && (h->cfg.flags & CDB_FLAG_CTA_PAIRS) && (pair_mask & pair_bit) && p.BN >= 128;
+    if (pair) *pair = use_pair;
+    const int x_rows = use_pair ? p.BN / 2 : p.BN;                   // activation rows a CTA loads per k-block
+    const int stage_bytes = (mode == kModeSwiGLU ? 2 : 1) * BM * BK * 2 + x_rows * BK * 2;
     static const int smem_cap = tuning_int("CDB_GEMM_SMEM_KB", kMaxSmem / 1024) * 1024;       // tuning hook
     int budget = smem_cap < kMaxSmem ? smem_cap : kMaxSmem;
     if (h->gemm_smem_cap > 0 && h->gemm_smem_cap < budget) budget = h->gemm_smem_cap;
@@ -895,9 +936,9 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
     } else {
         if (!make_map(map_w, W, N, K, BM) || !make_map(map_w2, W2 ? W2 : W, N, K, BM)) return 0;
     }
-    if (!make_map(map_x, x, n, K, p.BN)) return 0;
+    if (!make_map(map_x, x, n, K, x_rows)) return 0;
     *smem = (size_t)p.stages * stage_bytes + stage_out + 1024;
-    return n_ft * ((n + p.BN - 1) / p.BN) * k_splits;
+    return (use_pair ? (n_ft + 1) / 2 : n_ft) * ((n + p.BN - 1) / p.BN) * k_splits;      // tiles (of a pair: 256 features)
 }
 
 static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* W2, float* y, __nv_bfloat16* act, int n,
@@ -905,15 +946,17 @@ static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* 
     static bool attr_set_dev[kMaxDevices] = {};
     bool& attr_set = attr_set_dev[h->device];
     if (!attr_set) {
-        cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (tuning_int("CDB_GEMM_CARVEOUT", -2) > -2)           // tuning hook
-            cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, tuning_int("CDB_GEMM_CARVEOUT", -2));
+            cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout, tuning_int("CDB_GEMM_CARVEOUT", -2));
         attr_set = true;
     }
     GemmParams p;
     CUtensorMap map_w, map_w2, map_x;
     size_t smem = 0;
-    const int n_tiles = setup_gemm(h, x, W, W2, y, act, n, N, K, mode, k_splits, split_stride, p, &map_w, &map_w2, &map_x, &smem);
+    bool pair = false;
+    const int n_tiles = setup_gemm(h, x, W, W2, y, act, n, N, K, mode, k_splits, split_stride, p, &map_w, &map_w2, &map_x, &smem, &pair);
     if (!n_tiles) return false;
 #ifdef CDB_TUNING
     // tuning hook: device address of a stamp buffer (8 words per CTA), optionally for one launch kind only
@@ -922,8 +965,21 @@ static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* 
 #endif
     static const int part_sms = tuning_int("CDB_GEMM_SMS", 0);      // tuning hook (two-stream step only): CTA count of a projection
     const int sms = (part_sms > 0 && part_sms <= h->sms && h->attn_ctas_per_sm_cap > 0) ? part_sms : h->sms;
+    if (pair) {
+        // one persistent pair per two SMs, launched as clusters of two
+        const int pairs = n_tiles < sms / 2 ? n_tiles : sms / 2;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 2;
+        return cudaLaunchKernelEx(&cfg, gemm_bf16_tcgen05_kernel<true>, map_w, map_w2, map_x, p) == cudaSuccess;
+    }
     const int grid = n_tiles < sms ? n_tiles : sms;
-    launch_pdl(gemm_bf16_tcgen05_kernel, dim3(grid), dim3(kThreads), smem, st, map_w, map_w2, map_x, p);
+    launch_pdl(gemm_bf16_tcgen05_kernel<false>, dim3(grid), dim3(kThreads), smem, st, map_w, map_w2, map_x, p);
     return true;
 }
 

@@ -223,15 +223,17 @@ def test_in_cluster_sums_equal_workspace_sums_and_do_not_depend_on_the_batch(n_r
     """A model wide enough for real split-K (4 parts for the QKV and output projections, 8 for the down projection).
     Default flow: the parts are summed inside thread-block clusters, with RoPE and the KV page write in the QKV
     projection's epilogue.  Cross-check flow (flag 32): the parts go through a workspace and row-wise kernels.
-    Both add the same parts in the same order, so states, gate values, exit signals and the K/V written must agree
-    bit for bit - between the flows, and between a full batch (one to two 256-row tiles, ragged) and subsets."""
+    Flags 64 and 96 repeat both flows with the projections of 128 rows and more run by CTA pairs (one MMA over two
+    SMs that share the activation tile).  All of them add the same parts in the same order, so states, gate values, exit
+    signals and the K/V written must agree bit for bit - between the flows, and between a full batch (one to two
+    256-row tiles, ragged) and subsets."""
     ctxs = [1, 16, 17, 40, 255, 256, 257, 300, 33] + [int(c) for c in np.random.default_rng(2).integers(1, 90, n_rows - 9)]
     n = len(ctxs)
     rng = np.random.default_rng(1)
     h_np = rng.standard_normal((n, WIDE.d)).astype(np.float32)
     depth = rng.integers(1, WIDE.R + 1, n)
     results = {}
-    for flags in (0, 32):
+    for flags in (0, 32, 64, 96):
         B, cdb, _, table_np, pool, pool_np = setup(ctxs, max_rows=n, dims=WIDE, flags=flags)
         table = dev(table_np)
 
@@ -260,7 +262,7 @@ def test_in_cluster_sums_equal_workspace_sums_and_do_not_depend_on_the_batch(n_r
         cdb.destroy()
     full = results[0][0]
     assert all(np.isfinite(v[0].view(np.float32)).all() for v in full.values())
-    for flags in (0, 32):
+    for flags in (0, 32, 64, 96):
         for part in results[flags]:
             for i, (hh, gg, ff, kv) in part.items():
                 assert np.array_equal(kv, full[i][3]), (flags, i, "K/V")
