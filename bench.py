@@ -164,6 +164,7 @@ def main():
     ap.add_argument("--simt-gemm", action="store_true", help="run projections on the plain-FMA cross-check kernel")
     ap.add_argument("--two-stream", action="store_true", help="split the step into two half-batches on two streams (experimental)")
     ap.add_argument("--workspace-parts", action="store_true", help="split-K parts through a workspace instead of in-cluster sums (cross-check flow)")
+    ap.add_argument("--sm-partition", action="store_true", help="two half-batches with the SMs split between attention and projections (experimental)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cdb" else args.warmup
 
@@ -210,7 +211,7 @@ def main():
     from paper_2608_09444_b200 import binding as B
     from paper_2608_09444_b200.workloads import LoopStepWorkload
     wl = LoopStepWorkload(dims, n_rows=args.rows, seed=D.rank_seed(1, rank), ctx_lo=args.ctx_lo, ctx_hi=args.ctx_hi,
-                          permute=not args.contiguous_pages, device=f"cuda:{local_rank}", flags=(B.FLAG_SIMT_GEMM if args.simt_gemm else 0) | (B.FLAG_TWO_STREAM if args.two_stream else 0) | (B.FLAG_WORKSPACE_PARTS if args.workspace_parts else 0))
+                          permute=not args.contiguous_pages, device=f"cuda:{local_rank}", flags=(B.FLAG_SIMT_GEMM if args.simt_gemm else 0) | (B.FLAG_TWO_STREAM if args.two_stream else 0) | (B.FLAG_WORKSPACE_PARTS if args.workspace_parts else 0) | (B.FLAG_SM_PARTITION if args.sm_partition else 0))
     alg = wl.algorithmic()
     cores = len(os.sched_getaffinity(0))
 

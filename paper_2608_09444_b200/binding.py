@@ -28,6 +28,7 @@ FLAG_SIMT_PREFILL = 8
 FLAG_FUSED_STAGES = 16
 FLAG_WORKSPACE_PARTS = 32
 FLAG_CTA_PAIRS = 64
+FLAG_SM_PARTITION = 128
 
 EXPORTS = ["cdb_create", "cdb_destroy", "cdb_last_error", "cdb_kv_bind", "cdb_set_gate", "cdb_boundary_embed",
            "cdb_boundary_prelude", "cdb_loop_step", "cdb_compact", "cdb_gather_rows", "cdb_boundary_coda_lmhead",

@@ -335,7 +335,7 @@ static void launch_attention_t(const cdb* h, const AttnParams& p, void* o, cudaS
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, attn_split_kernel<T, DH, LPT, CPL, LAT>, 128, 0);
         if (blocks_per_sm < 1) blocks_per_sm = 1;
     }
-    const int sms = h->sms;
+    const int sms = h->part_active ? h->part_attn_sms : h->sms;
     const int max_items = p.rows.n_rows * p.pool.H * p.max_splits;
     // Warps are independent, so the CTA shape only decides how the block scheduler packs the SMs.
     // Alone: CTAs of 4 warps, as many as fit.  Sharing the GPU with the other half-batch's kernels: one
@@ -351,7 +351,17 @@ static void launch_attention_t(const cdb* h, const AttnParams& p, void* o, cudaS
     if (part_sms > 0 && part_sms <= sms && h->attn_ctas_per_sm_cap > 0) { grid = part_sms; threads = 128 * blocks_per_sm; }
     const int warps_per_cta = threads / 32;
     if ((max_items + warps_per_cta - 1) / warps_per_cta < grid) grid = (max_items + warps_per_cta - 1) / warps_per_cta;
-    {
+    if (h->part_active) {
+        // SM-partitioned step: the KV stream runs on the attention partition's stream (both half-batches in turn),
+        // fenced by events against this half-batch's own stream on the projection partition
+        const int half = h->part_active - 1;
+        cudaEventRecord(h->ev_pre[half], st);
+        cudaStreamWaitEvent(h->part_attn, h->ev_pre[half], 0);
+        CDB_LAUNCH(h);
+        launch_pdl(attn_split_kernel<T, DH, LPT, CPL, LAT>, dim3(grid), dim3(threads), 0, h->part_attn, p);
+        cudaEventRecord(h->ev_post[half], h->part_attn);
+        cudaStreamWaitEvent(st, h->ev_post[half], 0);
+    } else {
         ProfScope ps(h, kProfAttention, st);
         CDB_LAUNCH(h);
         launch_pdl(attn_split_kernel<T, DH, LPT, CPL, LAT>, dim3(grid), dim3(threads), 0, st, p);

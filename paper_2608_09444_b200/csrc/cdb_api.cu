@@ -7,6 +7,8 @@
 #include <new>
 #include <vector>
 
+#include <cuda.h>
+
 #include "cdb_internal.h"
 
 using namespace cdbk;
@@ -145,7 +147,7 @@ void layer_forward_tc(cdb_t* h, int ln, int layer, const RowsDev& rows, float* x
     // and the KV page write in its epilogue wins up to 128 rows (one launch fewer), the in-cluster residual sums up
     // to 64 rows (-4 % step time at 64 rows, -7.5 % at 16); at 256 rows the exchange through distributed shared
     // memory costs as much as the workspace round trip it replaces and the step is 1 % slower.
-    const bool in_cluster = !(c.flags & (CDB_FLAG_WORKSPACE_PARTS | CDB_FLAG_FUSED_STAGES));
+    const bool in_cluster = !(c.flags & (CDB_FLAG_WORKSPACE_PARTS | CDB_FLAG_FUSED_STAGES)) && !h->part_active;
     static const int cluster_mask = tuning_int("CDB_CLUSTER_MASK", 7);       // tuning hook: 1 QKV, 2 output, 4 down projection
     static const int cluster_rows_qkv = tuning_int("CDB_CLUSTER_ROWS_QKV", 128), cluster_rows_res = tuning_int("CDB_CLUSTER_ROWS_RES", 64);
     {
@@ -251,11 +253,80 @@ void lm_head(cdb_t* h, int ln, const RowsDev& rows, const float* x, int32_t* tok
     launch_argmax(h, logits, rows.n_rows, token_out, st);
 }
 
+// ---- SM partition: two green contexts (driver API, looked up at run time like the tensor-map encoder) ------------
+constexpr int kPartitionAttnSms = 112;     // SMs of the attention partition (a multiple of 8); the rest run the projections
+
+template <typename F> bool driver_fn(const char* name, F* out) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPointByVersion(name, &p, CUDA_VERSION, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess || !p) return false;
+    *out = (F)p;
+    return true;
+}
+
+void free_sm_partition(cdb_t* h) {
+    if (h->part_attn) cudaStreamDestroy(h->part_attn);
+    for (cudaStream_t& s : h->part_proj) if (s) cudaStreamDestroy(s);
+    h->part_attn = nullptr; h->part_proj[0] = h->part_proj[1] = nullptr;
+    for (int i = 0; i < 2; ++i) {
+        if (h->ev_pre[i]) cudaEventDestroy(h->ev_pre[i]);
+        if (h->ev_post[i]) cudaEventDestroy(h->ev_post[i]);
+        h->ev_pre[i] = h->ev_post[i] = nullptr;
+    }
+    CUresult (*destroy)(CUgreenCtx) = nullptr;
+    if ((h->green[0] || h->green[1]) && driver_fn("cuGreenCtxDestroy", &destroy))
+        for (void*& g : h->green) { if (g) destroy((CUgreenCtx)g); g = nullptr; }
+}
+
+// Leaves h->green[0] == NULL (and the flag without effect) when the driver cannot partition the SMs.
+void make_sm_partition(cdb_t* h) {
+    CUresult (*get_res)(CUdevice, CUdevResource*, CUdevResourceType) = nullptr;
+    CUresult (*split)(CUdevResource*, unsigned int*, const CUdevResource*, CUdevResource*, unsigned int, unsigned int) = nullptr;
+    CUresult (*gen_desc)(CUdevResourceDesc*, CUdevResource*, unsigned int) = nullptr;
+    CUresult (*create)(CUgreenCtx*, CUdevResourceDesc, CUdevice, unsigned int) = nullptr;
+    CUresult (*stream_create)(CUstream*, CUgreenCtx, unsigned int, int) = nullptr;
+    CUresult (*dev_get)(CUdevice*, int) = nullptr;
+    if (!driver_fn("cuDeviceGetDevResource", &get_res) || !driver_fn("cuDevSmResourceSplitByCount", &split) ||
+        !driver_fn("cuDevResourceGenerateDesc", &gen_desc) || !driver_fn("cuGreenCtxCreate", &create) ||
+        !driver_fn("cuGreenCtxStreamCreate", &stream_create) || !driver_fn("cuDeviceGet", &dev_get)) {
+        if (kTuningBuild) fprintf(stderr, "sm partition: driver entry points missing\n");
+        return;
+    }
+    static const int attn_sms = tuning_int("CDB_PART_ATTN_SMS", kPartitionAttnSms);     // tuning hook
+    CUdevice dev;
+    CUdevResource all, part[2];
+    unsigned int groups = 1;
+    if (dev_get(&dev, h->device) != CUDA_SUCCESS || get_res(dev, &all, CU_DEV_RESOURCE_TYPE_SM) != CUDA_SUCCESS ||
+        split(&part[0], &groups, &all, &part[1], 0, (unsigned int)attn_sms) != CUDA_SUCCESS || groups != 1 || part[1].sm.smCount < 8) {
+        if (kTuningBuild) fprintf(stderr, "sm partition: split failed (groups %u)\n", groups);
+        return;
+    }
+    CUgreenCtx g[2] = {nullptr, nullptr};
+    for (int i = 0; i < 2; ++i) {
+        CUdevResourceDesc desc;
+        if (gen_desc(&desc, &part[i], 1) != CUDA_SUCCESS || create(&g[i], desc, dev, CU_GREEN_CTX_DEFAULT_STREAM) != CUDA_SUCCESS) { g[i] = nullptr; break; }
+    }
+    CUstream sa = nullptr, sp[2] = {nullptr, nullptr};
+    const bool ok = g[0] && g[1] && stream_create(&sa, g[0], CU_STREAM_NON_BLOCKING, 0) == CUDA_SUCCESS &&
+                    stream_create(&sp[0], g[1], CU_STREAM_NON_BLOCKING, 0) == CUDA_SUCCESS &&
+                    stream_create(&sp[1], g[1], CU_STREAM_NON_BLOCKING, 0) == CUDA_SUCCESS;
+    h->green[0] = g[0]; h->green[1] = g[1];
+    h->part_attn = (cudaStream_t)sa; h->part_proj[0] = (cudaStream_t)sp[0]; h->part_proj[1] = (cudaStream_t)sp[1];
+    h->part_attn_sms = (int)part[0].sm.smCount; h->part_proj_sms = (int)part[1].sm.smCount;
+    for (int i = 0; i < 2; ++i) {
+        cudaEventCreateWithFlags(&h->ev_pre[i], cudaEventDisableTiming);
+        cudaEventCreateWithFlags(&h->ev_post[i], cudaEventDisableTiming);
+    }
+    if (kTuningBuild) fprintf(stderr, "sm partition: %s, attention %d SMs, projections %d SMs\n", ok ? "ready" : "stream / context creation failed", h->part_attn_sms, h->part_proj_sms);
+    if (!ok) free_sm_partition(h);
+}
+
 void free_all(cdb_t* h) {
     for (int i = 0; i < h->n_allocs; ++i) cudaFree(h->alloc_base[i]);     // every scratch buffer (with its guards)
     h->n_allocs = 0;
     for (int i = 0; i < h->n_tiled; ++i) if (h->tiled[i].tiled) cudaFree(h->tiled[i].tiled);
     h->n_tiled = 0;
+    free_sm_partition(h);
     if (h->side) cudaStreamDestroy(h->side);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
@@ -398,6 +469,7 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
         cudaMemset(h->grid_sync, 0, 3 * sizeof(unsigned int));
         for (int ln = 0; ln < 3; ++ln) cudaMemset(h->lane[ln].attn_counters, 0, sizeof(int32_t) * L);
         if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess) h->side = nullptr;
+        if (c.flags & CDB_FLAG_SM_PARTITION) make_sm_partition(h);
         cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
         cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
         cudaEventCreateWithFlags(&h->ev_attn[0], cudaEventDisableTiming);
@@ -498,7 +570,29 @@ int cdb_loop_step(cdb_t* h, const cdb_rows_t* rows, float* h_inout, float* gate_
         cudaMemcpyAsync(h->h_prev, h_inout, (size_t)rd.n_rows * c.d * sizeof(float), cudaMemcpyDeviceToDevice, st);
     const int n0 = (rd.n_rows + 1) / 2;
     const bool split = (c.flags & CDB_FLAG_TWO_STREAM) && h->side && rd.n_rows >= kMinSplitRows && !rd.n_live;   // (a half-batch view cannot shift a device-side count)
-    if (!split) {
+    const bool partitioned = (c.flags & CDB_FLAG_SM_PARTITION) && h->green[0] && rd.n_rows >= kMinSplitRows && !rd.n_live && use_tc_layers(h);
+    if (partitioned) {
+        // Two half-batches, the GPU's SMs split between two green contexts: the attention kernels of both halves run
+        // one after the other on the attention partition (the KV stream never stops), everything else of a half runs
+        // on the projection partition while the OTHER half's KV streams.
+        RowsDev half[2] = {rd, rd};
+        half[0].n_rows = n0;
+        half[1].n_rows = rd.n_rows - n0;
+        half[1].seq_id += n0; half[1].loop_depth += n0; half[1].position += n0; half[1].kv_slot += n0;
+        if (half[1].forced_exit) half[1].forced_exit += n0;
+        float* xs[2] = {h_inout, h_inout + (size_t)n0 * c.d};
+        cudaEventRecord(h->ev_fork, st);
+        for (int i = 0; i < 2; ++i) cudaStreamWaitEvent(h->part_proj[i], h->ev_fork, 0);
+        cudaStreamWaitEvent(h->part_attn, h->ev_fork, 0);
+        for (int i = 0; i < 2; ++i) { h->part_active = i + 1; launch_attention_plan(h, i, half[i], h->part_proj[i]); }
+        for (int l = c.L_pre; l < c.L_pre + c.L_core; ++l)
+            for (int i = 0; i < 2; ++i) {
+                h->part_active = i + 1;
+                core_layers(h, i, half[i], xs[i], h->part_proj[i], nullptr, nullptr, nullptr, l);
+            }
+        h->part_active = 0;
+        for (int i = 0; i < 2; ++i) { cudaEventRecord(h->ev_post[i], h->part_proj[i]); cudaStreamWaitEvent(st, h->ev_post[i], 0); }
+    } else if (!split) {
         h->attn_ctas_per_sm_cap = 0;
         launch_attention_plan(h, 0, rd, st);
         for (int l = c.L_pre; l < c.L_pre + c.L_core; ++l) core_layers(h, 0, rd, h_inout, st, nullptr, nullptr, nullptr, l);

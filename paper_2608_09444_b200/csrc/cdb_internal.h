@@ -130,6 +130,13 @@ struct cdb {
     size_t alloc_bytes[kMaxAllocs];
     int n_allocs;
 
+    // SM-partitioned execution of a loop step (CDB_FLAG_SM_PARTITION): two green contexts split the GPU's SMs;
+    // the attention kernels of both half-batches run on part_attn (in order), everything else of half i on part_proj[i]
+    void* green[2];                 // CUgreenCtx of the attention and of the projection partition (NULL: not available)
+    cudaStream_t part_attn, part_proj[2];
+    int part_attn_sms, part_proj_sms;
+    cudaEvent_t ev_pre[2], ev_post[2];
+    mutable int part_active;        // != 0 while such a step is being enqueued
     // two-stream execution of a loop step: second half-batch on `side`, joined by events
     cudaStream_t side;
     cudaEvent_t ev_fork, ev_join, ev_attn[2];

@@ -891,7 +891,7 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
     // prompt processing): narrower row tiles then give more CTAs a share of the weight stream.  The tile
     // width changes which CTA computes an output element, never how it is summed.
     {
-        const int sms = h->sms;
+        const int sms = h->part_active ? h->part_proj_sms : h->sms;
         auto tiles = [&](int bn) { return n_ft * ((n + bn - 1) / bn) * k_splits; };
         while (p.BN > 64 && tiles(p.BN) * 2 < sms && n > p.BN / 2) p.BN /= 2;
         // ... or when the tiles of the last wave would keep a few CTAs busy while the others idle (192 tiles of 256
@@ -964,7 +964,7 @@ static bool launch_gemm(const cdb* h, const void* x, const void* W, const void* 
     if (getenv("CDB_GEMM_DBG_ONLY") && atoi(getenv("CDB_GEMM_DBG_ONLY")) != mode * 100000 + N) p.dbg = nullptr;
 #endif
     static const int part_sms = tuning_int("CDB_GEMM_SMS", 0);      // tuning hook (two-stream step only): CTA count of a projection
-    const int sms = (part_sms > 0 && part_sms <= h->sms && h->attn_ctas_per_sm_cap > 0) ? part_sms : h->sms;
+    const int sms = h->part_active ? h->part_proj_sms : (part_sms > 0 && part_sms <= h->sms && h->attn_ctas_per_sm_cap > 0) ? part_sms : h->sms;
     if (pair) {
         // one persistent pair per two SMs, launched as clusters of two
         const int pairs = n_tiles < sms / 2 ? n_tiles : sms / 2;

@@ -226,14 +226,15 @@ def test_in_cluster_sums_equal_workspace_sums_and_do_not_depend_on_the_batch(n_r
     Flags 64 and 96 repeat both flows with the projections of 128 rows and more run by CTA pairs (one MMA over two
     SMs that share the activation tile).  All of them add the same parts in the same order, so states, gate values, exit
     signals and the K/V written must agree bit for bit - between the flows, and between a full batch (one to two
-    256-row tiles, ragged) and subsets."""
+    256-row tiles, ragged) and subsets.  Flag 128 runs batches of 64 rows and more as two half-batches with the SMs
+    split between an attention and a projection partition (green contexts): the same numbers again."""
     ctxs = [1, 16, 17, 40, 255, 256, 257, 300, 33] + [int(c) for c in np.random.default_rng(2).integers(1, 90, n_rows - 9)]
     n = len(ctxs)
     rng = np.random.default_rng(1)
     h_np = rng.standard_normal((n, WIDE.d)).astype(np.float32)
     depth = rng.integers(1, WIDE.R + 1, n)
     results = {}
-    for flags in (0, 32, 64, 96):
+    for flags in (0, 32, 64, 96, 128):
         B, cdb, _, table_np, pool, pool_np = setup(ctxs, max_rows=n, dims=WIDE, flags=flags)
         table = dev(table_np)
 
@@ -262,7 +263,7 @@ def test_in_cluster_sums_equal_workspace_sums_and_do_not_depend_on_the_batch(n_r
         cdb.destroy()
     full = results[0][0]
     assert all(np.isfinite(v[0].view(np.float32)).all() for v in full.values())
-    for flags in (0, 32, 64, 96):
+    for flags in (0, 32, 64, 96, 128):
         for part in results[flags]:
             for i, (hh, gg, ff, kv) in part.items():
                 assert np.array_equal(kv, full[i][3]), (flags, i, "K/V")
