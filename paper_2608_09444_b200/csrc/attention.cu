@@ -748,3 +748,5 @@ void launch_attention_prefill(const cdb* h, int ln, int layer, const RowsDev& ro
 }
 
 }  // namespace cdbk
+
+CDB_TRACE_SETTER(trace_set_attention)

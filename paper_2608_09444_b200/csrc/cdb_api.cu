@@ -93,6 +93,11 @@ const void* layer_ptr(const cdb_t* h, const void* base, int layer, size_t elems_
 }
 
 bool use_tc_layers(const cdb_t* h);
+}
+#ifdef CDB_TUNING
+namespace cdbk { void trace_set_attention(unsigned long long*); void trace_set_misc(unsigned long long*); void trace_set_gemm(unsigned long long*); }
+#endif
+namespace {
 
 // One transformer layer on `x` (fp32 [n_rows, d], updated in place).  Steps A1-A6 of the loop step:
 // RMSNorm + QKV projection, RoPE + KV page write, paged attention, output projection + residual,
@@ -477,6 +482,12 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
         e = cudaDeviceSynchronize();
     }
     if (e != cudaSuccess) { free_all(h); delete h; cudaGetLastError(); return CDB_ERR_CUDA; }
+#ifdef CDB_TUNING
+    if (const char* t = getenv("CDB_TRACE")) {                   // tuning hook: device buffer for the kernels' start times
+        unsigned long long* p = (unsigned long long*)strtoull(t, nullptr, 0);
+        trace_set_attention(p); trace_set_misc(p); trace_set_gemm(p);
+    }
+#endif
     *out = h;
     return CDB_OK;
 }

@@ -167,7 +167,25 @@ __device__ __forceinline__ float rope_lo(float a1, float a2, float c, float s) {
 __device__ __forceinline__ float rope_hi(float a1, float a2, float c, float s) { return __fmaf_rn(a2, c, __fmul_rn(a1, s)); }
 
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#ifdef CDB_TUNING
+// Tuning builds: every kernel's thread 32 of block 0 records the time at which its wait for the previous kernel ended
+// (one shared buffer: word 0 counts, the times follow in launch order).  Each translation unit has its own copy of
+// the pointer, set by trace_set_*().
+static __device__ unsigned long long* t_trace;
+__device__ __forceinline__ void pdl_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (t_trace != nullptr && threadIdx.x == 32 && blockIdx.x == 0 && blockIdx.y == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t) :: "memory");
+        const unsigned long long i = atomicAdd(t_trace, 1ULL);
+        if (i < (1ULL << 20) - 2) t_trace[1 + i] = t;
+    }
+}
+#define CDB_TRACE_SETTER(name) namespace cdbk { void name(unsigned long long* p) { cudaMemcpyToSymbol(t_trace, &p, sizeof(p)); } }
+#else
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#define CDB_TRACE_SETTER(name)
+#endif
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {

@@ -920,11 +920,18 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
     static const int smem_cap = tuning_int("CDB_GEMM_SMEM_KB", kMaxSmem / 1024) * 1024;       // tuning hook
     int budget = smem_cap < kMaxSmem ? smem_cap : kMaxSmem;
     if (h->gemm_smem_cap > 0 && h->gemm_smem_cap < budget) budget = h->gemm_smem_cap;
-    const int stage_out = mode == kModeSwiGLU ? p.BN * BM * 2 : 0;   // output staging tile of the SwiGLU epilogue
+    // Output staging tile of the SwiGLU epilogue.  When every CTA has a single tile (decode batches), the tile is
+    // staged in the ring itself - idle by then: all its stages were consumed before the accumulator completed and
+    // nothing refills it - which leaves the whole budget to the ring (4 instead of 3 stages of 48 KB).
+    const int tiles_now = (use_pair ? (n_ft + 1) / 2 : n_ft) * ((n + p.BN - 1) / p.BN) * k_splits;
+    const int ctas_now = (h->part_active ? h->part_proj_sms : h->sms) / (use_pair ? 2 : 1);
+    static const int alias_ok = tuning_int("CDB_GEMM_ALIAS", 1);      // tuning hook
+    const bool alias_out = mode == kModeSwiGLU && alias_ok && tiles_now <= ctas_now && !(h->cfg.flags & CDB_FLAG_FUSED_STAGES) && p.BN * BM * 2 <= 2 * stage_bytes;
+    const int stage_out = mode == kModeSwiGLU && !alias_out ? p.BN * BM * 2 : 0;
     p.stages = (budget - 1024 - stage_out) / stage_bytes;
     if (p.stages < 2) p.stages = 2;
     if (p.stages > 8) p.stages = 8;
-    p.stage_out_off = (uint32_t)(p.stages * stage_bytes);
+    p.stage_out_off = alias_out ? 0u : (uint32_t)(p.stages * stage_bytes);
     p.status = h->status;
     p.dbg = nullptr;
     const int n_kb = (K + BK - 1) / BK;
@@ -1179,3 +1186,5 @@ int launch_layer_tail_tc(const cdb* h, int ln, const RowsDev& rows, float* x, co
 }
 
 }  // namespace cdbk
+
+CDB_TRACE_SETTER(trace_set_gemm)

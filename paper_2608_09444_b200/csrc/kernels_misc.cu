@@ -478,3 +478,5 @@ void launch_copy_on_exit(const cdb* h, const RowsDev& rows, const int32_t* exit_
 }
 
 }  // namespace cdbk
+
+CDB_TRACE_SETTER(trace_set_misc)

@@ -28,14 +28,18 @@ def test_c2_full_size_step_matches_oracle_on_sampled_rows():
     wl = LoopStepWorkload(synth.OURO_1P4B, n_rows=256, seed=1)
     dm = wl.dims
     r = wl.rows_np
-    # ---- sample: shortest and longest context, one row per loop depth, two exits, two survivors
+    # ---- sample of 16 rows: shortest and longest context, one row per loop depth, two exits, two survivors, ...
     flags = np.array([O.exit_now(int(r["loop_depth"][i]), dm.R, int(r["fire_prev"][i]), 0, 1) for i in range(256)])
     sample = {int(np.argmin(wl.ctx)), int(np.argmax(wl.ctx))}
     for d in range(1, dm.R + 1):
         sample.add(int(np.flatnonzero(r["loop_depth"] == d)[0]))
     sample.update(int(i) for i in np.flatnonzero(flags)[:2])
     sample.update(int(i) for i in np.flatnonzero(~flags)[:2])
+    for i in range(5, 256, 19):                            # ... and rows spread over the batch, up to 16 in all
+        if len(sample) < 16:
+            sample.add(i)
     sample = sorted(sample)
+    assert len(sample) == 16
     items = wl.oracle_inputs(sample)                       # before the step: the step overwrites the rows' slots
 
     wl.step_resident()
@@ -97,4 +101,4 @@ def test_c2_full_size_step_matches_oracle_on_sampled_rows():
     print(f"sampled rows {sample}: hidden {worst_h:.2e}, kv {worst_kv:.2e}, logits {worst_logit:.2e}; "
           f"near-threshold gates excluded {near_threshold}, near-tie tokens {explained}")
     assert worst_h <= TOL and worst_kv <= TOL and worst_logit <= TOL
-    assert near_threshold <= 1 and explained <= 1
+    assert near_threshold <= 2 and explained <= 2
