@@ -1026,7 +1026,8 @@ static int splitk_parts(const cdb* h, int N, int K, int max_splits) {
     if (splits > n_kb / 4) splits = n_kb / 4;
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
-    if (!(h->cfg.flags & CDB_FLAG_FUSED_STAGES))
+    static const int fit_aware = tuning_int("CDB_SPLITK_FIT", 1);      // tuning hook: 0 = part counts ignore what clusters fit
+    if (fit_aware && !(h->cfg.flags & CDB_FLAG_FUSED_STAGES))
         while (splits > 1 && cluster_fit(h, splits) > 0 && cluster_fit(h, splits) < n_ft) --splits;
     return splits;
 }
