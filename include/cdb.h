@@ -84,8 +84,9 @@ enum { CDB_FLAG_SIMT_GEMM = 1,         /* run bf16 projections on the plain-FMA 
                                          * the stages (experimental: measured slower than the separate, programmatically chained launches) */
        CDB_FLAG_WORKSPACE_PARTS = 32,  /* split-K parts of the decode projections through a workspace and a row-wise kernel instead of being
                                          * summed inside thread-block clusters (cross-check: the sums and their order are the same) */
-       CDB_FLAG_CTA_PAIRS = 64,      /* projections on 128 rows and more run as CTA pairs (one 256-feature MMA over two SMs, each CTA loading
-                                         * its own weights and half of the activation tile); same results bit for bit, measured no faster */
+       CDB_FLAG_CTA_PAIRS = 64,        /* projections on 128 rows and more run as CTA pairs (one 256-feature MMA over two SMs, each CTA loading
+                                         * its own weights and half of the activation tile); same results bit for bit.  Without the flag pairs
+                                         * are used from 512 rows on (prompt processing, very large batches), where they are faster */
        CDB_FLAG_SM_PARTITION = 128 };  /* a loop step of >= 64 rows runs as two half-batches with the SMs split between two green contexts:
                                          * the attention kernels of both halves back to back on one partition, everything else on the other
                                          * (experimental; same results bit for bit; uses the boundary calls' scratch like the two-stream flag;

@@ -875,6 +875,8 @@ void launch_repack_tiled(const void* W, void* Wt, int layers, int N, int K, cuda
     repack_tiled_kernel<<<148 * 8, 256, 0, st>>>((const __nv_bfloat16*)W, (__nv_bfloat16*)Wt, layers, N, K);
 }
 
+static int cluster_fit(const cdb* h, int size);
+
 // Parameters and tensor maps of one projection.  W2 / act only in SwiGLU mode.  k_splits > 1 only with
 // kModeStore (y = workspace).  Returns the number of tiles, 0 on failure.
 static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2, float* y, __nv_bfloat16* act, int n,
@@ -907,13 +909,15 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
         }
     }
     if ((forced_bn == 64 || forced_bn == 128 || forced_bn == 256) && forced_bn <= bn_max) p.BN = forced_bn;
-    // CTA pairs (CDB_FLAG_CTA_PAIRS): two CTAs share every activation tile of 128 or 256 rows, each loads half of it.
-    // Same sums in the same order as the single-CTA form.  Measured on the 2048-wide model it halves a CTA's activation
-    // traffic and changes the step time by -0.8 % (1024 rows) to +0.7 % (256 rows): at these sizes the main loop waits
-    // for the tensor pipe and the per-k-block hand-shake, not for L2, so the flag is off by default.
+    // CTA pairs: two CTAs share every activation tile of 128 or 256 rows, each loads half of it.  Same sums in the
+    // same order as the single-CTA form.  Measured on the 2048-wide model: prompt calls (thousands of rows, where the
+    // projections are bound by the tensor pipe and the L2-to-SM traffic) get 3.5-4.5 % faster and decode steps of 512 and
+    // 1024 rows 0.4-0.9 %; at 256 rows the step is 0.2-0.7 % slower (there the main loop waits for the per-k-block
+    // hand-shake, not for L2).  So pairs are used from 512 rows on; CDB_FLAG_CTA_PAIRS forces them from 128 rows on.
     static const int pair_mask = tuning_int("CDB_GEMM_PAIR", 7);      // tuning hook: 1 store / split-K, 2 SwiGLU, 4 residual epilogue
     const int pair_bit = mode == kModeSwiGLU ? 2 : mode == kModeAccumulate ? 4 : 1;
-    const bool use_pair = pair != nullptr && (h->cfg.flags & CDB_FLAG_CTA_PAIRS) && (pair_mask & pair_bit) && p.BN >= 128;
+    const bool use_pair = pair != nullptr && ((h->cfg.flags & CDB_FLAG_CTA_PAIRS) || n >= 512) && (pair_mask & pair_bit) && p.BN >= 128 &&
+                          !h->part_active && cluster_fit(h, 2) > 0;
     if (pair) *pair = use_pair;
     const int x_rows = use_pair ? p.BN / 2 : p.BN;                   // activation rows a CTA loads per k-block
     const int stage_bytes = (mode == kModeSwiGLU ? 2 : 1) * BM * BK * 2 + x_rows * BK * 2;
