@@ -59,15 +59,17 @@ class Engine:
             self.n_pages_b = boundary_pages or max(1, n_pages // self.n_slots)
             self.pool_b = torch.zeros((dims.L_pre + dims.L_coda, self.n_pages_b, 2, dims.H, dims.page_size, dims.Dh), dtype=dt, device=self.dev)
             self.free_pages_b = list(range(self.n_pages_b - 1, -1, -1))
-            self.page_table_b_host = np.full((max_live, self.max_pages), -1, dtype=np.int32)
-            self.page_table_b = torch.from_numpy(self.page_table_b_host.copy()).to(self.dev)
+            self._page_table_b_pin = torch.full((max_live, self.max_pages), -1, dtype=torch.int32).pin_memory()
+            self.page_table_b_host = self._page_table_b_pin.numpy()       # the host's table lives in pinned memory: row updates go out as asynchronous copies
+            self.page_table_b = self._page_table_b_pin.to(self.dev)
             self.cdb.kv_bind_boundary(self.pool_b, self.page_table_b)
         self.pool = torch.zeros((dims.L_core if self.split_kv else dims.L, n_pages, 2, dims.H, dims.page_size, dims.Dh), dtype=dt, device=self.dev)
         self.cdb.kv_bind(self.pool)
         self.n_pages = n_pages
         self.free_pages = list(range(n_pages - 1, -1, -1))            # pop() hands out the lowest id first
-        self.page_table_host = np.full((max_live * self.n_slots, self.max_pages), -1, dtype=np.int32)
-        self.page_table = torch.from_numpy(self.page_table_host.copy()).to(self.dev)
+        self._page_table_pin = torch.full((max_live * self.n_slots, self.max_pages), -1, dtype=torch.int32).pin_memory()
+        self.page_table_host = self._page_table_pin.numpy()
+        self.page_table = self._page_table_pin.to(self.dev)
         i32 = dict(dtype=torch.int32, device=self.dev)
         f32 = dict(dtype=torch.float32, device=self.dev)
         d = dims.d
@@ -93,8 +95,9 @@ class Engine:
         # Recurrent step as a CUDA graph per row-count bucket (rows padded with seq_id = -1 to a multiple of 32):
         # the descriptor lives in fixed device arrays refreshed by one host-to-device copy per step.
         self.use_graphs = use_graphs
-        self.desc_host = torch.zeros((6, max_rows), dtype=torch.int32).pin_memory()    # five descriptor rows; [5, 0] = live rows
-        self.desc_dev = torch.zeros((6, max_rows), **i32)
+        # five descriptor rows; [5, 0] = live rows; row 6 = h_ready slots of the rows that join (pipelined engine)
+        self.desc_host = torch.zeros((7, max_rows), dtype=torch.int32).pin_memory()
+        self.desc_dev = torch.zeros((7, max_rows), **i32)
         self.graphs = {}
         # optional accounting of device time: CUDA-event pairs around every GPU phase the engine enqueues
         self.time_device = time_device
@@ -123,13 +126,40 @@ class Engine:
         """Brackets the GPU work enqueued inside with an event pair (no-op unless time_device)."""
         return Engine._Phase(self, name)
 
+    def _mark_decode_start(self):
+        """Event at the start of the decode phase: brackets recorded before it are left out of the busy time."""
+        if self.time_device:
+            self._decode_start_ev = torch.cuda.Event(enable_timing=True)
+            self._decode_start_ev.record()
+
     def _collect_device_time(self):
-        """stats["device_ms"][phase] = summed event time of that phase's brackets (after a synchronize)."""
+        """stats["device_ms"][phase] = summed event time of that phase's brackets (after a synchronize).
+        stats["device_busy_ms"] = length of the UNION of all brackets of the decode phase, whatever stream they were
+        recorded on (phases that overlap on two streams count once): wall - busy is the time the GPU had nothing of
+        the engine to run, the per-step device idle of the paper's Fig. 3."""
         out = {}
         for name, a, b in self._dev_events:
             out[name] = out.get(name, 0.0) + a.elapsed_time(b)
-        self._dev_events = []
         self.stats["device_ms"] = out
+        spans = []
+        if self._dev_events:
+            base = self._dev_events[0][1]
+            t0 = base.elapsed_time(self._decode_start_ev) if getattr(self, "_decode_start_ev", None) is not None else 0.0
+            for name, a, b in self._dev_events:
+                s0, s1 = base.elapsed_time(a), base.elapsed_time(b)
+                if name != "prefill" and s1 > t0:
+                    spans.append((max(s0, t0), s1))
+        spans.sort()
+        busy, end = 0.0, None
+        for s0, s1 in spans:
+            if end is None or s0 > end:
+                busy += s1 - s0
+                end = s1
+            elif s1 > end:
+                busy += s1 - end
+                end = s1
+        self.stats["device_busy_ms"] = busy
+        self._dev_events = []
 
     # ------------------------------------------------------------------ descriptor helpers
     def _rows(self, seq_ids, positions, depths=None, slots=None, forced=None):
@@ -155,13 +185,14 @@ class Engine:
                 return False
             for j in range(need):
                 self.page_table_b_host[slot_id, j] = self.free_pages_b.pop()
-            self.page_table_b[slot_id].copy_(torch.from_numpy(self.page_table_b_host[slot_id]))
+            self.page_table_b[slot_id].copy_(self._page_table_b_pin[slot_id], non_blocking=True)
         for s in range(self.n_slots):
             row = slot_id * self.n_slots + s
             for j in range(need):
                 self.page_table_host[row, j] = self.free_pages.pop()
         rows = slice(slot_id * self.n_slots, (slot_id + 1) * self.n_slots)
-        self.page_table[rows].copy_(torch.from_numpy(self.page_table_host[rows]))
+        # (a sequence's rows are next written when it has finished, i.e. after every step that reads this copy)
+        self.page_table[rows].copy_(self._page_table_pin[rows], non_blocking=True)
         return True
 
     def _release_pages(self, slot_id: int):
@@ -348,6 +379,7 @@ class Engine:
             if "decode_start" not in self.stats and not waiting and not future:   # every prompt processed: decode phase begins
                 torch.cuda.synchronize(self.dev)
                 self.stats["decode_start"] = time.perf_counter()
+                self._mark_decode_start()
             # survivors are already at the front of h_rec in stable order; append refills (FIFO)
             n_keep = len(rec)
             take = []

@@ -107,7 +107,7 @@ class PipelinedEngine(Engine):
         ready, ready_free = [], list(range(self.cap - 1, -1, -1))     # (sid, slot in h_ready, event, iteration)
         coda_q, coda_free = [], list(range(self.cap - 1, -1, -1))     # (sid, depth, slot in h_coda)
         pending_tokens, pending_release = [], []
-        ring = [torch.zeros((6, self.max_rows), dtype=torch.int32).pin_memory() for _ in range(4)]
+        ring = [torch.zeros((7, self.max_rows), dtype=torch.int32).pin_memory() for _ in range(4)]
         tok_ring = [torch.zeros(self.cap, dtype=torch.int32).pin_memory() for _ in range(16)]
         tok_dev = torch.zeros(self.cap, dtype=torch.int32, device=dev)
         tokp_dev = torch.zeros(self.cap, dtype=torch.int32, device=dev)      # first tokens of a prompt call
@@ -268,41 +268,43 @@ class PipelinedEngine(Engine):
             with torch.cuda.stream(side):
                 if prev is not None and prev["ne"]:
                     side.wait_event(prev["G"])
-                    slots = [coda_free.pop() for _ in range(prev["ne"])]
-                    self.h_coda.index_copy_(0, i64(slots), self.h_exit2[prev["parity"]][:prev["ne"]])
+                with self._phase("boundary"):
+                    if prev is not None and prev["ne"]:
+                        slots = [coda_free.pop() for _ in range(prev["ne"])]
+                        self.h_coda.index_copy_(0, i64(slots), self.h_exit2[prev["parity"]][:prev["ne"]])
+                        ev = torch.cuda.Event()
+                        ev.record(side)
+                        x_done[prev["parity"]] = ev
+                        coda_q.extend((s, r, slot) for (s, r), slot in zip(prev["exits"], slots))
+                    if not coda_q or (len(coda_q) < self.min_coda_batch and not force):
+                        return
+                    items = list(coda_q)
+                    coda_q.clear()
+                    m = len(items)
+                    hin = self.h_coda_in[:m]
+                    cdb.gather_rows(self.h_coda, i32([it_[2] for it_ in items]), None, m, hin, stream=side)
+                    sids = [it_[0] for it_ in items]
+                    rows = B.Rows(i32([live_slot[s] for s in sids]), i32([P[s] + gen[s] - 1 for s in sids]), self.page_table)
+                    if self.kv_layout == B.KV_DEPTH_INDEXED:
+                        cdb.kv_copy_on_exit(rows, i32([it_[1] for it_ in items]), stream=side)
+                    cdb.boundary_coda_lmhead(rows, hin, tok_dev[:m], stream=side)
+                    buf = tok_ring[tok_calls % len(tok_ring)][:m]
+                    tok_calls += 1
+                    buf.copy_(tok_dev[:m], non_blocking=True)
                     ev = torch.cuda.Event()
                     ev.record(side)
-                    x_done[prev["parity"]] = ev
-                    coda_q.extend((s, r, slot) for (s, r), slot in zip(prev["exits"], slots))
-                if not coda_q or (len(coda_q) < self.min_coda_batch and not force):
-                    return
-                items = list(coda_q)
-                coda_q.clear()
-                m = len(items)
-                hin = self.h_coda_in[:m]
-                cdb.gather_rows(self.h_coda, i32([it_[2] for it_ in items]), None, m, hin, stream=side)
-                sids = [it_[0] for it_ in items]
-                rows = B.Rows(i32([live_slot[s] for s in sids]), i32([P[s] + gen[s] - 1 for s in sids]), self.page_table)
-                if self.kv_layout == B.KV_DEPTH_INDEXED:
-                    cdb.kv_copy_on_exit(rows, i32([it_[1] for it_ in items]), stream=side)
-                cdb.boundary_coda_lmhead(rows, hin, tok_dev[:m], stream=side)
-                buf = tok_ring[tok_calls % len(tok_ring)][:m]
-                tok_calls += 1
-                buf.copy_(tok_dev[:m], non_blocking=True)
-                ev = torch.cuda.Event()
-                ev.record(side)
-                pending_tokens.append((ev, buf, [(s, gen[s]) for s in sids]))
-                self.stats["coda_calls"] += 1
-                cont = []
-                for j, (s, r, slot) in enumerate(items):
-                    coda_free.append(slot)
-                    gen[s] += 1
-                    if gen[s] >= Ts[s]:
-                        pending_release.append((ev, s))
-                    else:
-                        cont.append(j)
-                if cont:
-                    enqueue_prelude([sids[j] for j in cont], fed_back([sids[j] for j in cont], tok_dev[:m][i64(cont)].contiguous()), side, it)
+                    pending_tokens.append((ev, buf, [(s, gen[s]) for s in sids]))
+                    self.stats["coda_calls"] += 1
+                    cont = []
+                    for j, (s, r, slot) in enumerate(items):
+                        coda_free.append(slot)
+                        gen[s] += 1
+                        if gen[s] >= Ts[s]:
+                            pending_release.append((ev, s))
+                        else:
+                            cont.append(j)
+                    if cont:
+                        enqueue_prelude([sids[j] for j in cont], fed_back([sids[j] for j in cont], tok_dev[:m][i64(cont)].contiguous()), side, it)
 
         rec, prev, it = [], None, 0
         while True:
@@ -321,21 +323,15 @@ class PipelinedEngine(Engine):
             if "decode_start" not in self.stats and not waiting and not future and not prefill_inflight:
                 torch.cuda.synchronize(dev)
                 self.stats["decode_start"] = time.perf_counter()
+                self._mark_decode_start()
             # ---- refills whose prelude was enqueued in an earlier iteration join this step
             take = []
             while ready and len(rec) + len(take) < self.max_batch and ready[0][3] < it:
                 take.append(ready.pop(0))
-            if take:
-                for _, _, ev, _ in take:
-                    if ev is not None:
-                        main.wait_event(ev)
-                cdb.gather_rows(self.h_ready, i32([t[1] for t in take]), None, len(take),
-                                self.h_rec[len(rec):len(rec) + len(take)])
-                gather_done = torch.cuda.Event()
-                gather_done.record(main)
-                for s, slot, _, _ in take:
-                    ready_free.append(slot)
-                    rec.append([s, 1])
+            n_keep = len(rec)
+            for s, slot, _, _ in take:
+                ready_free.append(slot)                     # (a reuse of the slot waits for this step's gather: gather_done)
+                rec.append([s, 1])
             k = len(rec)
             step = None
             if k:
@@ -348,8 +344,19 @@ class PipelinedEngine(Engine):
                 dh[3, :k] = torch.as_tensor(np.asarray([self._slot(r) for _, r in rec], dtype=np.int32))
                 dh[4, :k] = torch.as_tensor(np.asarray([forced_for(s) for s, _ in rec], dtype=np.int32))
                 dh[5, 0] = k                                # device-side live count: the rows behind it are pads
+                if take:
+                    dh[6, :len(take)] = torch.as_tensor(np.asarray([t[1] for t in take], dtype=np.int32))
                 with self._phase("recurrent"):
+                    # one pinned block carries everything the step needs from the host (a pageable copy here would
+                    # make the host wait for the previous step and leave the GPU idle while the next one is enqueued)
                     self.desc_dev.copy_(dh, non_blocking=True)
+                    if take:
+                        for _, _, ev, _ in take:
+                            if ev is not None:
+                                main.wait_event(ev)
+                        cdb.gather_rows(self.h_ready, self.desc_dev[6, :len(take)], None, len(take), self.h_rec[n_keep:n_keep + len(take)])
+                        gather_done = torch.cuda.Event()
+                        gather_done.record(main)
                     g, rows = self.pgraphs[(nb, parity)]
                     cdb.compact(rows, self.surv_idx, self.exit_idx, self.counts)
                     lists_ready = torch.cuda.Event()

@@ -47,7 +47,9 @@ def run(dims, weights, prompts, T, *, mode, gate_kind, q_or_eps=0.5, forced_dept
            "generated_tokens_per_s_end_to_end": sum(len(t) for t in res["tokens"]) / (st["end"] - st["start"]),
            "decode_s": decode_s, "prefill_s": st["decode_start"] - st["start"],
            "decode_tokens_per_s": len(depths) / decode_s, "token_loop_steps_per_s": st["row_steps"] / decode_s,
-           "device_ms": st.get("device_ms"), "wall_ms_per_recurrent_step": 1e3 * decode_s / max(st["recurrent_steps"], 1),
+           "device_ms": st.get("device_ms"), "device_busy_ms": st.get("device_busy_ms"),
+           "device_idle_fraction": (1.0 - st["device_busy_ms"] / (1e3 * decode_s)) if st.get("device_busy_ms") else None,
+           "wall_ms_per_recurrent_step": 1e3 * decode_s / max(st["recurrent_steps"], 1),
            "recurrent_steps": st["recurrent_steps"], "row_steps": st["row_steps"], "coda_calls": st["coda_calls"],
            "mean_depth": float(depths.mean()), "depth_histogram": np.bincount(depths, minlength=dims.R + 1)[1:].tolist(),
            "status": eng.cdb.poll_status()}
