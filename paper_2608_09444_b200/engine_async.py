@@ -27,7 +27,7 @@ from .engine import Engine, _bucket, _static_rows
 
 
 class PipelinedEngine(Engine):
-    def __init__(self, *a, background_prefill=True, prefill_priority=0, **kw):
+    def __init__(self, *a, background_prefill=True, prefill_priority=0, eager_refill=True, **kw):
         kw.setdefault("mode", "refill")
         kw.setdefault("lookahead", True)
         super().__init__(*a, **kw)
@@ -41,6 +41,17 @@ class PipelinedEngine(Engine):
         self.background_prefill = background_prefill
         # (prefill_priority 0 = below the decode streams, -1 = level with them)
         self.pstream = torch.cuda.Stream(device=self.dev, priority=prefill_priority)
+        # While the batch has free rows, the boundary stages of the rows that left after step N-1 can be enqueued
+        # BEFORE step N, which then waits for them on the device (no host wait): those tokens rejoin at once instead
+        # of sitting out a step, at the price of a bubble of one boundary pass for the surviving rows.  Taken when the
+        # rows that rejoin outweigh that bubble, boundary_ratio being the cost of a boundary pass in loop steps
+        # (twice the FLOP ratio: small steps are latency-bound): Ouro-like models (no boundary layers) take it at
+        # every step with free rows, Huginn-like ones (boundary as heavy as the core) never.  With a full batch
+        # (more live sequences than rows) the boundary stages run beside step N as described above.
+        self.eager_refill = eager_refill
+        dm = self.dims
+        per_layer = 4 * dm.d * dm.d + 3 * dm.d * dm.F
+        self.boundary_ratio = 2.0 * ((dm.L_pre + dm.L_coda) * per_layer + dm.V * dm.d) / (dm.L_core * per_layer)
         d = self.dims.d
         self.h_exit2 = [torch.zeros((self.max_rows, d), dtype=torch.float32, device=self.dev) for _ in range(2)]
         self.h_coda_in = torch.zeros((self.cap, d), dtype=torch.float32, device=self.dev)
@@ -117,6 +128,27 @@ class PipelinedEngine(Engine):
         exit_h = torch.zeros(self.max_rows, dtype=torch.int32).pin_memory()
         i64 = lambda a: torch.tensor(a, dtype=torch.int64, device=dev)
         i32 = lambda a: torch.tensor(np.asarray(a, dtype=np.int32), dtype=torch.int32, device=dev)
+        # index arrays of the side stream's boundary calls: one pinned block and one asynchronous copy per call (a
+        # copy from pageable memory would hold the host until the side stream has caught up with the running step)
+        width = max(self.cap, self.max_rows)
+        stage_ring = [(torch.zeros((9, width), dtype=torch.int32).pin_memory(),
+                       torch.zeros((9, width), dtype=torch.int32, device=dev), [None]) for _ in range(8)]
+        stage_calls = [0]
+
+        def staged(stream, *arrays):
+            """device copies of the given integer lists, sent as one block on `stream`"""
+            host, devb, ev = stage_ring[stage_calls[0] % len(stage_ring)]
+            stage_calls[0] += 1
+            if ev[0] is not None:
+                ev[0].synchronize()                     # the block's previous copy has left the pinned buffer
+            for j, a in enumerate(arrays):
+                if len(a):
+                    host[j, :len(a)] = torch.as_tensor(np.asarray(a, dtype=np.int32))
+            with torch.cuda.stream(stream):
+                devb.copy_(host, non_blocking=True)
+                ev[0] = torch.cuda.Event()
+                ev[0].record(stream)
+            return [devb[j, :len(a)] for j, a in enumerate(arrays)]
         self._capture_all()
         self.stats["start"] = time.perf_counter()
         self.stats["first_token_s"], self.stats["finish_s"] = [None] * n, [None] * n
@@ -151,17 +183,21 @@ class PipelinedEngine(Engine):
                 self._release_pages(live_slot[s])
                 free_slots.append(live_slot.pop(s))
 
-        def enqueue_prelude(sids, tok_t, stream, it):
-            """prelude of the device-resident input tokens tok_t of sequences sids -> h_ready; on `stream`"""
+        def enqueue_prelude(sids, tok_t, stream, it, pick=None):
+            """prelude of the device-resident input tokens of sequences sids -> h_ready; on `stream`.  The tokens
+            are tok_t, or its entries `pick` (indices into it)."""
             sl = [live_slot[s] for s in sids]
             pos = [P[s] + gen[s] - 1 for s in sids]
-            rows = B.Rows(i32(sl), i32(pos), self.page_table)
+            slots = [ready_free.pop() for _ in sids]
+            sl_d, pos_d, slots_d, pick_d = staged(stream, sl, pos, slots, pick if pick is not None else [])
+            if pick is not None:
+                tok_t = tok_t[pick_d.long()]
+            rows = B.Rows(sl_d, pos_d, self.page_table)
             out = self.h_pre_out[:len(sids)]
             (cdb.boundary_prelude if dims.L_pre > 0 else cdb.boundary_embed)(tok_t, rows, out, stream=stream)
-            slots = [ready_free.pop() for _ in sids]
             if gather_done is not None:
                 stream.wait_event(gather_done)          # a freed h_ready slot may still be read by the last refill gather
-            self.h_ready.index_copy_(0, i64(slots), out)
+            self.h_ready.index_copy_(0, slots_d.long(), out)
             ev = torch.cuda.Event()
             ev.record(stream)
             ready.extend((s, slot, ev, it) for s, slot in zip(sids, slots))
@@ -219,7 +255,8 @@ class PipelinedEngine(Engine):
                     cont.append(j)
             if cont:                                     # boundary calls share one scratch lane: all of them on the side stream
                 with torch.cuda.stream(side):
-                    enqueue_prelude([batch[j] for j in cont], fed_back([batch[j] for j in cont], i32(vals[cont])), side, it)
+                    first = staged(side, vals[cont])[0] if teacher_tokens is None else fed_back([batch[j] for j in cont], None)
+                    enqueue_prelude([batch[j] for j in cont], first, side, it)
 
         def admit():
             """prompt processing of waiting requests while live slots and pages are free (drains the pipeline)"""
@@ -271,7 +308,7 @@ class PipelinedEngine(Engine):
                 with self._phase("boundary"):
                     if prev is not None and prev["ne"]:
                         slots = [coda_free.pop() for _ in range(prev["ne"])]
-                        self.h_coda.index_copy_(0, i64(slots), self.h_exit2[prev["parity"]][:prev["ne"]])
+                        self.h_coda.index_copy_(0, staged(side, slots)[0].long(), self.h_exit2[prev["parity"]][:prev["ne"]])
                         ev = torch.cuda.Event()
                         ev.record(side)
                         x_done[prev["parity"]] = ev
@@ -282,11 +319,13 @@ class PipelinedEngine(Engine):
                     coda_q.clear()
                     m = len(items)
                     hin = self.h_coda_in[:m]
-                    cdb.gather_rows(self.h_coda, i32([it_[2] for it_ in items]), None, m, hin, stream=side)
                     sids = [it_[0] for it_ in items]
-                    rows = B.Rows(i32([live_slot[s] for s in sids]), i32([P[s] + gen[s] - 1 for s in sids]), self.page_table)
+                    from_d, sl_d, pos_d, depth_d = staged(side, [it_[2] for it_ in items], [live_slot[s] for s in sids],
+                                                          [P[s] + gen[s] - 1 for s in sids], [it_[1] for it_ in items])
+                    cdb.gather_rows(self.h_coda, from_d, None, m, hin, stream=side)
+                    rows = B.Rows(sl_d, pos_d, self.page_table)
                     if self.kv_layout == B.KV_DEPTH_INDEXED:
-                        cdb.kv_copy_on_exit(rows, i32([it_[1] for it_ in items]), stream=side)
+                        cdb.kv_copy_on_exit(rows, depth_d, stream=side)
                     cdb.boundary_coda_lmhead(rows, hin, tok_dev[:m], stream=side)
                     buf = tok_ring[tok_calls % len(tok_ring)][:m]
                     tok_calls += 1
@@ -303,8 +342,10 @@ class PipelinedEngine(Engine):
                             pending_release.append((ev, s))
                         else:
                             cont.append(j)
-                    if cont:
-                        enqueue_prelude([sids[j] for j in cont], fed_back([sids[j] for j in cont], tok_dev[:m][i64(cont)].contiguous()), side, it)
+                    if cont and teacher_tokens is None:
+                        enqueue_prelude([sids[j] for j in cont], tok_dev[:m], side, it, pick=cont)
+                    elif cont:
+                        enqueue_prelude([sids[j] for j in cont], fed_back([sids[j] for j in cont], None), side, it)
 
         rec, prev, it = [], None, 0
         while True:
@@ -324,6 +365,12 @@ class PipelinedEngine(Engine):
                 torch.cuda.synchronize(dev)
                 self.stats["decode_start"] = time.perf_counter()
                 self._mark_decode_start()
+            # ---- free rows in the batch: the rows that left after the previous step pass their boundary stages first
+            if (self.eager_refill and prev is not None and len(rec) + len(ready) < self.max_batch
+                    and prev["ne"] > self.boundary_ratio * (len(rec) + prev["ne"])):
+                boundary_for(prev, it - 1, force=self.min_coda_batch <= 1)
+                self.stats["eager_boundaries"] = self.stats.get("eager_boundaries", 0) + 1
+                prev = None
             # ---- refills whose prelude was enqueued in an earlier iteration join this step
             take = []
             while ready and len(rec) + len(take) < self.max_batch and ready[0][3] < it:

@@ -27,13 +27,14 @@ def flop_bound(dims, mean_depth):
 
 
 def run(dims, weights, prompts, T, *, mode, gate_kind, q_or_eps=0.5, forced_depths=None, max_batch=None, max_live=None,
-        min_coda_batch=1, max_prefill_rows=4096, pipelined=False, use_graphs=True, time_device=False, kv_layout=B.KV_SHARED):
+        min_coda_batch=1, max_prefill_rows=4096, pipelined=False, use_graphs=True, time_device=False, kv_layout=B.KV_SHARED,
+        eager_refill=True):
     n, P = len(prompts), max(len(p) for p in prompts)
     live = min(n, max_live or n)
     n_slots = {B.KV_SHARED: 1, B.KV_DEPTH_INDEXED: dims.R, B.KV_FIRST_THEN_SHARED: 2}[kv_layout]
     pages = live * n_slots * ((P + T + dims.page_size - 1) // dims.page_size)
     # all sequences live: prompts first, then the timed decode phase; a queue of waiting sequences: prompts overlap decode
-    kw = {"background_prefill": live < n} if pipelined else {}
+    kw = {"background_prefill": live < n, "eager_refill": eager_refill} if pipelined else {}
     eng = (PipelinedEngine if pipelined else Engine)(dims, weights, max_batch=min(max_batch or n, live), max_live=live, max_len=P + T, n_pages=pages, gate_kind=gate_kind, kv_layout=kv_layout,
                  q_or_eps=q_or_eps, lookahead=True, mode=mode, min_coda_batch=min_coda_batch,
                  max_prefill_rows=max_prefill_rows, record_ticks=False, use_graphs=use_graphs, time_device=time_device, **kw)
@@ -50,7 +51,7 @@ def run(dims, weights, prompts, T, *, mode, gate_kind, q_or_eps=0.5, forced_dept
            "device_ms": st.get("device_ms"), "device_busy_ms": st.get("device_busy_ms"),
            "device_idle_fraction": (1.0 - st["device_busy_ms"] / (1e3 * decode_s)) if st.get("device_busy_ms") else None,
            "wall_ms_per_recurrent_step": 1e3 * decode_s / max(st["recurrent_steps"], 1),
-           "recurrent_steps": st["recurrent_steps"], "row_steps": st["row_steps"], "coda_calls": st["coda_calls"],
+           "eager_boundaries": st.get("eager_boundaries", 0), "recurrent_steps": st["recurrent_steps"], "row_steps": st["row_steps"], "coda_calls": st["coda_calls"],
            "mean_depth": float(depths.mean()), "depth_histogram": np.bincount(depths, minlength=dims.R + 1)[1:].tolist(),
            "status": eng.cdb.poll_status()}
     eng.cdb.destroy()
@@ -110,6 +111,8 @@ def main():
                     help="depth_indexed = last-exited cache (copy-on-exit), section 4.2")
     ap.add_argument("--exits", default="forced", choices=["forced", "criterion"],
                     help="huginn: replayed geometric exit depths, or the convergence criterion with a calibrated threshold")
+    ap.add_argument("--no-eager-refill", action="store_true",
+                    help="pipelined engine: always run the boundary stages beside the next step (tokens rejoin one step late)")
     ap.add_argument("--time-device", action="store_true", help="bracket every GPU phase with CUDA events and report device_ms")
     args = ap.parse_args()
     known = {"cb", "refill", "no_refill", "refill_nographs", "cb_pipelined", "refill_pipelined"}
@@ -149,7 +152,7 @@ def main():
         mode = mode.replace("_pipelined", "").replace("_nographs", "")
         fixed = mode == "cb" and pipelined              # continuous batching on the pipelined engine: every token replays depth R
         out, _ = run(dims, w, prompts, args.tokens, mode="refill" if fixed else mode, pipelined=pipelined, use_graphs=not nographs,
-                     time_device=args.time_device, gate_kind=B.GATE_NONE if fixed else gate_kind, q_or_eps=q_or_eps,
+                     time_device=args.time_device, eager_refill=not args.no_eager_refill, gate_kind=B.GATE_NONE if fixed else gate_kind, q_or_eps=q_or_eps,
                      forced_depths=[[dims.R] * (args.tokens - 1)] * args.seqs if fixed else None if mode == "cb" else forced,
                      max_batch=args.max_batch or None, max_live=args.max_live or None, min_coda_batch=min_coda,
                      kv_layout={"shared": B.KV_SHARED, "depth_indexed": B.KV_DEPTH_INDEXED, "first_then_shared": B.KV_FIRST_THEN_SHARED}[args.kv_layout])

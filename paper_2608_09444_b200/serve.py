@@ -67,10 +67,10 @@ def merge_replicas(parts, n_requests):
 
 def run(dims, weights, arrivals, prompts, out_lens, *, mode, pipelined, gate_kind, q_or_eps=0.5, forced_depths=None,
         max_batch=256, max_live=320, pool_tokens=400000, min_coda_batch=1, max_prefill_rows=4096,
-        admit_min=1, admit_wait_s=0.0, prefill_priority=0, device="cuda:0"):
+        admit_min=1, admit_wait_s=0.0, prefill_priority=0, eager_refill=True, device="cuda:0"):
     max_len = max(len(p) + t for p, t in zip(prompts, out_lens))
     pages = (pool_tokens + dims.page_size - 1) // dims.page_size
-    extra = {"prefill_priority": prefill_priority} if pipelined else {}
+    extra = {"prefill_priority": prefill_priority, "eager_refill": eager_refill} if pipelined else {}
     eng = (PipelinedEngine if pipelined else Engine)(
         dims, weights, **extra, max_batch=max_batch, max_live=max_live, max_len=max_len, n_pages=pages, gate_kind=gate_kind,
         q_or_eps=q_or_eps, lookahead=True, mode=mode, min_coda_batch=min_coda_batch,
@@ -104,6 +104,8 @@ def main():
     ap.add_argument("--admit-wait-ms", type=float, default=0.0, help="... or the oldest has waited this long")
     ap.add_argument("--prefill-priority", type=int, default=0, choices=[0, -1],
                     help="pipelined engine: CUDA stream priority of prompt processing (0 = below the decode streams, -1 = level with them)")
+    ap.add_argument("--no-eager-refill", action="store_true",
+                    help="pipelined engine: always run the boundary stages beside the next step (tokens rejoin one step late)")
     ap.add_argument("--first-rate-index", type=int, default=0,
                     help="position of the first of --rates in the sweep it belongs to (the trace seed follows the position): "
                          "--rates 2 --first-rate-index 5 repeats the last trace of --rates 64,32,16,8,4,2")
@@ -148,7 +150,7 @@ def main():
                          max_batch=args.max_batch, max_live=args.max_live,
                          pool_tokens=args.pool_tokens, min_coda_batch=args.min_coda_batch or (1 if args.model == "ouro" else 8),
                          admit_min=args.admit_min, admit_wait_s=args.admit_wait_ms * 1e-3,
-                         prefill_priority=args.prefill_priority, device=f"cuda:{local_rank}")
+                         prefill_priority=args.prefill_priority, eager_refill=not args.no_eager_refill, device=f"cuda:{local_rank}")
             out["mode"] = mode
             parts = D.gather_objects({"ids": mine, "finish_s": out.pop("finish_s"), "first_token_s": out.pop("first_token_s"),
                                       "counters": {k: out[k] for k in ("recurrent_steps", "row_steps", "prefill_calls", "coda_calls")}})
