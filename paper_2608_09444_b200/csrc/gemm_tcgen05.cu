@@ -43,7 +43,8 @@ struct GemmParams {
     float* y;                   // store / accumulate: [k_splits][n][N] fp32 (split s at y + s * split_stride)
     __nv_bfloat16* act;         // SwiGLU mode: [n][N] bf16 = SiLU(x.Wg^T) * (x.Wu^T)
     int n, N, K;
-    int BN;                     // rows per tile (MMA N): 64, 128 or 256 (<= 128 in SwiGLU mode)
+    int BN;                     // rows per tile (MMA N): a multiple of 16, 64 to 256
+    int n_acc;                  // accumulator sets in TMEM: 2 (the epilogue of a tile runs beside the main loop of the next) or 1
     int stages;
     int mode;
     int k_splits;               // the K range is cut into this many parts, each a tile of its own
@@ -179,8 +180,8 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
             bool ok = true;
             const long long mma_t0 = clock64();
             for (int t = cta; t < n_tiles && ok; t += n_cta, ++it) {
-                const int acc = it & 1;
-                const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
+                const int acc = p.n_acc == 2 ? it & 1 : 0;
+                const uint32_t acc_ph = (uint32_t)(p.n_acc == 2 ? it >> 1 : it) & 1u;
                 if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, cx.abortp)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = cx.tmem_base + (uint32_t)acc * acc_cols;
@@ -217,8 +218,8 @@ __device__ __forceinline__ void gemm_roles(const CUtensorMap* map_w, const CUten
         int it = 0;
         bool ok = true;
         for (int t = cta; t < n_tiles && ok; t += n_cta, ++it) {
-            const int acc = it & 1;
-            const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
+            const int acc = p.n_acc == 2 ? it & 1 : 0;
+            const uint32_t acc_ph = (uint32_t)(p.n_acc == 2 ? it >> 1 : it) & 1u;
             const int f = (t % n_ftiles) * FT + (int)rank * BM + q * 32 + lane, r0 = (t / n_ftiles % n_rtiles) * BN;
             const int split = t / (n_ftiles * n_rtiles);
             if (!mbar_wait(acc_full_bar(acc), acc_ph, cx.abortp)) { ok = false; break; }
@@ -345,7 +346,8 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_w, const __grid
     auto empty_bar = [&](int s) { return bar0 + 8u * (8 + s); };
     auto acc_full_bar = [&](int a) { return bar0 + 8u * (16 + a); };
     auto acc_empty_bar = [&](int a) { return bar0 + 8u * (18 + a); };
-    const uint32_t tmem_cols = 2u * acc_cols;                               // double-buffered; 128, 256 or 512
+    uint32_t tmem_cols = 32;                                                // a power of two that holds the accumulator sets
+    while (tmem_cols < (uint32_t)p.n_acc * acc_cols) tmem_cols *= 2;
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -908,7 +910,12 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
             p.BN = best;
         }
     }
-    if ((forced_bn == 64 || forced_bn == 128 || forced_bn == 256) && forced_bn <= bn_max) p.BN = forced_bn;
+    static const int forced_bn_dual = tuning_int("CDB_GEMM_BN_SWIGLU", 0);      // tuning hook
+    {
+        const int f = mode == kModeSwiGLU ? forced_bn_dual : forced_bn;
+        if (f >= 64 && f <= 256 && f % 16 == 0) p.BN = f;
+    }
+    p.n_acc = (mode == kModeSwiGLU ? 4 : 2) * p.BN <= 512 ? 2 : 1;  // two accumulator sets when TMEM's 512 columns hold them
     // CTA pairs: two CTAs share every activation tile of 128 or 256 rows, each loads half of it.  Same sums in the
     // same order as the single-CTA form.  Measured on the 2048-wide model: prompt calls (thousands of rows, where the
     // projections are bound by the tensor pipe and the L2-to-SM traffic) get 3.5-4.5 % faster and decode steps of 512 and

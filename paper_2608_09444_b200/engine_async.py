@@ -5,7 +5,11 @@ which rows leave after it (the exit flag of step N depends only on the signal st
 compaction lists are computed at the START of step N), prepares the descriptor of step N+1 and enqueues
 it; the coda + sampling + prelude of the rows that left after step N-1 run on a second stream beside loop
 step N, and their tokens rejoin the recurrent batch at step N+1.  The main stream therefore never waits
-for the host or for a boundary stage.
+for the host or for a boundary stage.  While the batch has free rows and the boundary pass is cheap next to a
+step (no boundary layers), the boundary stages are instead enqueued before step N, which waits for them on the
+device: the tokens rejoin at step N (see eager_refill).  Either way the host never waits for the device
+except to read the exit lists of the step it has just enqueued, and everything it sends per step leaves
+from pinned memory.
 
 Streams and buffers
   main  H2D descriptor -> cdb_compact (lists) -> [event] -> CUDA graph (loop step, survivor gather to the
