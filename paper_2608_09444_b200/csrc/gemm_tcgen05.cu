@@ -910,6 +910,28 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
             p.BN = best;
         }
     }
+    // ... and a row tile need not be a power of two: any multiple of 16 rows is a valid MMA N.  r row tiles of
+    // ceil(n / r) rows (rounded up to 16) balance the tile count against the SM count: 512 rows of gate/up (44
+    // feature tiles) are 176 tiles of 128 rows - two waves, the second almost empty - or 132 tiles of 176 rows.
+    // Same cost measure as above; a width that no longer leaves TMEM room for two accumulator sets pays a
+    // quarter tile per extra wave (its epilogues are not hidden).
+    static const int chooser = tuning_int("CDB_GEMM_CHOOSER", 0);     // tuning hook: 1 = on
+    if (chooser && n > 64) {
+        const int sms = h->part_active ? h->part_proj_sms : h->sms;
+        const int dual = mode == kModeSwiGLU ? 2 : 1;
+        long best_cost = -1; int best_bn = p.BN;
+        for (int r = 1; r <= (n + 63) / 64; ++r) {
+            int bn = ((n + r - 1) / r + 15) / 16 * 16;
+            if (bn > 256 || bn * dual > 512) continue;
+            if (bn < 64) break;
+            const int r_eff = (n + bn - 1) / bn;
+            const long tiles = (long)n_ft * r_eff * k_splits, waves = (tiles + sms - 1) / sms;
+            const bool single = 2 * dual * bn > 512;
+            const long cost = waves * (bn + 32) + (single && waves > 1 ? (waves - 1) * (bn / 4) : 0);
+            if (best_cost < 0 || cost * 100 < best_cost * 95) { best_cost = cost; best_bn = bn; }
+        }
+        p.BN = best_bn;
+    }
     static const int forced_bn_dual = tuning_int("CDB_GEMM_BN_SWIGLU", 0);      // tuning hook
     {
         const int f = mode == kModeSwiGLU ? forced_bn_dual : forced_bn;
