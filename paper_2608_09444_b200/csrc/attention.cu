@@ -55,11 +55,6 @@ struct AttnParams {
     const int32_t* item_start; // [n_rows + 1]
     int32_t* counter;
     int32_t* status;
-    // Merge inside the split kernel: the warp that delivers the last partial of a (row, head) merges them all (in
-    // split order, like the merge kernel) and writes the output row.  done = arrival counts per (row, head), zero
-    // before the launch and zero again after it; out = [n_rows][H*Dh] (NULL: the merge kernel follows).
-    int32_t* done;
-    void* out;
 };
 
 // splits per row -> exclusive scan; zeroes the per-layer work counters.  One CTA.
@@ -68,7 +63,6 @@ struct AttnParams {
 // area's max_splits per (row, head).
 __global__ void __launch_bounds__(1024) attn_plan_kernel(RowsDev rows, int32_t* __restrict__ item_start,
                                                          int32_t* __restrict__ counters, int n_counters,
-                                                         int32_t* __restrict__ done, int n_done,
                                                          int max_position, int max_splits, int32_t* __restrict__ status) {
     pdl_trigger();
     pdl_wait();
@@ -77,7 +71,6 @@ __global__ void __launch_bounds__(1024) attn_plan_kernel(RowsDev rows, int32_t* 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) base = 0;
     for (int i = threadIdx.x; i < n_counters; i += 1024) counters[i] = 0;
-    for (int i = threadIdx.x; i < n_done; i += 1024) done[i] = 0;
     __syncthreads();
     for (int start = 0; start < rows.n_rows; start += 1024) {
         const int row = start + threadIdx.x;
@@ -107,20 +100,11 @@ __global__ void __launch_bounds__(1024) attn_plan_kernel(RowsDev rows, int32_t* 
     if (threadIdx.x == 0) item_start[rows.n_rows] = base;
 }
 
-template <typename T, int DH, bool CG>
-__device__ __forceinline__ void merge_parts(const float* __restrict__ part, int ns, T* __restrict__ o, int lane);
-// (a call, not inlined, with scalar arguments: the merge's registers must not weigh on the split kernel's main loop)
-template <typename T, int DH>
-__device__ __noinline__ void merge_in_split_kernel(const float* part, int ns, T* o, int lane) {
-    merge_parts<T, DH, true>(part, ns, o, lane);
-}
-
 // LAT: the variant for batches too small to fill the GPU, where a warp's own chain of memory latencies sets the
 // pace: the split's page ids come from one coalesced load, and the K/V tiles of the next page are in flight
 // while the current page is computed (twice the registers, which an almost empty GPU has to spare).  Same
 // arithmetic in the same order as the throughput variant.
-// FUSE: the kernel can also merge (see AttnParams::out); without it the merge is always a kernel of its own.
-template <typename T, int DH, int LPT, int CPL, bool LAT, bool FUSE>
+template <typename T, int DH, int LPT, int CPL, bool LAT>
 __global__ void __maxnreg__(LAT ? 208 : 96) attn_split_kernel(AttnParams p) {
     pdl_trigger();
     pdl_wait();
@@ -135,22 +119,12 @@ __global__ void __maxnreg__(LAT ? 208 : 96) attn_split_kernel(AttnParams p) {
     const int n_rows = p.rows.n_rows;
     const int total_items = p.item_start[n_rows] * H;
     const T* pool_base = (const T*)p.pool.base;
-    const bool fused_merge = FUSE && p.out != nullptr;
 
     for (;;) {
         int item = 0;
         if (lane == 0) item = atomicAdd(p.counter, 1);
         item = __shfl_sync(0xffffffffu, item, 0);
-        if (item >= total_items) {
-            // with the merge in this kernel, one more item per row: rows without any split (pads, rows the plan
-            // refused) get their output zeroed, which merge_row_head does for them
-            if (!fused_merge || item >= total_items + n_rows) break;
-            const int row = item - total_items;
-            const int sq = p.rows.seq_of(row);
-            if (sq < 0 || sq >= p.max_seqs || p.item_start[row + 1] - p.item_start[row] <= 0)
-                for (int head = 0; head < H; ++head) merge_in_split_kernel<T, DH>(nullptr, 0, (T*)p.out + ((size_t)row * H + head) * DH, lane);
-            continue;
-        }
+        if (item >= total_items) break;
         const int pair = item / H, head = item % H;
         int lo = 0, hi = n_rows;                 // last row with item_start[row] <= pair
         while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (p.item_start[mid] <= pair) lo = mid; else hi = mid; }
@@ -160,27 +134,7 @@ __global__ void __maxnreg__(LAT ? 208 : 96) attn_split_kernel(AttnParams p) {
         const int ctx = p.rows.position[row] + 1;
         float* part = p.part + ((size_t)(row * H + head) * p.max_splits + split) * (DH + 2);
         bool ok = seq >= 0 && seq < p.max_seqs && slot >= 0 && slot < p.rows.n_slots && split < p.max_splits;
-        // the last partial of a (row, head) to arrive brings the merge with it
-        // (everything it needs is derived again from the (row, head) index: nothing else stays live over the main loop)
-        const int rh = row * H + head;
-        auto arrive = [&](int rh_) {
-            if (!fused_merge) return;
-            __threadfence();
-            __syncwarp();
-            const int row_ = rh_ / p.pool.H;
-            const int ns = min(p.item_start[row_ + 1] - p.item_start[row_], p.max_splits);
-            int last = 0;
-            if (lane == 0) last = atomicAdd(p.done + rh_, 1) == ns - 1;
-            last = __shfl_sync(0xffffffffu, last, 0);
-            if (last) {
-                __threadfence();
-                const int sq = p.rows.seq_of(row_);
-                merge_in_split_kernel<T, DH>(p.part + (size_t)rh_ * p.max_splits * (DH + 2), sq >= 0 && sq < p.max_seqs ? ns : 0,
-                                             (T*)p.out + (size_t)rh_ * DH, lane);
-                if (lane == 0) p.done[rh_] = 0;
-            }
-        };
-        if (!ok) { if (lane == 0) atomicCAS(p.status, 0, kStatusSeq); arrive(rh); continue; }
+        if (!ok) { if (lane == 0) atomicCAS(p.status, 0, kStatusSeq); continue; }
         const int tok0 = split * kSplitTokens;
         const int tok1 = min(ctx, tok0 + kSplitTokens);
         const int32_t* table = p.rows.page_table + ((size_t)seq * p.rows.n_slots + slot) * p.rows.page_table_stride;
@@ -300,22 +254,30 @@ __global__ void __maxnreg__(LAT ? 208 : 96) attn_split_kernel(AttnParams p) {
                 for (int e = 0; e < EPC; ++e) part[(c + LPT * j) * EPC + e] = o[j][e];
             if (c == 0) { part[DH] = m; part[DH + 1] = l; }
         }
-        arrive(rh);
     }
 }
 
-// Merge of the ns partials of one (row, head) (at part, DH + 2 floats each) in split order, rounded to T, into the
-// DH outputs at o: the work of one warp.  ns <= 0 (pads, rows the plan or the split kernel skipped): zeros.
-// CG: the partials were written by other SMs during this kernel, so they are read from L2.
-template <typename T, int DH, bool CG>
-__device__ __forceinline__ void merge_parts(const float* __restrict__ part, int ns, T* __restrict__ o, int lane) {
+// Merge the splits of each (row, head) in split order and round to T.  One warp per (row, head).
+template <typename T, int DH>
+__global__ void __launch_bounds__(128) attn_merge_kernel(AttnParams p, T* __restrict__ out) {
+    pdl_trigger();
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const int H = p.pool.H;
+    const int wid = blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (blockIdx.x == 0 && threadIdx.x == 0) *p.counter = 0;      // the split kernel is done: re-arm its work counter
+    if (wid >= p.rows.n_rows * H) return;
+    const int row = wid / H, head = wid % H;
+    T* o = out + (size_t)row * H * DH + (size_t)head * DH;
     constexpr int PER = (DH + 31) / 32;
-    if (ns <= 0) {
+    const int ns = min(p.item_start[row + 1] - p.item_start[row], p.max_splits);
+    const int sq = p.rows.seq_of(row);
+    if (sq < 0 || sq >= p.max_seqs || ns <= 0) {          // pads and rows the plan or the split kernel skipped
 #pragma unroll
         for (int k = 0; k < PER; ++k) if (lane + 32 * k < DH) o[lane + 32 * k] = T(0.f);
         return;
     }
-    auto ld = [](const float* a) { return CG ? __ldcg(a) : *a; };
+    const float* part = p.part + (size_t)(row * H + head) * p.max_splits * (DH + 2);
     // Splits are taken four at a time with all their loads issued before the first use (a loop that waits for
     // each split's loads in turn costs one memory latency per split); the sums keep their split order.
     constexpr int U = 4;
@@ -323,7 +285,7 @@ __device__ __forceinline__ void merge_parts(const float* __restrict__ part, int 
     for (int s0 = 0; s0 < ns; s0 += U) {
         float mv[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) mv[u] = s0 + u < ns ? ld(part + (size_t)(s0 + u) * (DH + 2) + DH) : -INFINITY;
+        for (int u = 0; u < U; ++u) mv[u] = s0 + u < ns ? part[(size_t)(s0 + u) * (DH + 2) + DH] : -INFINITY;
 #pragma unroll
         for (int u = 0; u < U; ++u) M = fmaxf(M, mv[u]);
     }
@@ -336,9 +298,9 @@ __device__ __forceinline__ void merge_parts(const float* __restrict__ part, int 
         for (int u = 0; u < U; ++u) {
             const bool on = s0 + u < ns;
             const float* ps = part + (size_t)(on ? s0 + u : s0) * (DH + 2);
-            mv[u] = ld(ps + DH); lv[u] = ld(ps + DH + 1);
+            mv[u] = ps[DH]; lv[u] = ps[DH + 1];
 #pragma unroll
-            for (int k = 0; k < PER; ++k) ov[u][k] = lane + 32 * k < DH ? ld(ps + lane + 32 * k) : 0.f;
+            for (int k = 0; k < PER; ++k) ov[u][k] = lane + 32 * k < DH ? ps[lane + 32 * k] : 0.f;
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -355,40 +317,22 @@ __device__ __forceinline__ void merge_parts(const float* __restrict__ part, int 
     for (int k = 0; k < PER; ++k) if (lane + 32 * k < DH) o[lane + 32 * k] = T(acc[k] * inv);
 }
 
-// The merge as a kernel of its own (after a split kernel launched with out = NULL).  One warp per (row, head).
-template <typename T, int DH>
-__global__ void __launch_bounds__(128) attn_merge_kernel(AttnParams p, T* __restrict__ out) {
-    pdl_trigger();
-    pdl_wait();
-    const int lane = threadIdx.x & 31;
-    const int wid = blockIdx.x * 4 + (threadIdx.x >> 5);
-    if (blockIdx.x == 0 && threadIdx.x == 0) *p.counter = 0;      // the split kernel is done: re-arm its work counter
-    if (wid >= p.rows.n_rows * p.pool.H) return;
-    const int row = wid / p.pool.H;
-    const int ns = min(p.item_start[row + 1] - p.item_start[row], p.max_splits);
-    const int sq = p.rows.seq_of(row);
-    merge_parts<T, DH, false>(p.part + (size_t)wid * p.max_splits * (DH + 2), sq < 0 || sq >= p.max_seqs ? 0 : ns, out + (size_t)wid * DH, lane);
-}
-
 void launch_attention_plan(const cdb* h, int ln, const RowsDev& rows, cudaStream_t st) {
     CDB_LAUNCH(h);
     launch_pdl(attn_plan_kernel, dim3(1), dim3(1024), 0, st, rows, h->lane[ln].attn_item_start, h->lane[ln].attn_counters,
-               h->cfg.L_pre + h->cfg.L_core + h->cfg.L_coda, h->lane[ln].attn_done, rows.n_rows * h->cfg.H,
-               h->cfg.max_position, h->max_splits, h->status);
+               h->cfg.L_pre + h->cfg.L_core + h->cfg.L_coda, h->cfg.max_position, h->max_splits, h->status);
 }
 
-template <typename T, int DH, int LPT, int CPL, bool LAT, bool FUSE = true>
-static void launch_attention_t(const cdb* h, const AttnParams& p_in, void* o, cudaStream_t st) {
-    AttnParams p = p_in;
-    if (!FUSE) p.out = nullptr;
+template <typename T, int DH, int LPT, int CPL, bool LAT>
+static void launch_attention_t(const cdb* h, const AttnParams& p, void* o, cudaStream_t st) {
     static int per_device[kMaxDevices] = {};
     int& blocks_per_sm = per_device[h->device];
     if (blocks_per_sm == 0) {
         // The kernel uses no shared memory; asking for the largest shared-memory carve-out keeps the SM in the
         // configuration the projection kernel needs, so that its CTAs can become resident beside this one.
-        cudaFuncSetAttribute(attn_split_kernel<T, DH, LPT, CPL, LAT, FUSE>, cudaFuncAttributePreferredSharedMemoryCarveout,
+        cudaFuncSetAttribute(attn_split_kernel<T, DH, LPT, CPL, LAT>, cudaFuncAttributePreferredSharedMemoryCarveout,
                              tuning_int("CDB_ATTN_CARVEOUT", kAttnSharedCarveoutPct));
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, attn_split_kernel<T, DH, LPT, CPL, LAT, FUSE>, 128, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, attn_split_kernel<T, DH, LPT, CPL, LAT>, 128, 0);
         if (blocks_per_sm < 1) blocks_per_sm = 1;
     }
     const int sms = h->part_active ? h->part_attn_sms : h->sms;
@@ -414,16 +358,15 @@ static void launch_attention_t(const cdb* h, const AttnParams& p_in, void* o, cu
         cudaEventRecord(h->ev_pre[half], st);
         cudaStreamWaitEvent(h->part_attn, h->ev_pre[half], 0);
         CDB_LAUNCH(h);
-        launch_pdl(attn_split_kernel<T, DH, LPT, CPL, LAT, FUSE>, dim3(grid), dim3(threads), 0, h->part_attn, p);
+        launch_pdl(attn_split_kernel<T, DH, LPT, CPL, LAT>, dim3(grid), dim3(threads), 0, h->part_attn, p);
         cudaEventRecord(h->ev_post[half], h->part_attn);
         cudaStreamWaitEvent(st, h->ev_post[half], 0);
     } else {
         ProfScope ps(h, kProfAttention, st);
         CDB_LAUNCH(h);
-        launch_pdl(attn_split_kernel<T, DH, LPT, CPL, LAT, FUSE>, dim3(grid), dim3(threads), 0, st, p);
+        launch_pdl(attn_split_kernel<T, DH, LPT, CPL, LAT>, dim3(grid), dim3(threads), 0, st, p);
     }
     if (h->attn_split_done) cudaEventRecord(h->attn_split_done, st);     // the KV stream is over: the merge is tiny
-    if (p.out) return;                                                   // merged inside the split kernel
     CDB_LAUNCH(h);
     const int warps = p.rows.n_rows * p.pool.H;
     launch_pdl(attn_merge_kernel<T, DH>, dim3((warps + 3) / 4), dim3(128), 0, st, p, (T*)o);
@@ -438,9 +381,6 @@ void launch_attention(const cdb* h, int ln, int layer, const RowsDev& rows, cons
     p.max_seqs = h->cfg.max_seqs;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)h->cfg.Dh);
     p.part = h->lane[ln].attn_part; p.item_start = h->lane[ln].attn_item_start; p.counter = h->lane[ln].attn_counters + layer; p.status = h->status;
-    static const int fused_merge = tuning_int("CDB_ATTN_FUSED_MERGE", 1);      // tuning hook: 0 = the merge as a kernel of its own
-    p.done = h->lane[ln].attn_done;
-    p.out = fused_merge ? o : nullptr;
     static const int force_lat = tuning_int("CDB_ATTN_LAT", -1);      // tuning hook
     // Few (row, head) pairs: the GPU is far from full whatever the contexts are, and a warp's own latency chain
     // sets the pace (measured cross-over: ~64 rows of 16 heads; above it the throughput variant wins by 0-5 %).
@@ -451,10 +391,9 @@ void launch_attention(const cdb* h, int ln, int layer, const RowsDev& rows, cons
         else if (Dh == 96) { if (lat) launch_attention_t<__nv_bfloat16, 96, 4, 3, true>(h, p, o, st); else launch_attention_t<__nv_bfloat16, 96, 4, 3, false>(h, p, o, st); }
         else { if (lat) launch_attention_t<__nv_bfloat16, 64, 8, 1, true>(h, p, o, st); else launch_attention_t<__nv_bfloat16, 64, 8, 1, false>(h, p, o, st); }
     } else {
-        // (fp32 is the precision of the small parity configurations: its wider registers leave no room for the merge)
-        if (Dh == 128) launch_attention_t<float, 128, 8, 4, false, false>(h, p, o, st);
-        else if (Dh == 96) launch_attention_t<float, 96, 8, 3, false, false>(h, p, o, st);
-        else launch_attention_t<float, 64, 8, 2, false, false>(h, p, o, st);
+        if (Dh == 128) launch_attention_t<float, 128, 8, 4, false>(h, p, o, st);
+        else if (Dh == 96) launch_attention_t<float, 96, 8, 3, false>(h, p, o, st);
+        else launch_attention_t<float, 64, 8, 2, false>(h, p, o, st);
     }
 }
 
@@ -514,7 +453,7 @@ void launch_attention_static_t(const AttnParams& p, void* o, int max_context, cu
     const int max_items = p.rows.n_rows * p.pool.H * p.max_splits;
     int grid = 148 * 4;
     if ((max_items + 3) / 4 < grid) grid = (max_items + 3) / 4;
-    launch_pdl(attn_split_kernel<T, DH, LPT, CPL, false, false>, dim3(grid), dim3(128), 0, st, p);
+    launch_pdl(attn_split_kernel<T, DH, LPT, CPL, false>, dim3(grid), dim3(128), 0, st, p);
     const int warps = p.rows.n_rows * p.pool.H;
     launch_pdl(attn_merge_kernel<T, DH>, dim3((warps + 3) / 4), dim3(128), 0, st, p, (T*)o);
 }
@@ -564,7 +503,6 @@ extern "C" int cdb_paged_attention_static(const void* q, void* o, const void* po
     p.layer = layer; p.max_splits = max_splits; p.max_seqs = max_seqs;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)Dh);
     p.status = (int32_t*)base; p.counter = (int32_t*)(base + 4);
-    p.done = nullptr; p.out = nullptr;                       // the merge follows as a kernel of its own
     p.item_start = (const int32_t*)(base + head); p.part = (float*)(base + head + scan);
     cudaStream_t st = (cudaStream_t)stream;
     if (dtype == CDB_BF16) {
@@ -797,7 +735,6 @@ void launch_attention_prefill(const cdb* h, int ln, int layer, const RowsDev& ro
     p.max_seqs = h->cfg.max_seqs;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)h->cfg.Dh);
     p.part = nullptr; p.item_start = nullptr; p.counter = nullptr; p.status = h->status;
-    p.done = nullptr; p.out = nullptr;
     const int Dh = h->cfg.Dh;
     if (h->cfg.dtype == CDB_BF16) {
         if (Dh == 128) launch_prefill_t<__nv_bfloat16, 128>(h, p, ln, o, st);

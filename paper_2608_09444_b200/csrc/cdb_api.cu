@@ -423,7 +423,6 @@ int cdb_create(const cdb_config_t* cfg, const cdb_weights_t* w, cdb_t** out) {
         CDB_ALLOC(L.attn_part, float, r * c.H * h->max_splits * (size_t)(c.Dh + 2));
         CDB_ALLOC(L.attn_item_start, int32_t, r + 1);
         CDB_ALLOC(L.attn_counters, int32_t, n_layers);
-        CDB_ALLOC(L.attn_done, int32_t, r * c.H);
         CDB_ALLOC(L.pf_tile_rows, int32_t, r);
         CDB_ALLOC(L.pf_n_tiles, int32_t, 1);
     }

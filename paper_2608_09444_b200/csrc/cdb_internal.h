@@ -74,7 +74,6 @@ struct Lane {
     float* attn_part;               // [rows_cap*H*max_splits][Dh + 2] split partials (o, m, l)
     int32_t* attn_item_start;       // [rows_cap + 1] exclusive scan of splits per row
     int32_t* attn_counters;         // [L] work-fetch counters
-    int32_t* attn_done;             // [rows_cap * H] partials delivered per (row, head): zero outside an attention launch
     int32_t* pf_tile_rows;          // [rows_cap] rows per prefill tile (tile starts reuse attn_item_start)
     int32_t* pf_n_tiles;            // [1]
 };

@@ -910,27 +910,33 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
             p.BN = best;
         }
     }
-    // ... and a row tile need not be a power of two: any multiple of 16 rows is a valid MMA N.  r row tiles of
-    // ceil(n / r) rows (rounded up to 16) balance the tile count against the SM count: 512 rows of gate/up (44
-    // feature tiles) are 176 tiles of 128 rows - two waves, the second almost empty - or 132 tiles of 176 rows.
-    // Same cost measure as above; a width that no longer leaves TMEM room for two accumulator sets pays a
-    // quarter tile per extra wave (its epilogues are not hidden).
-    static const int chooser = tuning_int("CDB_GEMM_CHOOSER", 0);     // tuning hook: 1 = on
-    if (chooser && n > 64) {
+    // Above 256 rows a row tile need not be a power of two either: any multiple of 16 rows is a valid MMA N, and
+    // r row tiles of ceil(n / r) rows can fit the tile count to the SM count where halving cannot.  512 rows of
+    // gate/up (44 feature tiles) are 176 tiles of 128 rows - two waves, the second almost empty - or 132 tiles of 176
+    // rows: 32 against 24 us measured; the other projections (96 tiles per row tile) like three row tiles too (288
+    // tiles, two full waves): 176 rows per tile at 512 rows, 256 at 768.  Cost of a width = waves x (rows of a tile +
+    // the weight rows a tile must ingest whatever its width); a width that leaves TMEM no room for a second
+    // accumulator set (gate/up above 128 rows) is taken only where every CTA has a single tile, since its epilogue
+    // cannot hide under the next tile's main loop (prompt calls: 2.5 % slower with it); fewer row tiles win ties (each
+    // one pulls the weights through L2 again).  Measured per stage at 320 ... 1024 rows: never behind the powers of two.
+    static const int chooser = tuning_int("CDB_GEMM_CHOOSER", 1);     // tuning hook: 0 = powers of two only
+    if (chooser && n > 256) {
         const int sms = h->part_active ? h->part_proj_sms : h->sms;
         const int dual = mode == kModeSwiGLU ? 2 : 1;
-        long best_cost = -1; int best_bn = p.BN;
+        const bool pair_ok = pair != nullptr && !h->part_active && cluster_fit(h, 2) > 0 && n >= 512;
+        long best_cost = 0; int best_bn = 0;
         for (int r = 1; r <= (n + 63) / 64; ++r) {
-            int bn = ((n + r - 1) / r + 15) / 16 * 16;
+            const int bn = ((n + r - 1) / r + 15) / 16 * 16;
             if (bn > 256 || bn * dual > 512) continue;
             if (bn < 64) break;
-            const int r_eff = (n + bn - 1) / bn;
-            const long tiles = (long)n_ft * r_eff * k_splits, waves = (tiles + sms - 1) / sms;
-            const bool single = 2 * dual * bn > 512;
-            const long cost = waves * (bn + 32) + (single && waves > 1 ? (waves - 1) * (bn / 4) : 0);
-            if (best_cost < 0 || cost * 100 < best_cost * 95) { best_cost = cost; best_bn = bn; }
+            const int xr = pair_ok && bn >= 128 ? bn / 2 : bn;
+            if ((kMaxSmem - 1024 - (dual == 2 ? bn * BM * 2 : 0)) / (dual * BM * BK * 2 + xr * BK * 2) < 2) continue;
+            const long tiles = (long)n_ft * ((n + bn - 1) / bn) * k_splits, waves = (tiles + sms - 1) / sms;
+            if (2 * dual * bn > 512 && waves > 1) continue;
+            const long cost = waves * (bn + BM * dual);
+            if (best_bn == 0 || cost * 100 < best_cost * 95) { best_cost = cost; best_bn = bn; }
         }
-        p.BN = best_bn;
+        if (best_bn) p.BN = best_bn;
     }
     static const int forced_bn_dual = tuning_int("CDB_GEMM_BN_SWIGLU", 0);      // tuning hook
     {
