@@ -910,7 +910,7 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
             p.BN = best;
         }
     }
-    // Above 256 rows a row tile need not be a power of two either: any multiple of 16 rows is a valid MMA N, and
+    // Above 128 rows a row tile need not be a power of two either: any multiple of 16 rows is a valid MMA N, and
     // r row tiles of ceil(n / r) rows can fit the tile count to the SM count where halving cannot.  512 rows of
     // gate/up (44 feature tiles) are 176 tiles of 128 rows - two waves, the second almost empty - or 132 tiles of 176
     // rows: 32 against 24 us measured; the other projections (96 tiles per row tile) like three row tiles too (288
@@ -918,9 +918,11 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
     // the weight rows a tile must ingest whatever its width); a width that leaves TMEM no room for a second
     // accumulator set (gate/up above 128 rows) is taken only where every CTA has a single tile, since its epilogue
     // cannot hide under the next tile's main loop (prompt calls: 2.5 % slower with it); fewer row tiles win ties (each
-    // one pulls the weights through L2 again).  Measured per stage at 320 ... 1024 rows: never behind the powers of two.
+    // one pulls the weights through L2 again).  Measured per stage at 144 ... 1024 rows: never behind the powers of two
+    // (2-5 us per layer ahead up to 256 rows, where the rule mostly trims the padding of the last tile; 12-15 us at 448-512).
     static const int chooser = tuning_int("CDB_GEMM_CHOOSER", 1);     // tuning hook: 0 = powers of two only
-    if (chooser && n > 256) {
+    static const int chooser_min = tuning_int("CDB_GEMM_CHOOSER_MIN", 128);     // tuning hook
+    if (chooser && n > chooser_min) {
         const int sms = h->part_active ? h->part_proj_sms : h->sms;
         const int dual = mode == kModeSwiGLU ? 2 : 1;
         const bool pair_ok = pair != nullptr && !h->part_active && cluster_fit(h, 2) > 0 && n >= 512;
