@@ -218,15 +218,16 @@ def test_device_side_row_count_masks_the_tail_and_serves_one_graph_for_every_bat
 WIDE = synth.Dims(V=64, d=1024, H=8, Dh=128, F=2816, L_pre=0, L_core=2, L_coda=0, R=4, dtype="bf16")
 
 
-@pytest.mark.parametrize("n_rows", [9, 79, 209, 300])
+@pytest.mark.parametrize("n_rows", [9, 79, 209, 300, 530])
 def test_in_cluster_sums_equal_workspace_sums_and_do_not_depend_on_the_batch(n_rows):
     """A model wide enough for real split-K (4 parts for the QKV and output projections, 8 for the down projection).
     Default flow: the parts are summed inside thread-block clusters, with RoPE and the KV page write in the QKV
     projection's epilogue.  Cross-check flow (flag 32): the parts go through a workspace and row-wise kernels.
     Flags 64 and 96 repeat both flows with the projections of 128 rows and more run by CTA pairs (one MMA over two
     SMs that share the activation tile).  All of them add the same parts in the same order, so states, gate values, exit
-    signals and the K/V written must agree bit for bit - between the flows, and between a full batch (one to two
-    256-row tiles, ragged) and subsets.  Flag 128 runs batches of 64 rows and more as two half-batches with the SMs
+    signals and the K/V written must agree bit for bit - between the flows, and between a full batch and subsets.  The
+    batch sizes walk through the row-tile widths the projections choose (64 and 128 rows, then any multiple of 16:
+    112, 160 and 192-row tiles, ragged last tiles; at 530 rows CTA pairs by default).  Flag 128 runs batches of 64 rows and more as two half-batches with the SMs
     split between an attention and a projection partition (green contexts): the same numbers again."""
     ctxs = [1, 16, 17, 40, 255, 256, 257, 300, 33] + [int(c) for c in np.random.default_rng(2).integers(1, 90, n_rows - 9)]
     n = len(ctxs)
