@@ -162,6 +162,7 @@ def main():
     ap.add_argument("--contiguous-pages", action="store_true", help="ascending physical pages instead of a random permutation")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--simt-gemm", action="store_true", help="run projections on the plain-FMA cross-check kernel")
+    ap.add_argument("--cta-pairs", action="store_true", help="projections on 128 rows and more as CTA pairs (default: from 512 rows on)")
     ap.add_argument("--two-stream", action="store_true", help="split the step into two half-batches on two streams (experimental)")
     ap.add_argument("--workspace-parts", action="store_true", help="split-K parts through a workspace instead of in-cluster sums (cross-check flow)")
     ap.add_argument("--sm-partition", action="store_true", help="two half-batches with the SMs split between attention and projections (experimental)")
@@ -211,7 +212,7 @@ def main():
     from paper_2608_09444_b200 import binding as B
     from paper_2608_09444_b200.workloads import LoopStepWorkload
     wl = LoopStepWorkload(dims, n_rows=args.rows, seed=D.rank_seed(1, rank), ctx_lo=args.ctx_lo, ctx_hi=args.ctx_hi,
-                          permute=not args.contiguous_pages, device=f"cuda:{local_rank}", flags=(B.FLAG_SIMT_GEMM if args.simt_gemm else 0) | (B.FLAG_TWO_STREAM if args.two_stream else 0) | (B.FLAG_WORKSPACE_PARTS if args.workspace_parts else 0) | (B.FLAG_SM_PARTITION if args.sm_partition else 0))
+                          permute=not args.contiguous_pages, device=f"cuda:{local_rank}", flags=(B.FLAG_SIMT_GEMM if args.simt_gemm else 0) | (B.FLAG_TWO_STREAM if args.two_stream else 0) | (B.FLAG_WORKSPACE_PARTS if args.workspace_parts else 0) | (B.FLAG_SM_PARTITION if args.sm_partition else 0) | (B.FLAG_CTA_PAIRS if args.cta_pairs else 0))
     alg = wl.algorithmic()
     cores = len(os.sched_getaffinity(0))
 

@@ -925,7 +925,7 @@ static int setup_gemm(const cdb* h, const void* x, const void* W, const void* W2
     if (chooser && n > chooser_min) {
         const int sms = h->part_active ? h->part_proj_sms : h->sms;
         const int dual = mode == kModeSwiGLU ? 2 : 1;
-        const bool pair_ok = pair != nullptr && !h->part_active && cluster_fit(h, 2) > 0 && n >= 512;
+        const bool pair_ok = pair != nullptr && !h->part_active && cluster_fit(h, 2) > 0 && ((h->cfg.flags & CDB_FLAG_CTA_PAIRS) || n >= 512);
         long best_cost = 0; int best_bn = 0;
         for (int r = 1; r <= (n + 63) / 64; ++r) {
             const int bn = ((n + r - 1) / r + 15) / 16 * 16;
