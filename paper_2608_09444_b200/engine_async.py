@@ -30,6 +30,14 @@ from . import binding as B
 from .engine import Engine, _bucket, _static_rows
 
 
+def boundary_cost_in_steps(dims):
+    """Cost of one boundary pass (prelude and coda layers, LM head) in loop steps: twice the FLOP ratio, because small
+    steps are bound by latency rather than arithmetic.  ~0.16 for the Ouro shape (no boundary layers), ~2.4 for the
+    Huginn shape (2 + 2 boundary layers and a 65536-row LM head against a 4-layer core)."""
+    per_layer = 4 * dims.d * dims.d + 3 * dims.d * dims.F
+    return 2.0 * ((dims.L_pre + dims.L_coda) * per_layer + dims.V * dims.d) / (dims.L_core * per_layer)
+
+
 class PipelinedEngine(Engine):
     def __init__(self, *a, background_prefill=True, prefill_priority=0, eager_refill=True, **kw):
         kw.setdefault("mode", "refill")
@@ -53,9 +61,7 @@ class PipelinedEngine(Engine):
         # every step with free rows, Huginn-like ones (boundary as heavy as the core) never.  With a full batch
         # (more live sequences than rows) the boundary stages run beside step N as described above.
         self.eager_refill = eager_refill
-        dm = self.dims
-        per_layer = 4 * dm.d * dm.d + 3 * dm.d * dm.F
-        self.boundary_ratio = 2.0 * ((dm.L_pre + dm.L_coda) * per_layer + dm.V * dm.d) / (dm.L_core * per_layer)
+        self.boundary_ratio = boundary_cost_in_steps(self.dims)
         d = self.dims.d
         self.h_exit2 = [torch.zeros((self.max_rows, d), dtype=torch.float32, device=self.dev) for _ in range(2)]
         self.h_coda_in = torch.zeros((self.cap, d), dtype=torch.float32, device=self.dev)

@@ -65,3 +65,21 @@ def test_engines_reject_unknown_scheduling_modes_before_touching_the_gpu():
     from paper_2608_09444_b200.engine import Engine
     with pytest.raises(ValueError, match="unknown scheduling mode"):
         Engine(synth.TINY, None, max_batch=4, max_live=4, max_len=32, n_pages=8, mode="none")
+
+
+def test_flop_bound_and_the_early_rejoin_rule_on_the_two_model_shapes():
+    """Eq. 2 on the paper's shapes: F0 / Fr = 0.082 for the Ouro shape (LM head against one pass of the 24-layer core),
+    the bound is 1 at full depth and (F0 + R Fr) / (F0 + dbar Fr) below it.  The pipelined engine's rule for letting
+    tokens rejoin before the next step compares the rows that rejoin with the boundary cost in steps: cheap for the
+    Ouro shape, never worth it for the Huginn shape."""
+    from paper_2608_09444_b200 import synth
+    from paper_2608_09444_b200.engine_async import boundary_cost_in_steps
+    from paper_2608_09444_b200.offline import flop_bound
+    ouro, hug = synth.OURO_1P4B, synth.HUGINN_3P5B
+    f0 = ouro.V * ouro.d / (ouro.L_core * (4 * ouro.d ** 2 + 3 * ouro.d * ouro.F))
+    assert abs(f0 - 0.082) < 5e-4
+    assert flop_bound(ouro, ouro.R) == 1.0
+    assert abs(flop_bound(ouro, 2.5) - (f0 + 4) / (f0 + 2.5)) < 1e-12
+    assert abs(flop_bound(hug, 12.0) - 2.51) < 0.01
+    assert boundary_cost_in_steps(ouro) == 2 * f0 and boundary_cost_in_steps(ouro) < 0.2
+    assert boundary_cost_in_steps(hug) > 1.0
