@@ -65,7 +65,10 @@ class PipelinedEngine(Engine):
         d = self.dims.d
         self.h_exit2 = [torch.zeros((self.max_rows, d), dtype=torch.float32, device=self.dev) for _ in range(2)]
         self.h_coda_in = torch.zeros((self.cap, d), dtype=torch.float32, device=self.dev)
-        self.h_pre_out = torch.zeros((self.cap, d), dtype=torch.float32, device=self.dev)
+        # prelude outputs awaiting a batch row: a ring, each boundary call takes a contiguous run of rows (the prelude
+        # writes there directly, the refill gather reads by row index).  A sequence has at most one row in it, rows leave
+        # in the order they came, so four times the live set cannot wrap onto a row still waiting.
+        self.h_ready_ring = torch.zeros((4 * self.cap, d), dtype=torch.float32, device=self.dev)
         self.lists_host = torch.zeros((2 * self.max_rows + 2,), dtype=torch.int32).pin_memory()
         self.lists_dev = torch.zeros((2 * self.max_rows + 2,), dtype=torch.int32, device=self.dev)
         self.pgraphs = {}
@@ -125,7 +128,7 @@ class PipelinedEngine(Engine):
         waiting, live_slot = (list(range(n)) if arrivals is None else []), {}
         future = [] if arrivals is None else list(range(n))
         free_slots = list(range(self.max_live - 1, -1, -1))
-        ready, ready_free = [], list(range(self.cap - 1, -1, -1))     # (sid, slot in h_ready, event, iteration)
+        ready, ring_head = [], [0]                                    # (sid, row in h_ready_ring, event, iteration)
         coda_q, coda_free = [], list(range(self.cap - 1, -1, -1))     # (sid, depth, slot in h_coda)
         pending_tokens, pending_release = [], []
         ring = [torch.zeros((7, self.max_rows), dtype=torch.int32).pin_memory() for _ in range(4)]
@@ -198,19 +201,25 @@ class PipelinedEngine(Engine):
             are tok_t, or its entries `pick` (indices into it)."""
             sl = [live_slot[s] for s in sids]
             pos = [P[s] + gen[s] - 1 for s in sids]
-            slots = [ready_free.pop() for _ in sids]
-            sl_d, pos_d, slots_d, pick_d = staged(stream, sl, pos, slots, pick if pick is not None else [])
+            n_new = len(sids)
+            assert len(ready) + n_new <= self.cap
+            if ring_head[0] + n_new > self.h_ready_ring.shape[0]:
+                ring_head[0] = 0
+            first = ring_head[0]
+            ring_head[0] += n_new
+            if pick is not None and len(pick) == len(tok_t):
+                pick = None                             # everything goes on: no selection needed
+            sl_d, pos_d, pick_d = staged(stream, sl, pos, pick if pick is not None else [])
             if pick is not None:
                 tok_t = tok_t[pick_d.long()]
             rows = B.Rows(sl_d, pos_d, self.page_table)
-            out = self.h_pre_out[:len(sids)]
-            (cdb.boundary_prelude if dims.L_pre > 0 else cdb.boundary_embed)(tok_t, rows, out, stream=stream)
+            out = self.h_ready_ring[first:first + n_new]
             if gather_done is not None:
-                stream.wait_event(gather_done)          # a freed h_ready slot may still be read by the last refill gather
-            self.h_ready.index_copy_(0, slots_d.long(), out)
+                stream.wait_event(gather_done)          # rows of an earlier lap may still be read by the last refill gather
+            (cdb.boundary_prelude if dims.L_pre > 0 else cdb.boundary_embed)(tok_t, rows, out, stream=stream)
             ev = torch.cuda.Event()
             ev.record(stream)
-            ready.extend((s, slot, ev, it) for s, slot in zip(sids, slots))
+            ready.extend((s, first + j, ev, it) for j, s in enumerate(sids))
 
         prefill_inflight = []                           # at most one: (event, batch, pinned token buffer)
 
@@ -316,27 +325,38 @@ class PipelinedEngine(Engine):
                 if prev is not None and prev["ne"]:
                     side.wait_event(prev["G"])
                 with self._phase("boundary"):
-                    if prev is not None and prev["ne"]:
+                    # no minimum coda batch and nothing queued: the rows that left go to the coda where they are
+                    direct = prev is not None and prev["ne"] and self.min_coda_batch <= 1 and not coda_q
+                    if direct:
+                        items = [(s, r, None) for s, r in prev["exits"]]
+                    elif prev is not None and prev["ne"]:
                         slots = [coda_free.pop() for _ in range(prev["ne"])]
                         self.h_coda.index_copy_(0, staged(side, slots)[0].long(), self.h_exit2[prev["parity"]][:prev["ne"]])
                         ev = torch.cuda.Event()
                         ev.record(side)
                         x_done[prev["parity"]] = ev
                         coda_q.extend((s, r, slot) for (s, r), slot in zip(prev["exits"], slots))
-                    if not coda_q or (len(coda_q) < self.min_coda_batch and not force):
-                        return
-                    items = list(coda_q)
-                    coda_q.clear()
+                    if not direct:
+                        if not coda_q or (len(coda_q) < self.min_coda_batch and not force):
+                            return
+                        items = list(coda_q)
+                        coda_q.clear()
                     m = len(items)
-                    hin = self.h_coda_in[:m]
                     sids = [it_[0] for it_ in items]
-                    from_d, sl_d, pos_d, depth_d = staged(side, [it_[2] for it_ in items], [live_slot[s] for s in sids],
+                    from_d, sl_d, pos_d, depth_d = staged(side, [] if direct else [it_[2] for it_ in items], [live_slot[s] for s in sids],
                                                           [P[s] + gen[s] - 1 for s in sids], [it_[1] for it_ in items])
-                    cdb.gather_rows(self.h_coda, from_d, None, m, hin, stream=side)
+                    if direct:
+                        hin = self.h_exit2[prev["parity"]][:m]
+                    else:
+                        hin = self.h_coda_in[:m]
+                        cdb.gather_rows(self.h_coda, from_d, None, m, hin, stream=side)
                     rows = B.Rows(sl_d, pos_d, self.page_table)
                     if self.kv_layout == B.KV_DEPTH_INDEXED:
                         cdb.kv_copy_on_exit(rows, depth_d, stream=side)
                     cdb.boundary_coda_lmhead(rows, hin, tok_dev[:m], stream=side)
+                    if direct:                          # the exit buffer of this parity has been consumed
+                        x_done[prev["parity"]] = torch.cuda.Event()
+                        x_done[prev["parity"]].record(side)
                     buf = tok_ring[tok_calls % len(tok_ring)][:m]
                     tok_calls += 1
                     buf.copy_(tok_dev[:m], non_blocking=True)
@@ -346,7 +366,8 @@ class PipelinedEngine(Engine):
                     self.stats["coda_calls"] += 1
                     cont = []
                     for j, (s, r, slot) in enumerate(items):
-                        coda_free.append(slot)
+                        if slot is not None:
+                            coda_free.append(slot)
                         gen[s] += 1
                         if gen[s] >= Ts[s]:
                             pending_release.append((ev, s))
@@ -386,8 +407,7 @@ class PipelinedEngine(Engine):
             while ready and len(rec) + len(take) < self.max_batch and ready[0][3] < it:
                 take.append(ready.pop(0))
             n_keep = len(rec)
-            for s, slot, _, _ in take:
-                ready_free.append(slot)                     # (a reuse of the slot waits for this step's gather: gather_done)
+            for s, _, _, _ in take:
                 rec.append([s, 1])
             k = len(rec)
             step = None
@@ -411,7 +431,7 @@ class PipelinedEngine(Engine):
                         for _, _, ev, _ in take:
                             if ev is not None:
                                 main.wait_event(ev)
-                        cdb.gather_rows(self.h_ready, self.desc_dev[6, :len(take)], None, len(take), self.h_rec[n_keep:n_keep + len(take)])
+                        cdb.gather_rows(self.h_ready_ring, self.desc_dev[6, :len(take)], None, len(take), self.h_rec[n_keep:n_keep + len(take)])
                         gather_done = torch.cuda.Event()
                         gather_done.record(main)
                     g, rows = self.pgraphs[(nb, parity)]
