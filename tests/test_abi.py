@@ -83,3 +83,28 @@ def test_flop_bound_and_the_early_rejoin_rule_on_the_two_model_shapes():
     assert abs(flop_bound(hug, 12.0) - 2.51) < 0.01
     assert boundary_cost_in_steps(ouro) == 2 * f0 and boundary_cost_in_steps(ouro) < 0.2
     assert boundary_cost_in_steps(hug) > 1.0
+
+
+def test_reference_arm_of_the_bench_runs_on_the_host_alone_and_prints_the_contract_line():
+    """`bench.py --impl reference` times the CPU oracle on a bounded sample and needs neither a GPU nor the library: its
+    process must not load libcdb.so, and its single JSON line carries the keys the benchmark contract names."""
+    import json
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = ("import runpy, sys; sys.argv = ['bench.py', '--impl', 'reference', '--steps', '1', '--warmup', '0', '--layers', '1'];\n"
+            "try:\n    runpy.run_path('bench.py', run_name='__main__')\nexcept SystemExit:\n    pass\n"
+            "print('LIBCDB_LOADED' if 'libcdb' in open('/proc/self/maps').read() else 'LIBCDB_ABSENT')")
+    out = subprocess.run([sys.executable, "-c", code], cwd=root, capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.strip()]
+    assert lines[-1] == "LIBCDB_ABSENT"
+    line = json.loads(lines[-2])
+    for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+                "vs_baseline", "dtype", "data", "config", "cpu_baseline", "e2e"):
+        assert key in line, key
+    assert line["impl"] == "reference" and line["metric"] == "token_loop_steps_per_s" and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["value"] == line["value"]
+    assert line["e2e"]["value"] == line["value"] and line["e2e"]["h2d_bytes_per_step"] == 0
+    assert "workload" in line["config"] and "model" not in line["config"]
